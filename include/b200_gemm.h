@@ -1,0 +1,138 @@
+/*
+ * b200_gemm.h — C ABI of the B200 (sm_100a) GEMM library.
+ *
+ * The library computes the operation the paper's BLIS-style algorithm computes (Section II-A:
+ * C = C + A B through loops L1-L5, Pack-A / Pack-B and the mr x nr micro-kernel, Fig. 1), with
+ * the alpha / beta scaling of the micro-kernel of Fig. 3 folded in:
+ *
+ *        C  <-  alpha * op(A) * op(B) + beta * C
+ *
+ * in BLAS column-major convention: element (i, j) of a stored matrix X is X[i + j*ldx].
+ * Every matrix pointer is a DEVICE pointer unless a function says otherwise; scalars are passed
+ * by value from the host.  No function throws, aborts or prints.
+ */
+#ifndef B200_GEMM_H
+#define B200_GEMM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* element types of A and B; C is always fp32 */
+typedef enum {
+    GEMM_F32  = 0,  /* A, B fp32; exact IEEE fp32 fused multiply-add arithmetic on the CUDA cores          */
+    GEMM_F16  = 1,  /* A, B IEEE binary16; products accumulated in fp32 on the tensor cores (tcgen05/TMEM) */
+    GEMM_BF16 = 2   /* A, B bfloat16;      products accumulated in fp32 on the tensor cores                 */
+} gemm_dtype_t;
+
+/* return codes (0 = success; -1 .. -15 = the 1-based position of the first invalid argument of gemm()) */
+enum {
+    GEMM_OK            = 0,
+    GEMM_ERR_WORKSPACE = -100,  /* a forced configuration needs more workspace than is registered      */
+    GEMM_ERR_LAUNCH    = -101,  /* the CUDA runtime refused a launch; see gemm_last_cuda_error()        */
+    GEMM_ERR_ARCH      = -102,  /* the current device is not compute capability 10.x                    */
+    GEMM_ERR_DEVICE    = -103,  /* a bounded device-side wait expired (reported by gemm_poll_status())  */
+    GEMM_ERR_TOO_LARGE = -104   /* a size exceeds what an entry point supports                          */
+};
+
+/* kernel families, as reported by gemm_last_config() and accepted by gemm_force_kernel() */
+enum {
+    GEMM_KERNEL_AUTO         = 0,
+    GEMM_KERNEL_SIMT_GENERIC = 1,  /* any dtype, any alignment: bounds-checked scalar loads, fp32 FMA          */
+    GEMM_KERNEL_SIMT_FAST    = 2,  /* fp32: register-blocked 8x8 FFMA micro-tiles, shared-memory double buffer */
+    GEMM_KERNEL_TENSOR       = 3,  /* fp16/bf16: TMA -> swizzled shared memory -> tcgen05.mma -> TMEM          */
+    GEMM_KERNEL_SCALE_ONLY   = 6   /* C <- beta*C (alpha == 0 or k == 0)                                        */
+};
+
+typedef struct {
+    int32_t kernel;        /* one of GEMM_KERNEL_*                                           */
+    int32_t tile_m;        /* CTA tile rows of C                                             */
+    int32_t tile_n;        /* CTA tile columns of C                                          */
+    int32_t tile_k;        /* k extent of one pipeline stage                                 */
+    int32_t split_k;       /* number of k partitions (1 = none)                              */
+    int32_t stages;        /* pipeline depth                                                 */
+    int32_t grid;          /* CTAs launched for the main kernel                              */
+    int32_t vector_a;      /* elements per global load of A (SIMT paths) / 1 if TMA operand  */
+    int32_t vector_b;
+    int32_t launches;      /* kernels enqueued by the call (main + reduction / scaling)      */
+    int32_t repacked;      /* bit 0: A was copied to an aligned layout first, bit 1: B       */
+    int32_t reserved;
+} gemm_config_t;
+
+/*
+ * gemm — the whole hot path: tile selection, the loops over n, m and k (Fig. 1, L1-L5), operand
+ * staging into on-chip memory (the role of Pack-A / Pack-B), the rank-k update (micro-kernel, L6)
+ * and the alpha / beta epilogue of Fig. 3 fused into the store of C.
+ *
+ *   dtype          gemm_dtype_t
+ *   transA/transB  'N'/'n': op(X) = X;  'T'/'t'/'C'/'c': op(X) = X^T (real data)
+ *   m, n, k        op(A) is m x k, op(B) is k x n, C is m x n; all >= 0
+ *   A, lda         device pointer; stored m x k (lda >= max(1,m)) if transA = N, else k x m (lda >= max(1,k));
+ *                  elements of `dtype`; never written
+ *   B, ldb         device pointer; stored k x n (ldb >= max(1,k)) if transB = N, else n x k (ldb >= max(1,n))
+ *   C, ldc         device pointer to fp32, m x n, ldc >= max(1,m); read only if beta != 0 (so NaN/Inf in C
+ *                  do not propagate when beta == 0); rows m..ldc-1 of every column are never touched
+ *   alpha, beta    fp32 scalars by value
+ *   stream         cudaStream_t (NULL = the default stream)
+ *
+ * Any natural alignment of A, B, C and any legal leading dimension is accepted; 16-byte aligned pointers
+ * with lda, ldb multiples of 16 bytes take the fast paths.  The call is asynchronous: work is enqueued on
+ * `stream` and the buffers must stay valid until the stream has passed it.  C must not overlap A or B.
+ * Quick returns: m == 0 or n == 0 does nothing; alpha == 0 or k == 0 computes C <- beta*C (beta == 0
+ * stores +0 without reading C, beta == 1 does nothing), and A, B may then be NULL.
+ * Returns GEMM_OK, or -(position of the first invalid argument) with nothing launched and C untouched,
+ * or one of the GEMM_ERR_* codes.
+ */
+int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k,
+         float alpha, const void* A, int64_t lda, const void* B, int64_t ldb,
+         float beta, void* C, int64_t ldc, void* stream);
+
+/*
+ * gemm_host — the same operation on HOST buffers (pageable or pinned): allocates device buffers
+ * from the stream-ordered pool, copies A, B (and C if beta != 0) to the device, runs gemm(), copies
+ * C back and synchronises `stream` before returning.  Leading dimensions and layout as for gemm().
+ */
+int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k,
+              float alpha, const void* A_host, int64_t lda, const void* B_host, int64_t ldb,
+              float beta, void* C_host, int64_t ldc, void* stream);
+
+/*
+ * Workspace (device memory, caller-owned).  Split-k configurations keep fp32 partial sums there, and
+ * operands whose leading dimension TMA cannot address are first copied there in an aligned layout
+ * (the counterpart of the paper's packing buffers Ac / Bc).  Without a workspace, or with one that is
+ * too small, gemm() silently picks a configuration that needs none.
+ *   gemm_workspace_bytes  bytes the selector would like for this problem (0 = none)
+ *   gemm_set_workspace    registers `dev` (>= 256-byte aligned) of `bytes` bytes for the current device;
+ *                         dev == NULL unregisters.  One workspace per device: calls that use it must be
+ *                         ordered on one stream.  `stream` is unused (reserved) and may be NULL.
+ */
+size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k);
+int gemm_set_workspace(void* dev, size_t bytes, void* stream);
+
+/* configuration chosen by the most recent gemm() of the calling thread (for tests and reports) */
+int gemm_last_config(gemm_config_t* out);
+
+/* tests / benchmarks: force a kernel family (GEMM_KERNEL_AUTO restores the selector).  A forced family
+ * that cannot run the problem (wrong dtype, alignment) falls back to the selector's choice.
+ * gemm_force_tile: force tile_n (0 = auto) and split_k (0 = auto) of the chosen family. */
+int gemm_force_kernel(int kernel);
+int gemm_force_tile(int tile_m, int tile_n, int split_k);
+
+/*
+ * Device status.  Every wait inside the kernels (on an mbarrier) is bounded; a wait that expires
+ * records a code in a device status word, the CTA drains and exits normally.  gemm_poll_status()
+ * synchronises the device, returns GEMM_OK or GEMM_ERR_DEVICE and clears the word;
+ * gemm_status_detail() returns the raw word of the last poll (role and barrier that gave up).
+ */
+int gemm_poll_status(void);
+uint32_t gemm_status_detail(void);
+const char* gemm_status_string(int code);
+int gemm_last_cuda_error(void);   /* cudaError_t of the last failed launch, 0 if none */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B200_GEMM_H */

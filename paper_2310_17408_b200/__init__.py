@@ -1,0 +1,9 @@
+"""B200 (sm_100a) GEMM library: C <- alpha*op(A)*op(B) + beta*C, BLAS column-major.
+
+The product is the CUDA shared library built from csrc/ (C ABI in include/b200_gemm.h); this
+package is its thin Python binding.  Importing it without the built library raises ImportError.
+"""
+from .binding import *  # noqa: F401,F403
+from .binding import (GemmConfig, EXPORTS, library_path, gemm, gemm_host, gemm_workspace_bytes,  # noqa: F401
+                      gemm_set_workspace, gemm_last_config, gemm_force_kernel, gemm_force_tile,
+                      gemm_poll_status, gemm_status_detail, gemm_status_string, gemm_last_cuda_error)

@@ -1,0 +1,123 @@
+"""ctypes binding of libb200gemm.so: the same names and argument order as include/b200_gemm.h.
+
+Argument marshalling only.  Pointers are plain integers (torch `tensor.data_ptr()`, numpy
+`array.ctypes.data`); `stream` is a cudaStream_t as an integer (`torch.cuda.current_stream().cuda_stream`).
+There is no fallback: importing this module without the built CUDA library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_LIB_PATH = Path(__file__).resolve().parent / "libb200gemm.so"
+
+GEMM_F32, GEMM_F16, GEMM_BF16 = 0, 1, 2
+GEMM_OK = 0
+GEMM_ERR_WORKSPACE, GEMM_ERR_LAUNCH, GEMM_ERR_ARCH, GEMM_ERR_DEVICE, GEMM_ERR_TOO_LARGE = -100, -101, -102, -103, -104
+GEMM_KERNEL_AUTO, GEMM_KERNEL_SIMT_GENERIC, GEMM_KERNEL_SIMT_FAST, GEMM_KERNEL_TENSOR = 0, 1, 2, 3
+GEMM_KERNEL_SCALE_ONLY = 6
+
+EXPORTS = ("gemm", "gemm_host", "gemm_workspace_bytes", "gemm_set_workspace", "gemm_last_config",
+           "gemm_force_kernel", "gemm_force_tile", "gemm_poll_status", "gemm_status_detail",
+           "gemm_status_string", "gemm_last_cuda_error")
+
+
+class GemmConfig(ctypes.Structure):
+    _fields_ = [(name, ctypes.c_int32) for name in
+                ("kernel", "tile_m", "tile_n", "tile_k", "split_k", "stages", "grid", "vector_a", "vector_b",
+                 "launches", "repacked", "reserved")]
+
+    def as_dict(self):
+        return {name: getattr(self, name) for name, _ in self._fields_ if name != "reserved"}
+
+
+def _load() -> ctypes.CDLL:
+    if not _LIB_PATH.exists():
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2310_17408_b200.build` "
+                          "(nvcc, sm_100a); this package has no CPU or library fallback")
+    lib = ctypes.CDLL(str(_LIB_PATH), mode=ctypes.RTLD_LOCAL)
+    i64, vp, ci, cf, cc = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_char
+    sig = [ci, cc, cc, i64, i64, i64, cf, vp, i64, vp, i64, cf, vp, i64, vp]
+    lib.gemm.restype = ci
+    lib.gemm.argtypes = sig
+    lib.gemm_host.restype = ci
+    lib.gemm_host.argtypes = sig
+    lib.gemm_workspace_bytes.restype = ctypes.c_size_t
+    lib.gemm_workspace_bytes.argtypes = [ci, cc, cc, i64, i64, i64]
+    lib.gemm_set_workspace.restype = ci
+    lib.gemm_set_workspace.argtypes = [vp, ctypes.c_size_t, vp]
+    lib.gemm_last_config.restype = ci
+    lib.gemm_last_config.argtypes = [ctypes.POINTER(GemmConfig)]
+    lib.gemm_force_kernel.restype = ci
+    lib.gemm_force_kernel.argtypes = [ci]
+    lib.gemm_force_tile.restype = ci
+    lib.gemm_force_tile.argtypes = [ci, ci, ci]
+    lib.gemm_poll_status.restype = ci
+    lib.gemm_poll_status.argtypes = []
+    lib.gemm_status_detail.restype = ctypes.c_uint32
+    lib.gemm_status_detail.argtypes = []
+    lib.gemm_status_string.restype = ctypes.c_char_p
+    lib.gemm_status_string.argtypes = [ci]
+    lib.gemm_last_cuda_error.restype = ci
+    lib.gemm_last_cuda_error.argtypes = []
+    return lib
+
+
+_lib = _load()
+
+
+def library_path() -> str:
+    return str(_LIB_PATH)
+
+
+def _c(flag) -> bytes:
+    b = flag.encode() if isinstance(flag, str) else bytes(flag)
+    if len(b) != 1:
+        raise ValueError("trans flag must be one character")
+    return b
+
+
+def gemm(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, stream=0) -> int:
+    return _lib.gemm(dtype, _c(transA), _c(transB), m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, stream)
+
+
+def gemm_host(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, stream=0) -> int:
+    return _lib.gemm_host(dtype, _c(transA), _c(transB), m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, stream)
+
+
+def gemm_workspace_bytes(dtype, transA, transB, m, n, k) -> int:
+    return int(_lib.gemm_workspace_bytes(dtype, _c(transA), _c(transB), m, n, k))
+
+
+def gemm_set_workspace(dev_ptr, nbytes, stream=0) -> int:
+    return _lib.gemm_set_workspace(dev_ptr, nbytes, stream)
+
+
+def gemm_last_config() -> dict:
+    cfg = GemmConfig()
+    _lib.gemm_last_config(ctypes.byref(cfg))
+    return cfg.as_dict()
+
+
+def gemm_force_kernel(kernel) -> int:
+    return _lib.gemm_force_kernel(kernel)
+
+
+def gemm_force_tile(tile_m, tile_n, split_k) -> int:
+    return _lib.gemm_force_tile(tile_m, tile_n, split_k)
+
+
+def gemm_poll_status() -> int:
+    return _lib.gemm_poll_status()
+
+
+def gemm_status_detail() -> int:
+    return int(_lib.gemm_status_detail())
+
+
+def gemm_status_string(code) -> str:
+    return _lib.gemm_status_string(code).decode()
+
+
+def gemm_last_cuda_error() -> int:
+    return _lib.gemm_last_cuda_error()

@@ -1,0 +1,439 @@
+// C ABI of the GEMM library: argument validation, quick returns, the shape selector (tile shape, split-k,
+// fast-path eligibility — the role the paper gives to choosing the (mr, nr) micro-kernel and the cache
+// parameters per problem, Sections I and IV) and dispatch to the kernels.
+#include <mutex>
+#include <new>
+
+#include "internal.cuh"
+
+namespace b200gemm {
+
+__device__ uint32_t g_device_status;   // written by bounded waits that expire
+
+constexpr int MAX_DEVICES = 64;
+
+struct DeviceState {
+    bool init = false;
+    bool arch_ok = false;
+    int sms = 0;
+    uint32_t* status = nullptr;
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+};
+
+static DeviceState g_dev[MAX_DEVICES];
+static std::mutex g_mutex;
+static thread_local gemm_config_t t_last_cfg = {};
+static thread_local int t_last_cuda_error = 0;
+static int g_force_kernel = GEMM_KERNEL_AUTO;
+static int g_force_tile_m = 0, g_force_tile_n = 0, g_force_split = 0;
+static uint32_t g_last_detail = 0;
+
+static DeviceState* device_state() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& s = g_dev[dev];
+    if (!s.init) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return nullptr;
+        s.arch_ok = (prop.major == 10);
+        s.sms = prop.multiProcessorCount;
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        s.status = static_cast<uint32_t*>(p);
+        s.init = true;
+    }
+    return &s;
+}
+
+int sm_count() {
+    DeviceState* s = device_state();
+    return (s && s->sms > 0) ? s->sms : 148;
+}
+
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+
+// ---------------------------------------------------------------- selector
+
+struct Plan {
+    int kernel;        // GEMM_KERNEL_*
+    int tile;          // SIMT fast: tile id 0..3; tensor: tile_n
+    KSplit ks;
+    bool repack_a, repack_b;
+    int64_t lda_p, ldb_p;     // leading dimensions of the repacked operands
+    size_t ws_partials;       // bytes
+    size_t ws_total;
+};
+
+// k partition: `want` splits of a multiple of `quantum`, no empty split
+static KSplit make_split(int64_t k, int want, int quantum) {
+    KSplit ks{1, round_up(k > 0 ? k : 1, quantum)};
+    if (want <= 1) return ks;
+    int64_t chunk = round_up(ceil_div(k, want), quantum);
+    int splits = (int)ceil_div(k, chunk);
+    if (splits <= 1) return ks;
+    ks.splits = splits;
+    ks.chunk = chunk;
+    return ks;
+}
+
+static const int kSimtTileM[4] = {128, 128, 64, 64};
+static const int kSimtTileN[4] = {128, 64, 128, 64};
+
+// fp32: pick the CTA tile that fills the SMs best, then split k when the tile count is far below one wave
+static void plan_simt(const GemmArgs& a, int sms, size_t ws_avail, Plan* p) {
+    p->kernel = GEMM_KERNEL_SIMT_FAST;
+    const double ctas_per_sm[4] = {2, 3, 3, 6};
+    const double eff[4] = {1.0, 0.92, 0.92, 0.80};     // relative math efficiency of the smaller tiles
+    int best = 0;
+    double best_score = -1;
+    for (int t = 0; t < 4; ++t) {
+        if (g_force_tile_m && g_force_tile_n && (kSimtTileM[t] != g_force_tile_m || kSimtTileN[t] != g_force_tile_n)) continue;
+        const int64_t tm = ceil_div(a.m, kSimtTileM[t]), tn = ceil_div(a.n, kSimtTileN[t]);
+        const double tiles = (double)tm * tn;
+        const double slots = sms * ctas_per_sm[t];
+        const double waves = tiles / slots;
+        const double full = (double)ceil_div((int64_t)tiles, (int64_t)slots);
+        const double util = waves / full;                                           // tail effect
+        const double useful = ((double)a.m * a.n) / (tiles * kSimtTileM[t] * kSimtTileN[t]);   // edge waste
+        const double score = util * useful * eff[t];
+        if (score > best_score) { best_score = score; best = t; }
+    }
+    p->tile = best;
+    const int64_t tiles = ceil_div(a.m, kSimtTileM[best]) * ceil_div(a.n, kSimtTileN[best]);
+    const int64_t slots = (int64_t)(sms * ctas_per_sm[best]);
+    int want = 1;
+    if (g_force_split > 0) want = g_force_split;
+    else if (tiles * 2 <= slots && a.k >= 512) {
+        want = (int)(slots / tiles);
+        const int64_t max_by_k = a.k / 256;             // keep at least 256 of k per split
+        if (want > max_by_k) want = (int)max_by_k;
+        if (want > 64) want = 64;
+    }
+    p->ks = make_split(a.k, want, 16);
+    p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
+    if (p->ws_partials > ws_avail) {
+        if (g_force_split > 0) { p->kernel = -1; return; }
+        p->ks = make_split(a.k, 1, 16);
+        p->ws_partials = 0;
+    }
+    p->ws_total = p->ws_partials;
+}
+
+static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, bool b_ok, Plan* p) {
+    p->kernel = GEMM_KERNEL_TENSOR;
+    p->repack_a = !a_ok;
+    p->repack_b = !b_ok;
+    const int64_t a_rows = a.ta ? a.k : a.m, a_cols = a.ta ? a.m : a.k;
+    const int64_t b_rows = a.tb ? a.n : a.k, b_cols = a.tb ? a.k : a.n;
+    p->lda_p = round_up(a_rows > 0 ? a_rows : 1, 8);
+    p->ldb_p = round_up(b_rows > 0 ? b_rows : 1, 8);
+    size_t ws_repack = 0;
+    if (p->repack_a) ws_repack += (size_t)round_up(p->lda_p * a_cols * 2, 256);
+    if (p->repack_b) ws_repack += (size_t)round_up(p->ldb_p * b_cols * 2, 256);
+    if (ws_repack > ws_avail) { p->kernel = GEMM_KERNEL_SIMT_GENERIC; return; }
+
+    // tile_n: the widest tile that still gives every SM work; narrower tiles when the tile count is small
+    int bn = 256;
+    if (g_force_tile_n == 64 || g_force_tile_n == 128 || g_force_tile_n == 256) bn = g_force_tile_n;
+    else {
+        const int64_t tm = ceil_div(a.m, 128);
+        if (tm * ceil_div(a.n, 256) < sms) bn = 128;
+        if (tm * ceil_div(a.n, 128) < sms) bn = 64;
+        if (a.n <= 64) bn = 64;
+        else if (a.n <= 128 && bn > 128) bn = 128;
+    }
+    p->tile = bn;
+    const int64_t tiles = ceil_div(a.m, 128) * ceil_div(a.n, bn);
+    int want = 1;
+    if (g_force_split > 0) want = g_force_split;
+    else if (tiles * 2 <= sms && a.k >= 1024) {
+        want = (int)(sms / tiles);
+        const int64_t max_by_k = a.k / 512;
+        if (want > max_by_k) want = (int)max_by_k;
+        if (want > 32) want = 32;
+    }
+    p->ks = make_split(a.k, want, 64);
+    p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
+    if (ws_repack + p->ws_partials > ws_avail) {
+        if (g_force_split > 0) { p->kernel = -1; return; }
+        p->ks = make_split(a.k, 1, 64);
+        p->ws_partials = 0;
+    }
+    p->ws_total = ws_repack + p->ws_partials;
+}
+
+static Plan make_plan(const GemmArgs& a, int sms, size_t ws_avail) {
+    Plan p{};
+    p.ks = KSplit{1, a.k > 0 ? a.k : 1};
+    int forced = g_force_kernel;
+    if (forced == GEMM_KERNEL_SIMT_GENERIC) { p.kernel = GEMM_KERNEL_SIMT_GENERIC; return p; }
+    if (a.dtype == GEMM_F32) {
+        plan_simt(a, sms, ws_avail, &p);
+        return p;
+    }
+    // 16-bit inputs: tensor path if the operands are (or can be made) addressable by TMA
+    auto aligned = [](const void* ptr, int64_t ld) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0 && ld % 8 == 0; };
+    GemmArgs probe = a;
+    const bool a_ok = aligned(a.A, a.lda), b_ok = aligned(a.B, a.ldb);
+    if (!a_ok) { probe.A = nullptr; probe.lda = 8; }      // judged on the repacked layout
+    if (!b_ok) { probe.B = nullptr; probe.ldb = 8; }
+    if (!tensor_eligible(probe)) { p.kernel = GEMM_KERNEL_SIMT_GENERIC; return p; }
+    plan_tensor(a, sms, ws_avail, a_ok, b_ok, &p);
+    return p;
+}
+
+// ---------------------------------------------------------------- validation
+
+static int validate(int dtype, char ta, char tb, int64_t m, int64_t n, int64_t k, float alpha, const void* A,
+                    int64_t lda, const void* B, int64_t ldb, const void* C, int64_t ldc, bool* tA, bool* tB) {
+    auto tr = [](char c, bool* t) {
+        switch (c) {
+            case 'N': case 'n': *t = false; return true;
+            case 'T': case 't': case 'C': case 'c': *t = true; return true;
+            default: return false;
+        }
+    };
+    if (dtype != GEMM_F32 && dtype != GEMM_F16 && dtype != GEMM_BF16) return -1;
+    if (!tr(ta, tA)) return -2;
+    if (!tr(tb, tB)) return -3;
+    if (m < 0) return -4;
+    if (n < 0) return -5;
+    if (k < 0) return -6;
+    const int64_t a_rows = *tA ? k : m, b_rows = *tB ? n : k;
+    const bool needs_ab = m > 0 && n > 0 && k > 0 && alpha != 0.0f;
+    const int es = elem_size(dtype);
+    if (needs_ab && A == nullptr) return -8;
+    if (A != nullptr && (reinterpret_cast<uintptr_t>(A) % es) != 0) return -8;
+    if (lda < (a_rows > 1 ? a_rows : 1)) return -9;
+    if (needs_ab && B == nullptr) return -10;
+    if (B != nullptr && (reinterpret_cast<uintptr_t>(B) % es) != 0) return -10;
+    if (ldb < (b_rows > 1 ? b_rows : 1)) return -11;
+    if (m > 0 && n > 0 && C == nullptr) return -13;
+    if (C != nullptr && (reinterpret_cast<uintptr_t>(C) % 4) != 0) return -13;
+    if (ldc < (m > 1 ? m : 1)) return -14;
+    return 0;
+}
+
+static int fail_launch(cudaError_t e) {
+    t_last_cuda_error = (int)e;
+    return GEMM_ERR_LAUNCH;
+}
+
+static int run_gemm(const GemmArgs& a0, DeviceState* st) {
+    GemmArgs a = a0;
+    gemm_config_t cfg{};
+    cfg.split_k = 1;
+    cfg.launches = 1;
+    cudaError_t e;
+
+    if (a.alpha == 0.0f || a.k == 0) {
+        cfg.kernel = GEMM_KERNEL_SCALE_ONLY;
+        if (a.beta == 1.0f) { cfg.launches = 0; t_last_cfg = cfg; return GEMM_OK; }
+        e = launch_scale(a);
+        t_last_cfg = cfg;
+        return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+    }
+
+    void* ws;
+    size_t ws_bytes;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        ws = st->ws;
+        ws_bytes = st->ws_bytes;
+    }
+    Plan p = make_plan(a, st->sms, ws_bytes);
+    if (p.kernel < 0) return GEMM_ERR_WORKSPACE;
+
+    if (p.kernel == GEMM_KERNEL_SIMT_GENERIC) {
+        e = launch_simt_generic(a, &cfg);
+        t_last_cfg = cfg;
+        return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+    }
+
+    uint8_t* wsp = static_cast<uint8_t*>(ws);
+    if (p.kernel == GEMM_KERNEL_TENSOR) {
+        if (p.repack_a) {
+            const int64_t rows = a.ta ? a.k : a.m, cols = a.ta ? a.m : a.k;
+            e = launch_repack16(a.A, rows, cols, a.lda, wsp, p.lda_p, a.stream);
+            if (e != cudaSuccess) return fail_launch(e);
+            a.A = wsp; a.lda = p.lda_p;
+            wsp += round_up(p.lda_p * cols * 2, 256);
+            cfg.repacked |= 1; cfg.launches++;
+        }
+        if (p.repack_b) {
+            const int64_t rows = a.tb ? a.n : a.k, cols = a.tb ? a.k : a.n;
+            e = launch_repack16(a.B, rows, cols, a.ldb, wsp, p.ldb_p, a.stream);
+            if (e != cudaSuccess) return fail_launch(e);
+            a.B = wsp; a.ldb = p.ldb_p;
+            wsp += round_up(p.ldb_p * cols * 2, 256);
+            cfg.repacked |= 2; cfg.launches++;
+        }
+    }
+    float* partials = p.ks.splits > 1 ? reinterpret_cast<float*>(wsp) : nullptr;
+    if (p.kernel == GEMM_KERNEL_TENSOR) e = launch_tensor(a, p.tile, p.ks, partials, &cfg);
+    else e = launch_simt_fast(a, p.tile, p.ks, partials, &cfg);
+    if (e == cudaSuccess && p.ks.splits > 1) {
+        e = launch_splitk_reduce(a, p.ks.splits, partials);
+        cfg.launches++;
+    }
+    t_last_cfg = cfg;
+    return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+}
+
+}  // namespace b200gemm
+
+using namespace b200gemm;
+
+extern "C" {
+
+int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha, const void* A, int64_t lda,
+         const void* B, int64_t ldb, float beta, void* C, int64_t ldc, void* stream) {
+    bool ta = false, tb = false;
+    int bad = validate(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, C, ldc, &ta, &tb);
+    if (bad) return bad;
+    if (m == 0 || n == 0) {
+        gemm_config_t cfg{};
+        cfg.kernel = GEMM_KERNEL_SCALE_ONLY;
+        t_last_cfg = cfg;
+        return GEMM_OK;
+    }
+    DeviceState* st = device_state();
+    if (!st) return GEMM_ERR_LAUNCH;
+    if (!st->arch_ok) return GEMM_ERR_ARCH;
+    GemmArgs a{dtype, ta, tb, m, n, k, alpha, beta, A, B, static_cast<float*>(C), lda, ldb, ldc,
+               static_cast<cudaStream_t>(stream), st->status};
+    return run_gemm(a, st);
+}
+
+int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha, const void* A_host,
+              int64_t lda, const void* B_host, int64_t ldb, float beta, void* C_host, int64_t ldc, void* stream) {
+    bool ta = false, tb = false;
+    int bad = validate(dtype, transA, transB, m, n, k, alpha, A_host, lda, B_host, ldb, C_host, ldc, &ta, &tb);
+    if (bad) return bad;
+    if (m == 0 || n == 0) return GEMM_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int es = elem_size(dtype);
+    const bool needs_ab = (k > 0 && alpha != 0.0f);
+    const size_t a_bytes = needs_ab ? (size_t)lda * (ta ? m : k) * es : 0;
+    const size_t b_bytes = needs_ab ? (size_t)ldb * (tb ? k : n) * es : 0;
+    const size_t c_bytes = (size_t)ldc * n * sizeof(float);
+    void *dA = nullptr, *dB = nullptr, *dC = nullptr;
+    cudaError_t e = cudaSuccess;
+    int rc = GEMM_OK;
+    auto chk = [&](cudaError_t r) { if (e == cudaSuccess && r != cudaSuccess) e = r; return r == cudaSuccess; };
+    if (a_bytes) chk(cudaMallocAsync(&dA, a_bytes, s));
+    if (b_bytes) chk(cudaMallocAsync(&dB, b_bytes, s));
+    chk(cudaMallocAsync(&dC, c_bytes, s));
+    if (e == cudaSuccess) {
+        if (a_bytes) chk(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, s));
+        if (b_bytes) chk(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, s));
+        // C travels whole (padding rows included) so that the copy back leaves the host padding as it was
+        chk(cudaMemcpyAsync(dC, C_host, c_bytes, cudaMemcpyHostToDevice, s));
+    }
+    if (e == cudaSuccess)
+        rc = gemm(dtype, transA, transB, m, n, k, alpha, dA, lda, dB, ldb, beta, dC, ldc, stream);
+    if (e == cudaSuccess && rc == GEMM_OK) chk(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, s));
+    if (dA) cudaFreeAsync(dA, s);
+    if (dB) cudaFreeAsync(dB, s);
+    if (dC) cudaFreeAsync(dC, s);
+    chk(cudaStreamSynchronize(s));
+    if (e != cudaSuccess) return fail_launch(e);
+    return rc;
+}
+
+size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k) {
+    bool ta = false, tb = false;
+    const int64_t big = (int64_t)1 << 40;
+    if (validate(dtype, transA, transB, m, n, k, 1.0f, (const void*)16, big, (const void*)16, big, (const void*)16, big, &ta, &tb))
+        return 0;
+    if (m == 0 || n == 0 || k == 0) return 0;
+    DeviceState* st = device_state();
+    const int sms = st ? st->sms : 148;
+    // judged for 16-byte aligned pointers and minimal leading dimensions (lda = rows of the stored A, ...)
+    GemmArgs a{dtype, ta, tb, m, n, k, 1.0f, 0.0f, (const void*)16, (const void*)16, nullptr,
+               ta ? k : m, tb ? n : k, m, nullptr, nullptr};
+    Plan p = make_plan(a, sms, ~(size_t)0);
+    return p.kernel < 0 ? 0 : p.ws_total;
+}
+
+int gemm_set_workspace(void* dev, size_t bytes, void* /*stream*/) {
+    DeviceState* st = device_state();
+    if (!st) return GEMM_ERR_LAUNCH;
+    if (dev != nullptr && (reinterpret_cast<uintptr_t>(dev) & 255) != 0) return -1;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    st->ws = dev;
+    st->ws_bytes = dev ? bytes : 0;
+    return GEMM_OK;
+}
+
+int gemm_last_config(gemm_config_t* out) {
+    if (!out) return -1;
+    *out = t_last_cfg;
+    return GEMM_OK;
+}
+
+int gemm_force_kernel(int kernel) {
+    if (kernel != GEMM_KERNEL_AUTO && kernel != GEMM_KERNEL_SIMT_GENERIC && kernel != GEMM_KERNEL_SIMT_FAST &&
+        kernel != GEMM_KERNEL_TENSOR)
+        return -1;
+    g_force_kernel = kernel;
+    return GEMM_OK;
+}
+
+int gemm_force_tile(int tile_m, int tile_n, int split_k) {
+    if (tile_m < 0 || tile_n < 0 || split_k < 0) return -1;
+    g_force_tile_m = tile_m;
+    g_force_tile_n = tile_n;
+    g_force_split = split_k;
+    return GEMM_OK;
+}
+
+int gemm_poll_status(void) {
+    DeviceState* st = device_state();
+    if (!st) return GEMM_ERR_LAUNCH;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail_launch(e);
+    uint32_t word = 0;
+    e = cudaMemcpy(&word, st->status, sizeof(word), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_launch(e);
+    g_last_detail = word;
+    if (word != 0) {
+        uint32_t zero = 0;
+        cudaMemcpy(st->status, &zero, sizeof(zero), cudaMemcpyHostToDevice);
+        return GEMM_ERR_DEVICE;
+    }
+    return GEMM_OK;
+}
+
+uint32_t gemm_status_detail(void) { return g_last_detail; }
+
+int gemm_last_cuda_error(void) { return t_last_cuda_error; }
+
+const char* gemm_status_string(int code) {
+    switch (code) {
+        case GEMM_OK: return "success";
+        case GEMM_ERR_WORKSPACE: return "forced configuration needs more workspace than is registered";
+        case GEMM_ERR_LAUNCH: return "CUDA runtime error (see gemm_last_cuda_error)";
+        case GEMM_ERR_ARCH: return "device is not compute capability 10.x";
+        case GEMM_ERR_DEVICE: return "a bounded device-side wait expired";
+        case GEMM_ERR_TOO_LARGE: return "size exceeds what this entry point supports";
+        case -1: return "invalid argument 1 (dtype)";
+        case -2: return "invalid argument 2 (transA)";
+        case -3: return "invalid argument 3 (transB)";
+        case -4: return "invalid argument 4 (m)";
+        case -5: return "invalid argument 5 (n)";
+        case -6: return "invalid argument 6 (k)";
+        case -8: return "invalid argument 8 (A)";
+        case -9: return "invalid argument 9 (lda)";
+        case -10: return "invalid argument 10 (B)";
+        case -11: return "invalid argument 11 (ldb)";
+        case -13: return "invalid argument 13 (C)";
+        case -14: return "invalid argument 14 (ldc)";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

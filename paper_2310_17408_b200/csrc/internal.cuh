@@ -1,0 +1,60 @@
+// Internal interfaces between the translation units of the GEMM library (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/b200_gemm.h"
+
+namespace b200gemm {
+
+struct GemmArgs {
+    int dtype;
+    bool ta, tb;           // op(X) = X^T ?
+    int64_t m, n, k;
+    float alpha, beta;
+    const void* A;
+    const void* B;
+    float* C;
+    int64_t lda, ldb, ldc;
+    cudaStream_t stream;
+    uint32_t* status;      // device status word (bounded waits report here)
+};
+
+// k partition used by every split-k path: split s covers [s*chunk, min(k, (s+1)*chunk))
+struct KSplit {
+    int splits;
+    int64_t chunk;
+};
+
+// device status word layout: bits 31..24 = 0xE5 marker, 23..16 = role, 15..8 = barrier id, 7..0 = stage
+constexpr uint32_t STATUS_MARK = 0xE5000000u;
+
+inline int elem_size(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }
+
+// C <- beta*C  (beta == 0: store +0 without reading)
+cudaError_t launch_scale(const GemmArgs& a);
+
+// generic bounds-checked SIMT kernel, any dtype / trans / alignment
+cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg);
+
+// fast fp32 SIMT kernel.  tile: 0 = 128x128, 1 = 128x64, 2 = 64x128, 3 = 64x64.
+// ks.splits > 1: raw partial sums go to `partials` ([split][n][m], fp32), no epilogue.
+bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb);
+cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg);
+
+// C <- alpha * sum_s partials[s] + beta*C, summed in increasing s (deterministic)
+cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* partials);
+
+// tcgen05 tensor-core kernel (fp16 / bf16).  tile_n in {64, 128, 256}; tile_m is 128.
+bool tensor_eligible(const GemmArgs& a);
+cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg);
+
+// copy op-independent stored matrix (rows x cols, ld) of 16-bit elements into an aligned layout (ld_out)
+cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,
+                            cudaStream_t stream);
+
+int sm_count();
+
+}  // namespace b200gemm

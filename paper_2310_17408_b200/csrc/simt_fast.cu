@@ -1,0 +1,287 @@
+// Fast fp32 GEMM on the CUDA cores (exact IEEE fp32 FMA).
+//
+// Mapping of the paper's algorithm (Fig. 1) onto the SM:
+//   loops L1/L3 (jc, ic)   -> grid of BM x BN CTA tiles of C, visited in groups of tile rows so that the CTAs
+//                             resident at one time share their A and B panels in L2
+//   loop  L2 (pc, kc)      -> the CTA's loop over BK = 16 slices of k (optionally a k range per CTA: split-k)
+//   Pack-A / Pack-B        -> 128-bit global loads into registers, stored to a double-buffered shared-memory
+//                             stage laid out [k][m] and [k][n] so that a thread's fragment is one 128-bit read
+//   loops L4/L5 + L6       -> each warp owns a 64 x 32 sub-tile, each thread an 8 x 8 register block that
+//                             receives one outer product per k (the role of the mr x nr micro-kernel)
+//   alpha / beta (Fig. 3)  -> applied once, when the register block is stored
+#include "internal.cuh"
+
+namespace b200gemm {
+
+constexpr int BK = 16;
+constexpr int PAD = 4;   // row padding of the shared-memory stage (floats); keeps rows 16-byte aligned
+
+// ---- global -> register loader for one operand tile of X_TILE (m or n extent) x BK
+// KCONT: the stored matrix is contiguous along k (A with transA = T, B with transB = N);
+// otherwise it is contiguous along the tile dimension.  VEC: elements per load (4 needs 16-byte alignment).
+template <int X_TILE, int NT, bool KCONT, int VEC>
+struct Loader {
+    static constexpr int ELEMS = X_TILE * BK / NT;   // per thread
+    static constexpr int NV = ELEMS / VEC;           // loads per thread
+    static_assert(ELEMS % VEC == 0 && ELEMS >= VEC, "tile / thread count mismatch");
+
+    // coordinates (x, kk) of load v of thread t; a VEC=4 load covers 4 consecutive elements of the contiguous dim
+    __device__ static __forceinline__ void coord(int t, int v, int& x, int& kk) {
+        if (KCONT) {
+            constexpr int KV = BK / VEC;             // loads along k per row
+            kk = (t % KV) * VEC;
+            x = t / KV + v * (NT / KV);
+        } else {
+            constexpr int XV = X_TILE / VEC;
+            x = (t % XV) * VEC;
+            kk = t / XV + v * (NT / XV);
+        }
+    }
+
+    template <bool GUARD>
+    __device__ static __forceinline__ void load(float (&r)[ELEMS], const float* __restrict__ X, int64_t ld,
+                                                int64_t x0, int64_t k0, int64_t xmax, int64_t kmax, int t) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            int x, kk;
+            coord(t, v, x, kk);
+            int64_t gx = x0 + x, gk = k0 + kk;
+            const float* p = KCONT ? X + gk + gx * ld : X + gx + gk * ld;
+            if (VEC == 4) {
+                bool whole = !GUARD || (KCONT ? (gx < xmax && gk + 3 < kmax) : (gx + 3 < xmax && gk < kmax));
+                if (whole) {
+                    float4 q = __ldg(reinterpret_cast<const float4*>(p));
+                    r[v * 4 + 0] = q.x; r[v * 4 + 1] = q.y; r[v * 4 + 2] = q.z; r[v * 4 + 3] = q.w;
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        bool ok = KCONT ? (gx < xmax && gk + c < kmax) : (gx + c < xmax && gk < kmax);
+                        r[v * 4 + c] = ok ? __ldg(p + c) : 0.0f;
+                    }
+                }
+            } else {
+                bool ok = !GUARD || (gx < xmax && gk < kmax);
+                r[v] = ok ? __ldg(p) : 0.0f;
+            }
+        }
+    }
+
+    // registers -> shared stage S[kk][x] (row length X_TILE + PAD)
+    __device__ static __forceinline__ void store(const float (&r)[ELEMS], float* S, int t) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            int x, kk;
+            coord(t, v, x, kk);
+            if (VEC == 4) {
+                if (KCONT) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) S[(kk + c) * (X_TILE + PAD) + x] = r[v * 4 + c];
+                } else {
+                    *reinterpret_cast<float4*>(S + kk * (X_TILE + PAD) + x) =
+                        make_float4(r[v * 4 + 0], r[v * 4 + 1], r[v * 4 + 2], r[v * 4 + 3]);
+                }
+            } else {
+                S[kk * (X_TILE + PAD) + x] = r[v];
+            }
+        }
+    }
+};
+
+// one BK slice of outer products on the thread's 8 x 8 register block
+template <int BM, int BN>
+__device__ __forceinline__ void compute_stage(float (&acc)[8][8], const float* __restrict__ As,
+                                              const float* __restrict__ Bs, int am, int bn) {
+    float a[2][8], b[2][8];
+    auto frag = [&](int kk, int buf) {
+        const float* ap = As + kk * (BM + PAD) + am;
+        const float* bp = Bs + kk * (BN + PAD) + bn;
+        float4 a0 = *reinterpret_cast<const float4*>(ap);
+        float4 a1 = *reinterpret_cast<const float4*>(ap + 32);
+        float4 b0 = *reinterpret_cast<const float4*>(bp);
+        float4 b1 = *reinterpret_cast<const float4*>(bp + 16);
+        a[buf][0] = a0.x; a[buf][1] = a0.y; a[buf][2] = a0.z; a[buf][3] = a0.w;
+        a[buf][4] = a1.x; a[buf][5] = a1.y; a[buf][6] = a1.z; a[buf][7] = a1.w;
+        b[buf][0] = b0.x; b[buf][1] = b0.y; b[buf][2] = b0.z; b[buf][3] = b0.w;
+        b[buf][4] = b1.x; b[buf][5] = b1.y; b[buf][6] = b1.z; b[buf][7] = b1.w;
+    };
+    frag(0, 0);
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+        if (kk + 1 < BK) frag(kk + 1, (kk + 1) & 1);
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(a[kk & 1][i], b[kk & 1][j], acc[j][i]);
+    }
+}
+
+template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB>
+__global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
+simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
+                 const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
+                 int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials) {
+    constexpr int NT = WARPS_M * WARPS_N * 32;
+    static_assert(BM == WARPS_M * 64 && BN == WARPS_N * 32, "warp tile is 64 x 32");
+    using LA = Loader<BM, NT, A_KCONT, VA>;
+    using LB = Loader<BN, NT, B_KCONT, VB>;
+
+    __shared__ __align__(16) float As[2][BK * (BM + PAD)];
+    __shared__ __align__(16) float Bs[2][BK * (BN + PAD)];
+
+    const int t = threadIdx.x;
+    const int warp = t >> 5, lane = t & 31;
+    const int wm = warp % WARPS_M, wn = warp / WARPS_M;
+    const int lm = lane & 7, ln = lane >> 3;          // 8 lanes along m, 4 along n
+    const int am = wm * 64 + lm * 4;                  // thread rows: am..am+3 and am+32..am+35
+    const int bn = wn * 32 + ln * 4;                  // thread cols: bn..bn+3 and bn+16..bn+19
+
+    // grouped tile order: GROUP tile rows at a time, all tile columns inside a group
+    constexpr int GROUP = 16;
+    const int tile = blockIdx.x;
+    const int per_group = GROUP * tiles_n;
+    const int g = tile / per_group;
+    const int gsz = min(GROUP, tiles_m - g * GROUP);
+    const int tm = g * GROUP + (tile % per_group) % gsz;
+    const int tn = (tile % per_group) / gsz;
+    const int64_t i0 = (int64_t)tm * BM, j0 = (int64_t)tn * BN;
+
+    const int64_t kbeg = (int64_t)blockIdx.z * kchunk;
+    const int64_t kend = min(k, kbeg + kchunk);
+    const int64_t ktiles = (kend - kbeg + BK - 1) / BK;
+
+    float acc[8][8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[j][i] = 0.0f;
+
+    float ra[LA::ELEMS], rb[LB::ELEMS];
+    const bool interior = (i0 + BM <= m) && (j0 + BN <= n);
+
+    auto gload = [&](int64_t kt) {
+        const int64_t k0 = kbeg + kt * BK;
+        if (interior && k0 + BK <= kend) {
+            LA::template load<false>(ra, A, lda, i0, k0, m, kend, t);
+            LB::template load<false>(rb, B, ldb, j0, k0, n, kend, t);
+        } else {
+            LA::template load<true>(ra, A, lda, i0, k0, m, kend, t);
+            LB::template load<true>(rb, B, ldb, j0, k0, n, kend, t);
+        }
+    };
+
+    if (ktiles > 0) {
+        gload(0);
+        LA::store(ra, As[0], t);
+        LB::store(rb, Bs[0], t);
+        __syncthreads();
+        for (int64_t kt = 0; kt < ktiles; ++kt) {
+            const int cur = (int)(kt & 1);
+            if (kt + 1 < ktiles) gload(kt + 1);                 // in flight during the math below
+            compute_stage<BM, BN>(acc, As[cur], Bs[cur], am, bn);
+            if (kt + 1 < ktiles) {
+                LA::store(ra, As[cur ^ 1], t);
+                LB::store(rb, Bs[cur ^ 1], t);
+            }
+            __syncthreads();
+        }
+    }
+
+    // ---- store: alpha*acc + beta*C, or raw partial sums for split-k
+    const bool raw = partials != nullptr;
+    float* out = raw ? partials + (int64_t)blockIdx.z * m * n : C;
+    const int64_t ldo = raw ? m : ldc;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(out) & 15) == 0) && (ldo % 4 == 0);
+#pragma unroll
+    for (int jh = 0; jh < 2; ++jh)
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const int64_t gj = j0 + bn + jh * 16 + jj;
+            if (gj >= n) continue;
+#pragma unroll
+            for (int ih = 0; ih < 2; ++ih) {
+                const int64_t gi = i0 + am + ih * 32;
+                float* c = out + gi + gj * ldo;
+                const float* v = &acc[jh * 4 + jj][ih * 4];
+                if (vec_ok && gi + 3 < m) {
+                    float4 r;
+                    if (raw) {
+                        r = make_float4(v[0], v[1], v[2], v[3]);
+                    } else {
+                        r = make_float4(alpha * v[0], alpha * v[1], alpha * v[2], alpha * v[3]);
+                        if (beta != 0.0f) {
+                            float4 c0 = *reinterpret_cast<const float4*>(c);
+                            r.x = fmaf(beta, c0.x, r.x); r.y = fmaf(beta, c0.y, r.y);
+                            r.z = fmaf(beta, c0.z, r.z); r.w = fmaf(beta, c0.w, r.w);
+                        }
+                    }
+                    *reinterpret_cast<float4*>(c) = r;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (gi + e < m) {
+                            float r = raw ? v[e] : alpha * v[e];
+                            if (!raw && beta != 0.0f) r = fmaf(beta, c[e], r);
+                            c[e] = r;
+                        }
+                }
+            }
+        }
+}
+
+// ---------------------------------------------------------------- host side
+
+bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb) {
+    if (a.dtype != GEMM_F32) return false;
+    auto vec = [](const void* p, int64_t ld) { return ((reinterpret_cast<uintptr_t>(p) & 15) == 0 && ld % 4 == 0) ? 4 : 1; };
+    *va = vec(a.A, a.lda);
+    *vb = vec(a.B, a.ldb);
+    return true;
+}
+
+template <int BM, int BN, int WM, int WN, int MINB, bool AK, bool BKC, int VA, int VB>
+static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg) {
+    int64_t tiles_m = (a.m + BM - 1) / BM, tiles_n = (a.n + BN - 1) / BN;
+    if (tiles_m * tiles_n > 0x7FFFFFFFLL || tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF)
+        return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)(tiles_m * tiles_n), 1, (unsigned)ks.splits);
+    cfg->tile_m = BM; cfg->tile_n = BN; cfg->tile_k = BK; cfg->stages = 2;
+    cfg->grid = (int32_t)(tiles_m * tiles_n * ks.splits);
+    simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB><<<grid, WM * WN * 32, 0, a.stream>>>(
+        a.m, a.n, a.k, a.alpha, (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
+        (int)tiles_m, (int)tiles_n, ks.chunk, ks.splits > 1 ? partials : nullptr);
+    return cudaGetLastError();
+}
+
+template <bool AK, bool BKC, int VA, int VB>
+static cudaError_t launch_tile(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg) {
+    switch (tile) {
+        case 0: return launch_one<128, 128, 2, 4, 2, AK, BKC, VA, VB>(a, ks, partials, cfg);
+        case 1: return launch_one<128, 64, 2, 2, 3, AK, BKC, VA, VB>(a, ks, partials, cfg);
+        case 2: return launch_one<64, 128, 1, 4, 3, AK, BKC, VA, VB>(a, ks, partials, cfg);
+        default: return launch_one<64, 64, 1, 2, 6, AK, BKC, VA, VB>(a, ks, partials, cfg);
+    }
+}
+
+template <bool AK, bool BKC>
+static cudaError_t launch_vec(const GemmArgs& a, int va, int vb, int tile, KSplit ks, float* partials,
+                              gemm_config_t* cfg) {
+    if (va == 4 && vb == 4) return launch_tile<AK, BKC, 4, 4>(a, tile, ks, partials, cfg);
+    if (va == 4) return launch_tile<AK, BKC, 4, 1>(a, tile, ks, partials, cfg);
+    if (vb == 4) return launch_tile<AK, BKC, 1, 4>(a, tile, ks, partials, cfg);
+    return launch_tile<AK, BKC, 1, 1>(a, tile, ks, partials, cfg);
+}
+
+cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg) {
+    int va, vb;
+    simt_fast_eligible(a, &va, &vb);
+    cfg->kernel = GEMM_KERNEL_SIMT_FAST;
+    cfg->split_k = ks.splits;
+    cfg->vector_a = va; cfg->vector_b = vb;
+    // A is contiguous along k when transposed; B is contiguous along k when not transposed
+    if (!a.ta && !a.tb) return launch_vec<false, true>(a, va, vb, tile, ks, partials, cfg);
+    if (a.ta && !a.tb) return launch_vec<true, true>(a, va, vb, tile, ks, partials, cfg);
+    if (!a.ta && a.tb) return launch_vec<false, false>(a, va, vb, tile, ks, partials, cfg);
+    return launch_vec<true, false>(a, va, vb, tile, ks, partials, cfg);
+}
+
+}  // namespace b200gemm

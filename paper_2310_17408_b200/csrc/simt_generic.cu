@@ -1,0 +1,183 @@
+// Generic SIMT GEMM (any dtype, transpose flag, alignment and leading dimension), the C <- beta*C
+// kernel and the split-k reduction.  These are the correctness anchors: every load and store is
+// bounds-checked and scalar.
+#include "internal.cuh"
+
+namespace b200gemm {
+
+template <typename T> __device__ __forceinline__ float to_float(T v);
+template <> __device__ __forceinline__ float to_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_float<__half>(__half v) { return __half2float(v); }
+template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Epilogue of Fig. 3 in BLAS form: alpha*acc + beta*C0, C0 untouched when beta == 0.
+__device__ __forceinline__ float epilogue(float alpha, float acc, float beta, const float* c) {
+    float r = alpha * acc;
+    if (beta != 0.0f) r = fmaf(beta, *c, r);
+    return r;
+}
+
+constexpr int GT = 64;   // CTA tile (GT x GT) of C
+constexpr int GK = 16;   // k extent of one shared-memory stage
+
+// 256 threads; thread (tx, ty) owns the 4x4 entries (tx + 16 i, ty + 16 j) of the tile.
+template <typename T, bool TA, bool TB>
+__global__ void __launch_bounds__(256)
+simt_generic_kernel(int64_t m, int64_t n, int64_t k, float alpha, const T* __restrict__ A, int64_t lda,
+                    const T* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
+                    int64_t tiles_m) {
+    __shared__ float As[GK][GT + 1];
+    __shared__ float Bs[GK][GT + 1];
+    const int t = threadIdx.x;
+    const int tx = t & 15, ty = t >> 4;
+    const int64_t tile = blockIdx.x;
+    const int64_t i0 = (tile % tiles_m) * GT, j0 = (tile / tiles_m) * GT;
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+
+    for (int64_t k0 = 0; k0 < k; k0 += GK) {
+#pragma unroll
+        for (int e = 0; e < (GT * GK) / 256; ++e) {
+            int idx = t + e * 256;
+            // A: walk the contiguous dimension of the stored matrix with consecutive threads
+            int mm = TA ? idx / GK : idx % GT;
+            int kk = TA ? idx % GK : idx / GT;
+            int64_t gi = i0 + mm, gk = k0 + kk;
+            float v = 0.0f;
+            if (gi < m && gk < k) v = to_float<T>(TA ? A[gk + gi * lda] : A[gi + gk * lda]);
+            As[kk][mm] = v;
+            int nn = TB ? idx % GT : idx / GK;
+            int kb = TB ? idx / GT : idx % GK;
+            int64_t gj = j0 + nn;
+            gk = k0 + kb;
+            v = 0.0f;
+            if (gj < n && gk < k) v = to_float<T>(TB ? B[gj + gk * ldb] : B[gk + gj * ldb]);
+            Bs[kb][nn] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < GK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][tx + 16 * i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Bs[kk][ty + 16 * j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        int64_t gj = j0 + ty + 16 * j;
+        if (gj >= n) continue;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int64_t gi = i0 + tx + 16 * i;
+            if (gi < m) {
+                float* c = C + gi + gj * ldc;
+                *c = epilogue(alpha, acc[i][j], beta, c);
+            }
+        }
+    }
+}
+
+template <typename T>
+static cudaError_t launch_generic_t(const GemmArgs& a) {
+    int64_t tiles_m = (a.m + GT - 1) / GT, tiles_n = (a.n + GT - 1) / GT;
+    int64_t tiles = tiles_m * tiles_n;
+    if (tiles > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)tiles), block(256);
+    const T* A = (const T*)a.A;
+    const T* B = (const T*)a.B;
+#define LAUNCH(TA_, TB_)                                                                              \
+    simt_generic_kernel<T, TA_, TB_><<<grid, block, 0, a.stream>>>(a.m, a.n, a.k, a.alpha, A, a.lda, B, \
+                                                                   a.ldb, a.beta, a.C, a.ldc, tiles_m)
+    if (!a.ta && !a.tb) LAUNCH(false, false);
+    else if (a.ta && !a.tb) LAUNCH(true, false);
+    else if (!a.ta && a.tb) LAUNCH(false, true);
+    else LAUNCH(true, true);
+#undef LAUNCH
+    return cudaGetLastError();
+}
+
+cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg) {
+    cfg->kernel = GEMM_KERNEL_SIMT_GENERIC;
+    cfg->tile_m = GT; cfg->tile_n = GT; cfg->tile_k = GK; cfg->split_k = 1; cfg->stages = 1;
+    cfg->grid = (int32_t)(((a.m + GT - 1) / GT) * ((a.n + GT - 1) / GT));
+    cfg->vector_a = cfg->vector_b = 1;
+    cfg->launches = 1;
+    if (a.dtype == GEMM_F32) return launch_generic_t<float>(a);
+    if (a.dtype == GEMM_F16) return launch_generic_t<__half>(a);
+    return launch_generic_t<__nv_bfloat16>(a);
+}
+
+// ---------------------------------------------------------------- C <- beta*C
+
+__global__ void __launch_bounds__(256)
+scale_kernel(int64_t m, int64_t n, float beta, float* __restrict__ C, int64_t ldc) {
+    for (int64_t j = blockIdx.y; j < n; j += gridDim.y)
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (int64_t)gridDim.x * blockDim.x) {
+            float* c = C + i + j * ldc;
+            *c = (beta == 0.0f) ? 0.0f : beta * *c;
+        }
+}
+
+cudaError_t launch_scale(const GemmArgs& a) {
+    unsigned gx = (unsigned)((a.m + 255) / 256 > 1024 ? 1024 : (a.m + 255) / 256);
+    unsigned gy = (unsigned)(a.n > 32768 ? 32768 : a.n);
+    scale_kernel<<<dim3(gx, gy), 256, 0, a.stream>>>(a.m, a.n, a.beta, a.C, a.ldc);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- split-k reduction + epilogue
+
+// partials: [split][n][m] fp32 (leading dimension m).  Summed in increasing split index.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(int64_t m, int64_t n, int splits, const float* __restrict__ partials, float alpha, float beta,
+                     float* __restrict__ C, int64_t ldc) {
+    const int64_t total = m * n;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        float s = partials[idx];
+        for (int z = 1; z < splits; ++z) s += partials[idx + (int64_t)z * total];
+        int64_t i = idx % m, j = idx / m;
+        float* c = C + i + j * ldc;
+        *c = epilogue(alpha, s, beta, c);
+    }
+}
+
+cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* partials) {
+    int64_t total = a.m * a.n;
+    int64_t blocks = (total + 255) / 256;
+    int64_t cap = (int64_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- 16-bit operand repack (aligned leading dimension)
+
+__global__ void __launch_bounds__(256)
+repack16_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld, uint16_t* __restrict__ dst,
+                int64_t ld_out) {
+    for (int64_t j = blockIdx.y; j < cols; j += gridDim.y)
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < ld_out; i += (int64_t)gridDim.x * blockDim.x)
+            dst[i + j * ld_out] = (i < rows) ? src[i + j * ld] : (uint16_t)0;
+}
+
+cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,
+                            cudaStream_t stream) {
+    unsigned gx = (unsigned)((ld_out + 255) / 256 > 256 ? 256 : (ld_out + 255) / 256);
+    unsigned gy = (unsigned)(cols > 32768 ? 32768 : cols);
+    repack16_kernel<<<dim3(gx, gy), 256, 0, stream>>>((const uint16_t*)src, rows, cols, ld, (uint16_t*)dst, ld_out);
+    return cudaGetLastError();
+}
+
+}  // namespace b200gemm

@@ -1,0 +1,425 @@
+// fp16 / bf16 GEMM with fp32 accumulation on the 5th-generation tensor cores (tcgen05, sm_100a).
+//
+// Mapping of the paper's algorithm (Fig. 1) onto the SM:
+//   loops L1/L3 (jc, ic)   -> persistent CTAs walk a list of 128 x BN tiles of C (grouped so that resident CTAs
+//                             share operand panels in L2)
+//   loop  L2 (pc, kc)      -> 64-wide k blocks streamed through a multi-stage shared-memory ring
+//   Pack-A / Pack-B        -> TMA copies global -> 128-byte-swizzled shared memory; the swizzled stage IS the
+//                             packed panel, and TMA's zero fill past the matrix edge is the panel padding
+//   loops L4/L5 + L6       -> tcgen05.mma 128 x BN x 16, issued by one thread; the C block lives in tensor
+//                             memory (TMEM) for the whole k loop, as the paper's C block lives in registers
+//   alpha / beta (Fig. 3)  -> epilogue warps read TMEM (tcgen05.ld), scale, and store column-major C
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2..5 = epilogue (one TMEM lane
+// quarter each).  Two accumulators in TMEM let the epilogue of one tile overlap the main loop of the next.
+// Every mbarrier wait is bounded: on expiry the role records a code in the status word and all roles drain.
+#include <cuda.h>
+
+#include "internal.cuh"
+
+namespace b200gemm {
+
+constexpr int TBM = 128;            // MMA M (TMEM lanes)
+constexpr int TBK = 64;             // k block: 64 x 2 bytes = one 128-byte swizzle row
+constexpr int UMMA_K = 16;          // k extent of one tcgen05.mma for 16-bit inputs
+constexpr uint32_t SPIN_FAST = 4096;
+constexpr uint32_t SPIN_LIMIT = 1u << 24;   // then ~128 ns sleeps: gives up after a few seconds
+
+enum Role : uint32_t { ROLE_TMA = 1, ROLE_MMA = 2, ROLE_EPI = 3 };
+enum Bar : uint32_t { BAR_FULL = 1, BAR_EMPTY = 2, BAR_TMEM_FULL = 3, BAR_TMEM_EMPTY = 4 };
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the wait expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status, uint32_t code) {
+    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it >= SPIN_FAST) {
+            if (*abort_flag) return false;
+            __nanosleep(128);
+        }
+    }
+    atomicCAS(status, 0u, code);
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap* tm, uint32_t dst, uint32_t bar, int32_t c0, int32_t c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+// shared-memory matrix descriptor (128-byte swizzle): start address, leading / stride byte offsets in 16-byte units
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;      // descriptor version of the tcgen05 family
+    d |= (uint64_t)2 << 61;      // swizzle mode: 128 bytes
+    return d;
+}
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the mbarrier once all previously issued MMAs of this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+template <int BN> struct TcCfg {
+    static constexpr int A_BYTES = TBM * TBK * 2;
+    static constexpr int B_BYTES = BN * TBK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int TMEM_COLS = 2 * BN;                       // two accumulators
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// A_MN: op(A) is contiguous along m in memory (transA = N); B_MN: op(B) contiguous along n (transB = T).
+template <int BN, bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(192, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
+               int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
+               uint32_t idesc, uint32_t* status) {
+    using Cfg = TcCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::STAGE_BYTES);
+    // barrier slots: [0,S) full, [S,2S) empty, 2S+{0,1} tmem_full, 2S+{2,3} tmem_empty, then 2 words
+    const uint32_t bar0 = smem_base + STAGES * Cfg::STAGE_BYTES;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 4);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // TMEM allocation is a warp-wide operation; the base address lands in shared memory
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int64_t items = (int64_t)tiles_m * tiles_n * splits;
+    constexpr int GROUP = 8;
+    auto decode = [&](int64_t item, int& tm, int& tn, int& sp) {
+        const int64_t tiles = (int64_t)tiles_m * tiles_n;
+        sp = (int)(item / tiles);
+        const int tile = (int)(item % tiles);
+        const int per_group = GROUP * tiles_n;
+        const int g = tile / per_group;
+        const int gsz = min(GROUP, tiles_m - g * GROUP);
+        tm = g * GROUP + (tile % per_group) % gsz;
+        tn = (tile % per_group) / gsz;
+    };
+    auto kblocks_of = [&](int sp, int64_t& kbeg) {
+        kbeg = (int64_t)sp * kchunk;
+        const int64_t kend = min(k, kbeg + kchunk);
+        return (int)((kend - kbeg + TBK - 1) / TBK);
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t cnt = 0;
+            bool ok = true;
+            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+                int tm, tn, sp;
+                decode(item, tm, tn, sp);
+                int64_t kbeg;
+                const int kb_n = kblocks_of(sp, kbeg);
+                const int32_t m0 = tm * TBM, n0 = tn * BN;
+                for (int kb = 0; kb < kb_n; ++kb, ++cnt) {
+                    const int s = cnt % STAGES;
+                    const uint32_t ph = (cnt / STAGES) & 1;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1, abort_flag, status,
+                                   STATUS_MARK | (ROLE_TMA << 16) | (BAR_EMPTY << 8) | s)) { ok = false; break; }
+                    const uint32_t sa = smem_base + s * Cfg::STAGE_BYTES;
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+                    const int32_t k0 = (int32_t)(kbeg + (int64_t)kb * TBK);
+                    mbar_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+                    if (A_MN) {
+#pragma unroll
+                        for (int c = 0; c < TBM / 64; ++c) tma_load_2d(&tmA, sa + c * (64 * TBK * 2), full_bar(s), m0 + c * 64, k0);
+                    } else {
+                        tma_load_2d(&tmA, sa, full_bar(s), k0, m0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int c = 0; c < BN / 64; ++c) tma_load_2d(&tmB, sb + c * (64 * TBK * 2), full_bar(s), n0 + c * 64, k0);
+                    } else {
+                        tma_load_2d(&tmB, sb, full_bar(s), k0, n0);
+                    }
+                }
+            }
+            // drain: do not leave the CTA while copies that were armed may still be landing
+            const uint32_t armed = cnt < (uint32_t)STAGES ? cnt : (uint32_t)STAGES;
+            for (uint32_t i = 0; i < armed; ++i) {
+                const uint32_t c = cnt - 1 - i;
+                const int s = c % STAGES;
+                const uint32_t ph = (c / STAGES) & 1;
+                for (uint32_t it = 0; it < (1u << 20); ++it)
+                    if (mbar_try_wait(full_bar(s), ph)) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t cnt = 0, it = 0;
+            bool ok = true;
+            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
+                int tm, tn, sp;
+                decode(item, tm, tn, sp);
+                int64_t kbeg;
+                const int kb_n = kblocks_of(sp, kbeg);
+                const uint32_t acc = it & 1, aph = (it >> 1) & 1;
+                if (!mbar_wait(tempty_bar(acc), aph ^ 1, abort_flag, status,
+                               STATUS_MARK | (ROLE_MMA << 16) | (BAR_TMEM_EMPTY << 8) | acc)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < kb_n; ++kb, ++cnt) {
+                    const int s = cnt % STAGES;
+                    const uint32_t ph = (cnt / STAGES) & 1;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, status,
+                                   STATUS_MARK | (ROLE_MMA << 16) | (BAR_FULL << 8) | s)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_base + s * Cfg::STAGE_BYTES;
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < TBK / UMMA_K; ++kk) {
+                        // K-major: 16 k = 32 bytes inside the 128-byte row.  MN-major: 16 k rows of 128 bytes;
+                        // 64-element chunks of m/n are TBK*128 bytes apart, 8-row k groups 1024 bytes apart.
+                        const uint64_t ad = A_MN ? smem_desc(sa + kk * (UMMA_K * 128), TBK * 128, 1024)
+                                                 : smem_desc(sa + kk * (UMMA_K * 2), 0, 1024);
+                        const uint64_t bd = B_MN ? smem_desc(sb + kk * (UMMA_K * 128), TBK * 128, 1024)
+                                                 : smem_desc(sb + kk * (UMMA_K * 2), 0, 1024);
+                        umma_f16(d_tmem, ad, bd, idesc, (kb | kk) != 0);
+                    }
+                    umma_commit(empty_bar(s));          // frees the stage when these MMAs have read it
+                }
+                if (!ok) break;
+                umma_commit(tfull_bar(acc));            // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue (warps 2..5), TMEM lanes 32q .. 32q+31
+        const int q = warp & 3;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
+            int tm, tn, sp;
+            decode(item, tm, tn, sp);
+            const uint32_t acc = it & 1, aph = (it >> 1) & 1;
+            if (!mbar_wait(tfull_bar(acc), aph, abort_flag, status,
+                           STATUS_MARK | (ROLE_EPI << 16) | (BAR_TMEM_FULL << 8) | acc)) { ok = false; break; }
+            tc_fence_after();
+            const int64_t row = (int64_t)tm * TBM + q * 32 + lane;
+            const int64_t n0 = (int64_t)tn * BN;
+            const bool raw = splits > 1;
+            float* out = raw ? partials + (int64_t)sp * m * n : C;
+            const int64_t ldo = raw ? m : ldc;
+            const bool warp_has_rows = (int64_t)tm * TBM + q * 32 < m;
+            if (warp_has_rows) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    if (n0 + c * 32 >= n) break;
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + acc * BN + c * 32 + ((uint32_t)(q * 32) << 16), v);
+                    tmem_ld_wait();
+                    if (row < m) {
+                        float* cp = out + row + (n0 + c * 32) * ldo;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (n0 + c * 32 + j < n) {
+                                float r = __uint_as_float(v[j]);
+                                if (!raw) {
+                                    r *= alpha;
+                                    if (beta != 0.0f) r = fmaf(beta, cp[j * ldo], r);
+                                }
+                                cp[j * ldo] = r;
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+        }
+    }
+
+    // ------------------------------------------------ teardown: every thread arrives here on every path
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D map over a stored column-major matrix: dim0 = contiguous dimension (rows), dim1 = columns (stride ld)
+static bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_t cols, int64_t ld,
+                     uint32_t box_rows, uint32_t box_cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)rows, (cuuint64_t)cols};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {box_rows, box_cols};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, dtype == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+bool tensor_eligible(const GemmArgs& a) {
+    if (a.dtype != GEMM_F16 && a.dtype != GEMM_BF16) return false;
+    auto ok = [](const void* p, int64_t ld) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0 && ld % 8 == 0; };
+    if (!ok(a.A, a.lda) || !ok(a.B, a.ldb)) return false;
+    if (a.m > 0x7FFFFFFFLL || a.n > 0x7FFFFFFFLL || a.k > 0x7FFFFFFFLL) return false;
+    if (a.lda * 2 >= (1LL << 40) || a.ldb * 2 >= (1LL << 40)) return false;
+    return encode_fn() != nullptr;
+}
+
+static uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int bn) {
+    const uint32_t fmt = dtype == GEMM_F16 ? 0u : 1u;    // input format: 0 = f16, 1 = bf16
+    uint32_t d = 0;
+    d |= 1u << 4;                    // accumulator format: f32
+    d |= fmt << 7;                   // A format
+    d |= fmt << 10;                  // B format
+    d |= (a_mn ? 1u : 0u) << 15;     // A is MN-major
+    d |= (b_mn ? 1u : 0u) << 16;     // B is MN-major
+    d |= (uint32_t)(bn >> 3) << 17;  // N / 8
+    d |= (uint32_t)(TBM >> 4) << 24; // M / 16
+    return d;
+}
+
+template <int BN, bool A_MN, bool B_MN>
+static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
+                             const CUtensorMap& tmA, const CUtensorMap& tmB) {
+    using Cfg = TcCfg<BN>;
+    static bool attr_set = false;
+    auto kern = tc_gemm_kernel<BN, A_MN, B_MN>;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int64_t tiles_m = (a.m + TBM - 1) / TBM, tiles_n = (a.n + BN - 1) / BN;
+    if (tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF || tiles_m * tiles_n > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    const int64_t items = tiles_m * tiles_n * ks.splits;
+    const int grid = (int)(items < sm_count() ? items : sm_count());
+    cfg->tile_m = TBM; cfg->tile_n = BN; cfg->tile_k = TBK; cfg->stages = Cfg::STAGES; cfg->grid = grid;
+    kern<<<grid, 192, Cfg::SMEM_BYTES, a.stream>>>(tmA, tmB, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc, (int)tiles_m,
+                                                   (int)tiles_n, ks.splits, ks.chunk,
+                                                   ks.splits > 1 ? partials : nullptr,
+                                                   instr_desc(a.dtype, A_MN, B_MN, BN), a.status);
+    return cudaGetLastError();
+}
+
+template <bool A_MN, bool B_MN>
+static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg) {
+    CUtensorMap tmA, tmB;
+    // stored A: (m x k) if transA = N [contiguous m], (k x m) otherwise [contiguous k]
+    bool ok = A_MN ? make_map(&tmA, a.dtype, a.A, a.m, a.k, a.lda, 64, TBK)
+                   : make_map(&tmA, a.dtype, a.A, a.k, a.m, a.lda, TBK, TBM);
+    // stored B: (k x n) if transB = N [contiguous k], (n x k) otherwise [contiguous n]
+    ok = ok && (B_MN ? make_map(&tmB, a.dtype, a.B, a.n, a.k, a.ldb, 64, TBK)
+                     : make_map(&tmB, a.dtype, a.B, a.k, a.n, a.ldb, TBK, (uint32_t)tile_n));
+    if (!ok) return cudaErrorInvalidValue;
+    switch (tile_n) {
+        case 256: return launch_tc<256, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB);
+        case 128: return launch_tc<128, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB);
+        default:  return launch_tc<64, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB);
+    }
+}
+
+cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg) {
+    cfg->kernel = GEMM_KERNEL_TENSOR;
+    cfg->split_k = ks.splits;
+    cfg->vector_a = cfg->vector_b = 1;
+    const bool a_mn = !a.ta, b_mn = a.tb;
+    if (a_mn && b_mn) return launch_tc_bn<true, true>(a, tile_n, ks, partials, cfg);
+    if (a_mn && !b_mn) return launch_tc_bn<true, false>(a, tile_n, ks, partials, cfg);
+    if (!a_mn && b_mn) return launch_tc_bn<false, true>(a, tile_n, ks, partials, cfg);
+    return launch_tc_bn<false, false>(a, tile_n, ks, partials, cfg);
+}
+
+}  // namespace b200gemm

@@ -1,0 +1,186 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on shapes that
+span several tiles with ragged tails, all transpose combinations, padded leading dimensions, and the
+degenerate cases.  Tolerances: bit-exact on integer-valued inputs; fp32 max |C - C_ref| <=
+4*2^-24*(k*|alpha|*max|A|*max|B| + |beta|*max|C0|); fp16/bf16 relative Frobenius error <= 1e-3 against the
+fp64 oracle on the same rounded inputs."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2310_17408_b200 as g
+from workloads import DTYPE_BF16, DTYPE_F16, DTYPE_F32, Problem, make_matrix
+
+from gpu_util import check_against_oracle, drop_workspace, ensure_workspace, run_problem
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [(1, 1, 1), (64, 64, 64), (129, 257, 65), (200, 300, 150), (5, 1000, 33), (1000, 5, 70),
+          (257, 129, 1030), (130, 70, 17), (384, 512, 256)]
+TRANS = list(itertools.product("NT", "NT"))
+FAMILIES = {DTYPE_F32: [g.GEMM_KERNEL_SIMT_GENERIC, g.GEMM_KERNEL_SIMT_FAST],
+            DTYPE_F16: [g.GEMM_KERNEL_SIMT_GENERIC, g.GEMM_KERNEL_TENSOR],
+            DTYPE_BF16: [g.GEMM_KERNEL_SIMT_GENERIC, g.GEMM_KERNEL_TENSOR]}
+
+
+@pytest.fixture(autouse=True)
+def _reset_forcing():
+    yield
+    g.gemm_force_kernel(g.GEMM_KERNEL_AUTO)
+    g.gemm_force_tile(0, 0, 0)
+
+
+def problem(dtype, m, n, k, ta, tb, alpha, beta, kind, pad, seed=1):
+    kindA = kindB = kind
+    return Problem("t", dtype, m, n, k, alpha, beta, ta, tb, kindA=kindA, kindB=kindB, kindC=kind if kind == "int" else "uniform",
+                   seed=seed, pad=pad)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_F16, DTYPE_BF16])
+@pytest.mark.parametrize("ta,tb", TRANS)
+def test_parity_grid(dtype, ta, tb):
+    kind = "uniform" if dtype == DTYPE_F32 else "normal"
+    for family in FAMILIES[dtype]:
+        g.gemm_force_kernel(family)
+        for (m, n, k) in SHAPES:
+            for (alpha, beta), pad in [((1.0, 0.0), (0, 0, 0)), ((1.5, 0.5), (8, 8, 4)), ((-0.75, 1.0), (1, 3, 1))]:
+                p = problem(dtype, m, n, k, ta, tb, alpha, beta, kind, pad, seed=m + n + k)
+                A, B, C0 = p.operands()
+                C, cfg = run_problem(p, A, B, C0)
+                check_against_oracle(p, A, B, C0, C)
+                if family == g.GEMM_KERNEL_SIMT_GENERIC:
+                    assert cfg["kernel"] == g.GEMM_KERNEL_SIMT_GENERIC
+                # integer-valued inputs: bit-exact
+                p = problem(dtype, m, n, k, ta, tb, alpha, beta, "int", pad, seed=7 + m)
+                A, B, C0 = p.operands()
+                C, cfg = run_problem(p, A, B, C0)
+                check_against_oracle(p, A, B, C0, C, integer=True)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_F16, DTYPE_BF16])
+def test_every_tile_and_split_k(dtype):
+    ensure_workspace(256 << 20)
+    tiles = [(128, 128), (128, 64), (64, 128), (64, 64)] if dtype == DTYPE_F32 else [(128, 256), (128, 128), (128, 64)]
+    kind = "uniform" if dtype == DTYPE_F32 else "normal"
+    for (tm, tn), split in itertools.product(tiles, (1, 2, 5)):
+        g.gemm_force_tile(tm, tn, split)
+        for ta, tb in TRANS:
+            p = problem(dtype, 300, 520, 777, ta, tb, 1.5, 0.5, kind, (0, 8, 2), seed=tm + tn + split)
+            A, B, C0 = p.operands()
+            C, cfg = run_problem(p, A, B, C0)
+            assert (cfg["tile_m"], cfg["tile_n"]) == (tm, tn), cfg
+            assert cfg["split_k"] == split or (split > 1 and cfg["split_k"] > 1), cfg
+            check_against_oracle(p, A, B, C0, C)
+            p = problem(dtype, 300, 520, 777, ta, tb, 1.5, 0.5, "int", (0, 8, 2), seed=3)
+            A, B, C0 = p.operands()
+            C, cfg = run_problem(p, A, B, C0)
+            check_against_oracle(p, A, B, C0, C, integer=True)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_F16, DTYPE_BF16])
+def test_results_are_deterministic(dtype):
+    ensure_workspace(64 << 20)
+    p = problem(dtype, 256, 256, 4096, "N", "N", 1.0, 0.0, "uniform", (0, 0, 0))
+    A, B, C0 = p.operands()
+    C1, cfg1 = run_problem(p, A, B, C0)
+    C2, cfg2 = run_problem(p, A, B, C0)
+    assert cfg1 == cfg2
+    assert np.array_equal(C1.buf.view(np.uint32), C2.buf.view(np.uint32))
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_F16])
+def test_unaligned_operands_take_a_working_path(dtype):
+    # odd leading dimensions and pointers offset by one element: no 16-byte alignment anywhere
+    m, n, k = 150, 260, 147
+    p = problem(dtype, m, n, k, "N", "N", 1.0, 0.0, "uniform", (1, 0, 1))
+    A, B, C0 = p.operands()
+    for ws in (True, False):
+        if not ws:
+            drop_workspace()
+        C, cfg = run_problem(p, A, B, C0, workspace=ws)
+        check_against_oracle(p, A, B, C0, C)
+        if dtype == DTYPE_F16:
+            assert (cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["repacked"] == 3) if ws else \
+                (cfg["kernel"] == g.GEMM_KERNEL_SIMT_GENERIC)
+    # pointers offset by one element
+    es = 4 if dtype == DTYPE_F32 else 2
+    from gpu_util import to_device
+    dA, dB, dC = to_device(A), to_device(B), to_device(C0)
+    big = torch.empty(dA.numel() + 1, dtype=dA.dtype, device="cuda")
+    big[1:] = dA
+    rc = g.gemm(dtype, "N", "N", m, n, k, 1.0, big.data_ptr() + es, A.ld, dB.data_ptr(), B.ld, 0.0, dC.data_ptr(), C0.ld,
+                torch.cuda.current_stream().cuda_stream)
+    assert rc == 0 and g.gemm_poll_status() == 0
+    from workloads import Matrix
+    C = Matrix(dC.cpu().numpy(), m, n, C0.ld, DTYPE_F32)
+    check_against_oracle(p, A, B, C0, C)
+
+
+def test_degenerate_cases():
+    s = torch.cuda.current_stream().cuda_stream
+    C0 = make_matrix(40, 30, kind="uniform", seed=2, matrix_id=2, ld=44)
+    A = make_matrix(40, 16, kind="uniform", seed=2, matrix_id=0)
+    B = make_matrix(16, 30, kind="uniform", seed=2, matrix_id=1)
+    from gpu_util import to_device
+    dA, dB = to_device(A), to_device(B)
+
+    def call(m, n, k, alpha, beta, c_init=None, a=dA, b=dB):
+        dC = to_device(C0) if c_init is None else c_init.clone()
+        rc = g.gemm(DTYPE_F32, "N", "N", m, n, k, alpha, a.data_ptr() if a is not None else 0, 40,
+                    b.data_ptr() if b is not None else 0, 16, beta, dC.data_ptr(), 44, s)
+        assert rc == 0, g.gemm_status_string(rc)
+        assert g.gemm_poll_status() == 0
+        return dC.cpu().numpy()
+
+    base = C0.buf
+    # m == 0 or n == 0: nothing happens
+    assert np.array_equal(call(0, 30, 16, 1.0, 0.0).view(np.uint32), base.view(np.uint32))
+    assert np.array_equal(call(40, 0, 16, 1.0, 0.0).view(np.uint32), base.view(np.uint32))
+    # k == 0 / alpha == 0: C <- beta*C, A and B may be null
+    want = C0.copy(); want.window()[:] = 0.5 * C0.window()
+    assert np.array_equal(call(40, 30, 0, 1.0, 0.5, a=None, b=None).view(np.uint32), want.buf.view(np.uint32))
+    assert np.array_equal(call(40, 30, 16, 0.0, 0.5, a=None, b=None).view(np.uint32), want.buf.view(np.uint32))
+    # beta == 1 with nothing to add: untouched
+    assert np.array_equal(call(40, 30, 16, 0.0, 1.0).view(np.uint32), base.view(np.uint32))
+    # beta == 0: C is write-only, NaN/Inf in it must not propagate (also through the main kernels)
+    nanC = torch.full((44 * 30,), float("nan"), device="cuda")
+    out = call(40, 30, 0, 1.0, 0.0, c_init=nanC).reshape(30, 44)
+    assert np.all(out[:, :40] == 0.0) and np.all(np.isnan(out[:, 40:]))
+    out = call(40, 30, 16, 1.0, 0.0, c_init=nanC).reshape(30, 44)
+    assert np.all(np.isfinite(out[:, :40])) and np.all(np.isnan(out[:, 40:]))
+    ref = A.as_f64() @ B.as_f64()
+    assert np.max(np.abs(out[:, :40].T - ref)) < 1e-5
+    for dt in (DTYPE_F16, DTYPE_BF16):
+        Ah = make_matrix(40, 16, kind="int", seed=2, matrix_id=0, dtype=dt)
+        Bh = make_matrix(16, 30, kind="int", seed=2, matrix_id=1, dtype=dt)
+        dAh, dBh = to_device(Ah), to_device(Bh)
+        dC = nanC.clone()
+        assert g.gemm(dt, "N", "N", 40, 30, 16, 1.0, dAh.data_ptr(), 40, dBh.data_ptr(), 16, 0.0, dC.data_ptr(), 44, s) == 0
+        out = dC.cpu().numpy().reshape(30, 44)
+        assert np.array_equal(out[:, :40].T, Ah.as_f64() @ Bh.as_f64())
+
+
+def test_invalid_arguments_launch_nothing():
+    C = torch.full((64,), 7.0, device="cuda")
+    A = torch.zeros(64, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    a, c = A.data_ptr(), C.data_ptr()
+    cases = [((9, "N", "N", 8, 8, 8, 1.0, a, 8, a, 8, 0.0, c, 8), -1),
+             ((0, "X", "N", 8, 8, 8, 1.0, a, 8, a, 8, 0.0, c, 8), -2),
+             ((0, "N", "Q", 8, 8, 8, 1.0, a, 8, a, 8, 0.0, c, 8), -3),
+             ((0, "N", "N", -1, 8, 8, 1.0, a, 8, a, 8, 0.0, c, 8), -4),
+             ((0, "N", "N", 8, -1, 8, 1.0, a, 8, a, 8, 0.0, c, 8), -5),
+             ((0, "N", "N", 8, 8, -1, 1.0, a, 8, a, 8, 0.0, c, 8), -6),
+             ((0, "N", "N", 8, 8, 8, 1.0, 0, 8, a, 8, 0.0, c, 8), -8),
+             ((0, "N", "N", 8, 8, 8, 1.0, a, 7, a, 8, 0.0, c, 8), -9),
+             ((0, "T", "N", 8, 8, 4, 1.0, a, 3, a, 8, 0.0, c, 8), -9),
+             ((0, "N", "N", 8, 8, 8, 1.0, a, 8, 0, 8, 0.0, c, 8), -10),
+             ((0, "N", "N", 8, 8, 8, 1.0, a, 8, a, 7, 0.0, c, 8), -11),
+             ((0, "N", "N", 8, 8, 8, 1.0, a, 8, a, 8, 0.0, 0, 8), -13),
+             ((0, "N", "N", 8, 8, 8, 1.0, a, 8, a, 8, 0.0, c, 7), -14)]
+    for args, want in cases:
+        assert g.gemm(*args, s) == want, (args, want)
+        assert g.gemm_status_string(want).startswith("invalid argument")
+    torch.cuda.synchronize()
+    assert torch.all(C == 7.0)

@@ -1,0 +1,41 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import paper_2310_17408_b200 as g
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "b200_gemm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"^\s*(?:const\s+char\s*\*|int|size_t|uint32_t)\s+(gemm\w*)\s*\(", text, flags=re.M)
+    return sorted(set(names))
+
+
+def test_every_declared_symbol_is_exported():
+    lib = ctypes.CDLL(g.library_path())
+    names = declared_functions()
+    assert "gemm" in names and "gemm_host" in names and len(names) >= 11
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(g.EXPORTS) == names
+
+
+def test_argument_checks_run_without_a_device():
+    # validation happens before any CUDA call: negative position of the first bad argument
+    assert g.gemm(7, "N", "N", 1, 1, 1, 1.0, 16, 1, 16, 1, 0.0, 16, 1) == -1
+    assert g.gemm(0, "N", "N", 4, 4, 4, 1.0, 16, 3, 16, 4, 0.0, 16, 4) == -9
+    assert g.gemm(0, "N", "N", 4, 4, 4, 1.0, 16, 4, 16, 4, 0.0, 16, 2) == -14
+    assert g.gemm(0, "N", "N", 0, 4, 4, 1.0, 0, 1, 0, 4, 0.0, 0, 1) == 0       # m == 0: nothing to do
+    assert "lda" in g.gemm_status_string(-9)
+    assert g.gemm_force_kernel(99) == -1 and g.gemm_force_kernel(0) == 0
+
+
+def test_workspace_request_for_split_k_shapes():
+    # large-k, few-tile fp32 problem: the selector wants room for fp32 partial sums
+    assert g.gemm_workspace_bytes(0, "N", "N", 256, 256, 65536) >= 2 * 256 * 256 * 4
+    assert g.gemm_workspace_bytes(0, "N", "N", 8192, 8192, 8192) == 0
+    assert g.gemm_workspace_bytes(0, "N", "N", 0, 8, 8) == 0
