@@ -43,8 +43,9 @@ def run_problem(p: Problem, A: Matrix, B: Matrix, C0: Matrix, *, workspace=True,
     C = Matrix(dC.cpu().numpy(), p.m, p.n, C0.ld, DTYPE_F32)
     assert C.padding_intact(), "rows m..ldc-1 of C were written"
     if check_inputs:
-        assert np.array_equal(dA.cpu().numpy().view(A.buf.dtype), A.buf), "A was modified"
-        assert np.array_equal(dB.cpu().numpy().view(B.buf.dtype), B.buf), "B was modified"
+        bits = lambda x: x.view(np.uint32 if x.dtype.itemsize == 4 else np.uint16)   # NaN canaries: compare bit patterns
+        assert np.array_equal(bits(dA.cpu().numpy()), bits(A.buf)), "A was modified"
+        assert np.array_equal(bits(dB.cpu().numpy()), bits(B.buf)), "B was modified"
     return C, cfg
 
 
