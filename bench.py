@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the GEMM hot path on B200.
+
+One "step" is one pass over every problem of a workload (default: the square fp32 sweep
+m=n=k in {1024, 2048, 4096, 8192}, alpha=1.5, beta=0.5), each problem one call of the C-ABI `gemm`.
+Prints ONE JSON line: whole-job TFLOP/s with operands resident in HBM (`value`), the same metric
+through `gemm_host` with pinned host buffers (`e2e`), the roofline of the dominant kernel, the CPU
+oracle timed on the host cores on a bounded sample (`cpu_baseline`), and the SM clocks seen.
+
+`--impl reference` times the CPU oracle (as it stands) on the host cores instead.
+With N > 1 (torchrun) every rank runs an independent replica of the step on its own GPU: GEMM calls
+do not communicate, so there is no collective on the data path ("replicas only").
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from workloads import DTYPE_BF16, DTYPE_F16, DTYPE_F32, DTYPE_NAMES, config_problems  # noqa: E402
+
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+WORKLOADS = {
+    "cfg2_fp32_squares": lambda: config_problems(2),
+    "cfg1_fp32_512": lambda: config_problems(1),
+    "cfg3_fp32_im2row": lambda: config_problems(3),
+    "cfg4_fp32_nonsquarish": lambda: config_problems(4),
+    "cfg5_f16": lambda: config_problems(5, dtype=DTYPE_F16),
+    "cfg5_bf16": lambda: config_problems(5, dtype=DTYPE_BF16),
+    "cfg5_f16_squares": lambda: config_problems(5, dtype=DTYPE_F16)[:3],
+    "cfg5_bf16_squares": lambda: config_problems(5, dtype=DTYPE_BF16)[:3],
+}
+
+
+def load_peaks():
+    """Roofline denominators: measured on this machine (MEASURED_PEAKS.json) or the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), tensor_tflops=float(d["bf16_tflops"]),
+                    tensor_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    sm_max_mhz=float(d.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, tensor_tflops=1590.0, tensor_tflops_sustained=1400.0, sm_max_mhz=1965.0,
+                source="fallback")
+
+
+def fp32_alu_peak_tflops(sm_mhz: float) -> float:
+    # 148 SMs x 128 fp32 lanes x 2 flops per FMA x clock
+    return SM_COUNT * FP32_LANES_PER_SM * 2 * sm_mhz * 1e6 / 1e12
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only queries)."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2])); power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        # samples under load: the upper half of the power readings
+        cut = statistics.median(power)
+        loaded = [c for c, p in zip(sm, power) if p >= cut] or sm
+        return {"sm_mhz": statistics.median(loaded), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def roofline_class(p, peaks):
+    """(bound, peak, unit, algorithmic amount) of one problem: the slower of compute and HBM time decides."""
+    t_hbm = p.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
+    if p.dtype == DTYPE_F32:
+        peak_c = fp32_alu_peak_tflops(peaks["sm_max_mhz"])
+        t_cmp = p.flops / (peak_c * 1e12)
+        if t_cmp >= t_hbm:
+            return "alu", peak_c, "TFLOP/s", p.flops / 1e12
+    else:
+        peak_c = peaks["tensor_tflops"]
+        t_cmp = p.flops / (peak_c * 1e12)
+        if t_cmp >= t_hbm:
+            return "tensor", peak_c, "TFLOP/s", p.flops / 1e12
+    return "hbm", peaks["hbm_gbs"], "GB/s", p.algorithmic_bytes() / 1e9
+
+
+# ------------------------------------------------------------------------------------------ reference arm (CPU oracle)
+
+def reference_sample(problems):
+    """Bounded sample of the workload for the CPU oracle: its members with at most ~2e10 flops each."""
+    small = [p for p in problems if p.flops <= 2.0e10]
+    return small or [min(problems, key=lambda p: p.flops)]
+
+
+def oracle_call(oracle, p, ops):
+    A, B, C0 = ops
+    acc = oracle.ACC_F32 if p.dtype == DTYPE_F32 else oracle.ACC_F64
+    return oracle.gemm_l1(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, A.buf, A.ld, B.buf, B.ld, p.beta,
+                          C0.buf, C0.ld, acc=acc)
+
+
+def run_reference(args, problems, workload_name):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    sample = reference_sample(problems)
+    ops = [p.operands() for p in sample]
+    flops = sum(p.flops for p in sample)
+    for _ in range(args.warmup):
+        for p, o in zip(sample, ops):
+            oracle_call(oracle, p, o)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        for p, o in zip(sample, ops):
+            oracle_call(oracle, p, o)
+    dt = time.perf_counter() - t0
+    val = flops * args.steps / dt / 1e12
+    desc = "oracle L1 (blocked, packed, 8x12 micro-kernel, OpenMP) on " + ", ".join(p.name for p in sample)
+    line = {"impl": "reference", "metric": "gemm_tflops", "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": DTYPE_NAMES[problems[0].dtype], "data": "synthetic",
+            "config": {"workload": workload_name, "sample": [p.name for p in sample]},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": desc},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def cpu_baseline(problems, budget_s=20.0):
+    """The oracle as it stands, on the host cores, on the largest members of the workload that fit the budget."""
+    import oracle
+    probe = min(problems, key=lambda p: p.flops)
+    ops = probe.operands()
+    oracle_call(oracle, probe, ops)                      # builds / loads the library, warms the threads
+    t0 = time.perf_counter()
+    oracle_call(oracle, probe, ops)
+    rate = probe.flops / max(time.perf_counter() - t0, 1e-6)
+    chosen, spent = [], 0.0
+    for p in sorted(problems, key=lambda p: p.flops):
+        cost = p.flops / rate
+        if spent + cost > budget_s and chosen:
+            break
+        chosen.append(p)
+        spent += cost
+        if spent > budget_s:
+            break
+    flops, secs = 0.0, 0.0
+    for p in chosen:
+        o = ops if p is probe else p.operands()
+        t0 = time.perf_counter()
+        oracle_call(oracle, p, o)
+        secs += time.perf_counter() - t0
+        flops += p.flops
+    blk = oracle.DEFAULT_BLOCKING
+    return {"value": flops / secs / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"one call each of {', '.join(p.name for p in chosen)} ({flops / 1e9:.1f} GFLOP, {secs:.1f} s); "
+                      f"blocked packed GEMM, micro-kernel {blk['mr']}x{blk['nr']}, mc/kc/nc={blk['mc']}/{blk['kc']}/{blk['nc']}"}
+
+
+# ------------------------------------------------------------------------------------------ CUDA arm
+
+def run_cuda(args, problems, workload_name):
+    import torch
+    import paper_2310_17408_b200 as g
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream().cuda_stream
+
+    # CPU baseline first (rank 0, N = 1 only), before the GPU is busy
+    base = None
+    if world == 1 and not args.no_cpu_baseline:
+        base = cpu_baseline(problems, args.cpu_budget)
+
+    # operands: generated on the host (seeded), kept pinned for the end-to-end leg, resident copies for `value`
+    host, dev = [], []
+    ws_need = 0
+    for p in problems:
+        A, B, C0 = p.operands()
+        view = (lambda x: x.view(np.int16)) if p.dtype != DTYPE_F32 else (lambda x: x)
+        hA, hB, hC = (torch.from_numpy(view(A.buf)).pin_memory(), torch.from_numpy(view(B.buf)).pin_memory(),
+                      torch.from_numpy(C0.buf).pin_memory())
+        host.append((hA, hB, hC, A.ld, B.ld, C0.ld))
+        dev.append((hA.cuda(), hB.cuda(), hC.cuda(), hC.cuda()))      # A, B, C0 (pristine), C (working)
+        ws_need = max(ws_need, g.gemm_workspace_bytes(p.dtype, p.transA, p.transB, p.m, p.n, p.k))
+    ws = torch.empty(max(ws_need, 1 << 20), dtype=torch.uint8, device="cuda")
+    assert g.gemm_set_workspace(ws.data_ptr(), ws.numel(), 0) == 0
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    launches = 0
+
+    def one_step(events=None):
+        nonlocal launches
+        for i, p in enumerate(problems):
+            dA, dB, dC0, dC = dev[i]
+            _, _, _, lda, ldb, ldc = host[i]
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            rc = g.gemm(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), lda, dB.data_ptr(), ldb,
+                        p.beta, dC.data_ptr(), ldc, stream)
+            if rc != 0:
+                raise RuntimeError(f"gemm failed: {g.gemm_status_string(rc)} (cuda error {g.gemm_last_cuda_error()})")
+            if events is not None:
+                e1.record()
+                events[i].append((e0, e1))
+            launches += g.gemm_last_config()["launches"]
+
+    # ---- device-resident timing
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    events = [[] for _ in problems]
+    launches = 0
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record()
+    for _ in range(args.steps):
+        one_step(events)
+    t_end.record()
+    barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    clocks = sampler.stop()
+    timed_launches = launches
+    if g.gemm_poll_status() != 0:
+        raise RuntimeError(f"device status {hex(g.gemm_status_detail())}")
+    configs = []
+    for p in problems:   # what the selector chose (one untimed call each)
+        i = problems.index(p)
+        dA, dB, dC0, dC = dev[i]
+        g.gemm(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), host[i][3], dB.data_ptr(), host[i][4],
+               p.beta, dC.data_ptr(), host[i][5], stream)
+        configs.append(g.gemm_last_config())
+    torch.cuda.synchronize()
+
+    # ---- end to end: pinned host buffers through gemm_host, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        def host_step():
+            for i, p in enumerate(problems):
+                hA, hB, hC, lda, ldb, ldc = host[i]
+                rc = g.gemm_host(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, hA.data_ptr(), lda, hB.data_ptr(),
+                                 ldb, p.beta, hC.data_ptr(), ldc, stream)
+                if rc != 0:
+                    raise RuntimeError(f"gemm_host failed: {g.gemm_status_string(rc)}")
+        host_c0 = [h[2].clone() for h in host]
+        for _ in range(2):
+            host_step()
+        for h, c0 in zip(host, host_c0):
+            h[2].copy_(c0)
+        barrier()
+        t0 = time.perf_counter()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        for _ in range(e2e_steps):
+            host_step()
+        barrier()
+        e2e_s = time.perf_counter() - t0
+        h2d = sum(h[0].numel() * h[0].element_size() + h[1].numel() * h[1].element_size() + h[2].numel() * 4 for h in host)
+        d2h = sum(h[2].numel() * 4 for h in host)
+        e2e = (e2e_s / e2e_steps, h2d, d2h, e2e_steps)
+
+    # ---- reduce over ranks (max time), report on rank 0
+    step_ms = total_ms / args.steps
+    e2e_ms = e2e[0] * 1e3 if e2e else 0.0
+    if world > 1:
+        t = torch.tensor([step_ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms, e2e_ms = float(t[0]), float(t[1])
+    flops_step = sum(p.flops for p in problems)
+    value = world * flops_step / (step_ms * 1e-3) / 1e12
+
+    shapes, dominant, dom_ms = [], None, -1.0
+    for i, p in enumerate(problems):
+        ms = [a.elapsed_time(b) for a, b in events[i]]
+        avg = sum(ms) / len(ms)
+        bound, peak, unit, amount = roofline_class(p, peaks)
+        achieved = amount / (avg * 1e-3) * (1.0 if unit == "TFLOP/s" else 1.0)
+        shapes.append({"name": p.name, "m": p.m, "n": p.n, "k": p.k, "ms": avg, "ms_min": min(ms),
+                       "tflops": p.flops / (avg * 1e-3) / 1e12, "gbs": p.algorithmic_bytes() / (avg * 1e-3) / 1e9,
+                       "bound": bound, "frac": achieved / peak, "kernel": configs[i]["kernel"],
+                       "tile": [configs[i]["tile_m"], configs[i]["tile_n"]], "split_k": configs[i]["split_k"],
+                       "launches": configs[i]["launches"]})
+        if avg > dom_ms:
+            dom_ms, dominant = avg, (p, bound, peak, unit, achieved, configs[i])
+    if rank == 0:
+        p, bound, peak, unit, achieved, cfg = dominant
+        kernel_names = {1: "simt_generic_kernel", 2: "simt_fast_kernel", 3: "tc_gemm_kernel", 6: "scale_kernel"}
+        roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                "traffic": None, "kernel": kernel_names.get(cfg["kernel"], "?"), "problem": p.name,
+                "peak_source": (f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz (max SM clock)"
+                                if bound == "alu" else f"{peaks['source']} ({'MEASURED_PEAKS.json' if peaks['source'] == 'measured' else 'recipe fallback'})")}
+        if bound == "alu" and clocks.get("sm_mhz"):
+            roof["frac_at_sampled_clock"] = achieved / fp32_alu_peak_tflops(clocks["sm_mhz"])
+        line = {"metric": "gemm_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": DTYPE_NAMES[problems[0].dtype], "data": "synthetic",
+                "config": {"workload": workload_name, "problems": [f"{q.m}x{q.n}x{q.k}" for q in problems],
+                           "alpha": problems[0].alpha, "beta": problems[0].beta, "layout": "column-major N,N",
+                           "l2": "inputs larger than L2: one step touches more than 126 MB of operands"
+                                 if sum(q.algorithmic_bytes() for q in problems) > 126e6 else
+                                 "working set smaller than L2 (warm-cache number)",
+                           "parallelism": "replicas only" if world > 1 else "single GPU"},
+                "roofline": roof, "clocks": clocks, "gpu_launches": timed_launches, "shapes": shapes}
+        if e2e:
+            line["e2e"] = {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                           "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3],
+                           "api": "gemm_host (pinned host buffers, copies inside the timed region)"}
+        if base:
+            line["cpu_baseline"] = base
+        print(json.dumps(line))
+        if args.table:
+            with open(args.table, "w") as f:
+                json.dump(line, f, indent=1)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS))
+    ap.add_argument("--table", default=None, help="also write the JSON (indented, with per-shape rows) to this file")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    problems = WORKLOADS[args.workload]()
+    if args.impl == "reference":
+        return run_reference(args, problems, args.workload)
+    return run_cuda(args, problems, args.workload)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -315,6 +315,17 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     if (bad) return bad;
     if (m == 0 || n == 0) return GEMM_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    {   // keep freed staging buffers in the stream-ordered pool instead of returning them at every synchronise
+        static thread_local int pool_tuned_dev = -1;
+        int dev = 0;
+        cudaMemPool_t pool;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev != pool_tuned_dev &&
+            cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+            uint64_t keep = ~0ull;
+            cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+            pool_tuned_dev = dev;
+        }
+    }
     const int es = elem_size(dtype);
     const bool needs_ab = (k > 0 && alpha != 0.0f);
     const size_t a_bytes = needs_ab ? (size_t)lda * (ta ? m : k) * es : 0;
