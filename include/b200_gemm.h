@@ -112,6 +112,34 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
 size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k);
 int gemm_set_workspace(void* dev, size_t bytes, void* stream);
 
+/*
+ * gemm_f32_splitk_static — fp32 split-k GEMM that allocates nothing.  (The paper has no counterpart: this is a
+ * deployment variant of the split-k path of gemm(), not a step of its algorithm.)
+ *
+ * Who needs it: code that must not call cudaMalloc or any allocating routine around the GEMM.  Examples: a
+ * plugin that runs inside another program's memory budget and is handed only its inputs and outputs; a control
+ * or serving loop that cannot afford the device-wide synchronisation an allocation can cause; a thread from
+ * which no allocator is reachable.  Such callers cannot give gemm() a workspace, and without one gemm() does
+ * not split k, which leaves most SMs idle on problems with a small m*n and a large k.
+ *
+ * This entry point keeps the fp32 partial sums of the k partitions in a fixed array of GEMM_STATIC_SCRATCH_BYTES
+ * that is part of the library image: every GPU that loads the library holds that much memory until the process
+ * exits.  The caller passes only inputs and outputs (device pointers, fp32, layout and leading dimensions as
+ * for gemm()); split_k in 2..64 is the number of k partitions asked for (fewer are used when k is short).
+ *   - split_k * m * n * 4 bytes must fit the array; otherwise GEMM_ERR_TOO_LARGE is returned and nothing runs.
+ *   - k >= 1; alpha and beta as for gemm(); C is not read when beta == 0.
+ *   - The first call on each device looks up the array's device address (a symbol query, not an allocation).
+ *     Make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps what the previous call left in it.  Nothing has to be cleared:
+ *     each call overwrites every partial sum that it later reads.  Two calls that may be on the GPU at the same
+ *     time (different streams or host threads) race on the array: order them on one stream.
+ * Returns GEMM_OK, -(position of the first invalid argument), GEMM_ERR_TOO_LARGE or GEMM_ERR_LAUNCH.
+ */
+#define GEMM_STATIC_SCRATCH_BYTES (8u << 20)
+int gemm_f32_splitk_static(char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha,
+                           const float* A, int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
+                           int split_k, void* stream);
+
 /* configuration chosen by the most recent gemm() of the calling thread (for tests and reports) */
 int gemm_last_config(gemm_config_t* out);
 

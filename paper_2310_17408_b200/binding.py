@@ -19,7 +19,8 @@ GEMM_KERNEL_SCALE_ONLY = 6
 
 EXPORTS = ("gemm", "gemm_host", "gemm_workspace_bytes", "gemm_set_workspace", "gemm_last_config",
            "gemm_force_kernel", "gemm_force_tile", "gemm_poll_status", "gemm_status_detail",
-           "gemm_status_string", "gemm_last_cuda_error")
+           "gemm_status_string", "gemm_last_cuda_error", "gemm_f32_splitk_static")
+GEMM_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class GemmConfig(ctypes.Structure):
@@ -60,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.gemm_status_string.argtypes = [ci]
     lib.gemm_last_cuda_error.restype = ci
     lib.gemm_last_cuda_error.argtypes = []
+    lib.gemm_f32_splitk_static.restype = ci
+    lib.gemm_f32_splitk_static.argtypes = [cc, cc, i64, i64, i64, cf, vp, i64, vp, i64, cf, vp, i64, ci, vp]
     return lib
 
 
@@ -121,3 +124,10 @@ def gemm_status_string(code) -> str:
 
 def gemm_last_cuda_error() -> int:
     return _lib.gemm_last_cuda_error()
+
+
+def gemm_f32_splitk_static(transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, split_k, stream=0) -> int:
+    """fp32 split-k GEMM whose partial sums live in a fixed array inside the library: it allocates nothing.
+    Meant for callers that cannot allocate device memory or register a workspace (see include/b200_gemm.h)."""
+    return _lib.gemm_f32_splitk_static(_c(transA), _c(transB), m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
+                                       split_k, stream)
