@@ -164,19 +164,35 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 
 // ---------------------------------------------------------------- 16-bit operand repack (aligned leading dimension)
 
+// one thread per 8 destination elements (one 16-byte store); the source column is read with scalar loads
 __global__ void __launch_bounds__(256)
 repack16_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld, uint16_t* __restrict__ dst,
                 int64_t ld_out) {
-    for (int64_t j = blockIdx.y; j < cols; j += gridDim.y)
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < ld_out; i += (int64_t)gridDim.x * blockDim.x)
-            dst[i + j * ld_out] = (i < rows) ? src[i + j * ld] : (uint16_t)0;
+    const int64_t vec_per_col = ld_out / 8;
+    const int64_t total = vec_per_col * cols;
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t j = idx / vec_per_col, i = (idx % vec_per_col) * 8;
+        const uint16_t* sp = src + i + j * ld;
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t lo = (i + 2 * e < rows) ? sp[2 * e] : 0u;
+            const uint32_t hi = (i + 2 * e + 1 < rows) ? sp[2 * e + 1] : 0u;
+            w[e] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(dst + i + j * ld_out) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
 }
 
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,
                             cudaStream_t stream) {
-    unsigned gx = (unsigned)((ld_out + 255) / 256 > 256 ? 256 : (ld_out + 255) / 256);
-    unsigned gy = (unsigned)(cols > 32768 ? 32768 : cols);
-    repack16_kernel<<<dim3(gx, gy), 256, 0, stream>>>((const uint16_t*)src, rows, cols, ld, (uint16_t*)dst, ld_out);
+    const int64_t total = (ld_out / 8) * cols;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 32;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    repack16_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint16_t*)src, rows, cols, ld, (uint16_t*)dst, ld_out);
     return cudaGetLastError();
 }
 

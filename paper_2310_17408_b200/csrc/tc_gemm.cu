@@ -69,6 +69,18 @@ __device__ __forceinline__ void tma_load_2d(const CUtensorMap* tm, uint32_t dst,
         ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
+// shared memory -> global tile store (bulk async group); out-of-range parts of the box are clipped by the hardware
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int32_t c0, int32_t c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // shared-memory matrix descriptor (128-byte swizzle): start address, leading / stride byte offsets in 16-byte units
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     uint64_t d = 0;
@@ -112,14 +124,15 @@ template <int BN> struct TcCfg {
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
     static constexpr int TMEM_COLS = 2 * BN;                       // two accumulators
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int STORE_BYTES = 4 * 2 * 32 * 32 * 4;       // per epilogue warp: two 32 x 32 fp32 staging tiles
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STORE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 // A_MN: op(A) is contiguous along m in memory (transA = N); B_MN: op(B) contiguous along n (transB = T).
 template <int BN, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(192, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
+               const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
                uint32_t idesc, uint32_t* status) {
     using Cfg = TcCfg<BN>;
@@ -127,9 +140,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::STAGE_BYTES);
+    // layout: [stages][C staging tiles of the epilogue warps][barriers]
+    float* store_stage = reinterpret_cast<float*>(smem_al + STAGES * Cfg::STAGE_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::STAGE_BYTES + Cfg::STORE_BYTES);
     // barrier slots: [0,S) full, [S,2S) empty, 2S+{0,1} tmem_full, 2S+{2,3} tmem_empty, then 2 words
-    const uint32_t bar0 = smem_base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t bar0 = smem_base + STAGES * Cfg::STAGE_BYTES + Cfg::STORE_BYTES;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
@@ -157,7 +172,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tmem_base = *tmem_slot;
 
     const int64_t items = (int64_t)tiles_m * tiles_n * splits;
-    constexpr int GROUP = 8;
+    constexpr int GROUP = 16;
     auto decode = [&](int64_t item, int& tm, int& tn, int& sp) {
         const int64_t tiles = (int64_t)tiles_m * tiles_n;
         sp = (int)(item / tiles);
@@ -259,8 +274,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------ epilogue (warps 2..5), TMEM lanes 32q .. 32q+31
+        // Lane = row of C.  Each 32-column chunk is read from TMEM, scaled, and then either written straight to
+        // global memory (a warp stores 32 consecutive floats of one column per instruction) or, when C can be
+        // addressed by TMA, transposed through a 32 x 32 staging tile in shared memory and written by an
+        // asynchronous bulk tensor store, which also clips the tile at the matrix edge.
         const int q = warp & 3;
-        uint32_t it = 0;
+        float* stage = store_stage + (warp - 2) * (2 * 32 * 32);
+        uint32_t it = 0, sbuf = 0;
         bool ok = true;
         for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
             int tm, tn, sp;
@@ -269,32 +289,54 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!mbar_wait(tfull_bar(acc), aph, abort_flag, status,
                            STATUS_MARK | (ROLE_EPI << 16) | (BAR_TMEM_FULL << 8) | acc)) { ok = false; break; }
             tc_fence_after();
-            const int64_t row = (int64_t)tm * TBM + q * 32 + lane;
+            const int64_t row0 = (int64_t)tm * TBM + q * 32;
+            const int64_t row = row0 + lane;
             const int64_t n0 = (int64_t)tn * BN;
             const bool raw = splits > 1;
             float* out = raw ? partials + (int64_t)sp * m * n : C;
             const int64_t ldo = raw ? m : ldc;
-            const bool warp_has_rows = (int64_t)tm * TBM + q * 32 < m;
-            if (warp_has_rows) {
+            const bool via_tma = store_via_tma && !raw;
+            if (row0 < m) {
 #pragma unroll 1
                 for (int c = 0; c < BN / 32; ++c) {
-                    if (n0 + c * 32 >= n) break;
+                    const int64_t col0 = n0 + c * 32;
+                    if (col0 >= n) break;
                     uint32_t v[32];
                     tmem_ld32(tmem_base + acc * BN + c * 32 + ((uint32_t)(q * 32) << 16), v);
-                    tmem_ld_wait();
-                    if (row < m) {
-                        float* cp = out + row + (n0 + c * 32) * ldo;
+                    float* cp = out + row + col0 * ldo;
+                    float c0[32];
+                    const bool need_c0 = !raw && beta != 0.0f;
+                    if (need_c0) {      // issue all reads of C before waiting on anything
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (n0 + c * 32 + j < n) {
-                                float r = __uint_as_float(v[j]);
-                                if (!raw) {
-                                    r *= alpha;
-                                    if (beta != 0.0f) r = fmaf(beta, cp[j * ldo], r);
-                                }
-                                cp[j * ldo] = r;
-                            }
+                        for (int j = 0; j < 32; ++j) c0[j] = (row < m && col0 + j < n) ? cp[j * ldo] : 0.0f;
+                    }
+                    tmem_ld_wait();
+                    float r[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        r[j] = __uint_as_float(v[j]);
+                        if (!raw) {
+                            r[j] *= alpha;
+                            if (need_c0) r[j] = fmaf(beta, c0[j], r[j]);
                         }
+                    }
+                    if (via_tma) {
+                        if (lane == 0) bulk_wait_read<1>();      // the store that last used this staging tile has read it
+                        __syncwarp();
+                        float* st = stage + sbuf * (32 * 32);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) st[j * 32 + lane] = r[j];
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(&tmC, smem_u32(st), (int32_t)row0, (int32_t)col0);
+                            bulk_commit();
+                        }
+                        sbuf ^= 1;
+                    } else if (row < m) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < n) cp[j * ldo] = r[j];
                     }
                 }
             }
@@ -302,6 +344,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
         }
+        if (lane == 0) bulk_wait_all();       // staging tiles must outlive the stores that read them
     }
 
     // ------------------------------------------------ teardown: every thread arrives here on every path
@@ -349,6 +392,20 @@ static bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows,
     return r == CUDA_SUCCESS;
 }
 
+// map over the fp32 result for the epilogue's tile stores: 32 x 32 boxes, no swizzle
+static bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)n};
+    cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool tensor_eligible(const GemmArgs& a) {
     if (a.dtype != GEMM_F16 && a.dtype != GEMM_BF16) return false;
     auto ok = [](const void* p, int64_t ld) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0 && ld % 8 == 0; };
@@ -373,7 +430,7 @@ static uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int bn) {
 
 template <int BN, bool A_MN, bool B_MN>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
-                             const CUtensorMap& tmA, const CUtensorMap& tmB) {
+                             const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma) {
     using Cfg = TcCfg<BN>;
     static bool attr_set = false;
     auto kern = tc_gemm_kernel<BN, A_MN, B_MN>;
@@ -387,7 +444,7 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     const int64_t items = tiles_m * tiles_n * ks.splits;
     const int grid = (int)(items < sm_count() ? items : sm_count());
     cfg->tile_m = TBM; cfg->tile_n = BN; cfg->tile_k = TBK; cfg->stages = Cfg::STAGES; cfg->grid = grid;
-    kern<<<grid, 192, Cfg::SMEM_BYTES, a.stream>>>(tmA, tmB, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc, (int)tiles_m,
+    kern<<<grid, 192, Cfg::SMEM_BYTES, a.stream>>>(tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc, (int)tiles_m,
                                                    (int)tiles_n, ks.splits, ks.chunk,
                                                    ks.splits > 1 ? partials : nullptr,
                                                    instr_desc(a.dtype, A_MN, B_MN, BN), a.status);
@@ -404,10 +461,16 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
     ok = ok && (B_MN ? make_map(&tmB, a.dtype, a.B, a.n, a.k, a.ldb, 64, TBK)
                      : make_map(&tmB, a.dtype, a.B, a.k, a.n, a.ldb, TBK, (uint32_t)tile_n));
     if (!ok) return cudaErrorInvalidValue;
+    // the result goes out through TMA tile stores when C is 16-byte addressable and this is not a split-k pass
+    CUtensorMap tmC = tmA;
+    int store_via_tma = 0;
+    if (ks.splits == 1 && (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 && a.ldc % 4 == 0 &&
+        a.ldc * 4 < (1LL << 40))
+        store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc) ? 1 : 0;
     switch (tile_n) {
-        case 256: return launch_tc<256, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB);
-        case 128: return launch_tc<128, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB);
-        default:  return launch_tc<64, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB);
+        case 256: return launch_tc<256, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 128: return launch_tc<128, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        default:  return launch_tc<64, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
     }
 }
 
