@@ -66,6 +66,29 @@ struct Loader {
         }
     }
 
+    // Unguarded loads through a running pointer: `p0` addresses load 0 of this thread in the current k slice,
+    // `vstride` is the element distance between consecutive loads of the thread (fixed for the whole call).
+    __device__ static __forceinline__ int64_t load_stride(int64_t ld) {
+        return KCONT ? (int64_t)(NT / (BK / VEC)) * ld : (int64_t)(NT / (X_TILE / VEC)) * ld;
+    }
+    __device__ static __forceinline__ const float* first_load(const float* X, int64_t ld, int64_t x0, int64_t k0, int t) {
+        int x, kk;
+        coord(t, 0, x, kk);
+        return KCONT ? X + (k0 + kk) + (x0 + x) * ld : X + (x0 + x) + (k0 + kk) * ld;
+    }
+    __device__ static __forceinline__ void load_fast(float (&r)[ELEMS], const float* __restrict__ p0, int64_t vstride) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const float* p = p0 + v * vstride;
+            if (VEC == 4) {
+                float4 q = __ldg(reinterpret_cast<const float4*>(p));
+                r[v * 4 + 0] = q.x; r[v * 4 + 1] = q.y; r[v * 4 + 2] = q.z; r[v * 4 + 3] = q.w;
+            } else {
+                r[v] = __ldg(p);
+            }
+        }
+    }
+
     // registers -> shared stage S[kk][x] (row length X_TILE + PAD)
     __device__ static __forceinline__ void store(const float (&r)[ELEMS], float* S, int t) {
 #pragma unroll
@@ -158,12 +181,22 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
     float ra[LA::ELEMS], rb[LB::ELEMS];
     const bool interior = (i0 + BM <= m) && (j0 + BN <= n);
 
+    // interior tiles read whole k slices through running pointers; edge tiles and the k tail take the guarded path
+    const float* pa = LA::first_load(A, lda, i0, kbeg, t);
+    const float* pb = LB::first_load(B, ldb, j0, kbeg, t);
+    const int64_t va = LA::load_stride(lda), vb = LB::load_stride(ldb);
+    const int64_t step_a = A_KCONT ? (int64_t)BK : (int64_t)BK * lda;
+    const int64_t step_b = B_KCONT ? (int64_t)BK : (int64_t)BK * ldb;
+    const int64_t fast_tiles = interior ? (kend - kbeg) / BK : 0;
+
     auto gload = [&](int64_t kt) {
-        const int64_t k0 = kbeg + kt * BK;
-        if (interior && k0 + BK <= kend) {
-            LA::template load<false>(ra, A, lda, i0, k0, m, kend, t);
-            LB::template load<false>(rb, B, ldb, j0, k0, n, kend, t);
+        if (kt < fast_tiles) {
+            LA::load_fast(ra, pa, va);
+            LB::load_fast(rb, pb, vb);
+            pa += step_a;
+            pb += step_b;
         } else {
+            const int64_t k0 = kbeg + kt * BK;
             LA::template load<true>(ra, A, lda, i0, k0, m, kend, t);
             LB::template load<true>(rb, B, ldb, j0, k0, n, kend, t);
         }

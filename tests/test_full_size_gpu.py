@@ -1,0 +1,90 @@
+"""Parity at the full sizes of the workloads, in the configuration the selector picks for them (the one
+bench.py times).  The CPU oracle cannot compute whole results of this size in reasonable time, so each
+result is checked (a) over the whole matrix by a randomised fp64 identity (C x against alpha A (B x) + beta C0 x
+for +-1 probe vectors) and (b) entry by entry against exact fp64 dot products on corners, tile-edge positions,
+thousands of scattered entries and sampled full rows and columns; integer-valued runs are compared bitwise on
+the sampled entries."""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2310_17408_b200 as g
+from workloads import DTYPE_BF16, DTYPE_F16, DTYPE_F32, config_problems
+
+from gpu_util import check_large, run_problem, sample_positions
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_check(p, seed=0):
+    A, B, C0 = p.operands()
+    C, cfg = run_problem(p, A, B, C0, check_inputs=False)
+    err = check_large(p, A, B, C0, C, cfg, seed=seed)
+    return cfg, err
+
+
+def test_config1_512_full_oracle_and_integer_bit_exact():
+    from gpu_util import check_against_oracle
+    p = config_problems(1)[0]
+    A, B, C0 = p.operands()
+    C, cfg = run_problem(p, A, B, C0)
+    check_against_oracle(p, A, B, C0, C)
+    p = config_problems(1, integer=True)[0]
+    A, B, C0 = p.operands()
+    C, cfg = run_problem(p, A, B, C0)
+    check_against_oracle(p, A, B, C0, C, integer=True)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_config2_square_fp32_sweep(idx):
+    p = config_problems(2)[idx]
+    cfg, _ = run_and_check(p, seed=idx)
+    assert cfg["kernel"] == g.GEMM_KERNEL_SIMT_FAST
+
+
+def test_config3_im2row_fp32_all_layers():
+    for i, p in enumerate(config_problems(3)):
+        cfg, _ = run_and_check(p, seed=i)
+        assert cfg["kernel"] == g.GEMM_KERNEL_SIMT_FAST, (p.name, cfg)
+
+
+def test_config4_nonsquarish_fp32():
+    for i, p in enumerate(config_problems(4)):
+        cfg, _ = run_and_check(p, seed=i)
+        assert cfg["kernel"] == g.GEMM_KERNEL_SIMT_FAST
+    assert cfg["split_k"] > 1          # 256 x 256 x 65536: split-k is mandatory
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+def test_config5_half_squares_4096_8192(dtype):
+    for i, p in enumerate(config_problems(5, dtype=dtype)[:2]):
+        cfg, _ = run_and_check(p, seed=i)
+        assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
+
+
+def test_config5_f16_square_16384():
+    p = config_problems(5, dtype=DTYPE_F16)[2]
+    cfg, _ = run_and_check(p)
+    assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+def test_config5_half_im2row_all_layers(dtype):
+    for i, p in enumerate(config_problems(5, dtype=dtype)[3:]):
+        cfg, _ = run_and_check(p, seed=i)
+        assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR, (p.name, cfg)
+
+
+def test_integer_valued_large_shapes_bit_exact_on_samples():
+    # integer entries in [-4, 4]: every partial sum is exact in fp32, so sampled entries must match bitwise
+    cases = [config_problems(2, integer=True)[2], config_problems(4, integer=True)[3],
+             config_problems(5, integer=True, dtype=DTYPE_BF16)[0], config_problems(5, integer=True, dtype=DTYPE_F16)[5]]
+    for p in cases:
+        A, B, C0 = p.operands()
+        C, cfg = run_problem(p, A, B, C0, check_inputs=False)
+        rng = np.random.default_rng(1)
+        rows, cols = sample_positions(p.m, p.n, cfg["tile_m"], cfg["tile_n"], rng, scattered=2048)
+        ref = oracle.gemm_samples_f64(p.dtype, p.transA, p.transB, p.k, p.alpha, A.buf, A.ld, B.buf, B.ld, p.beta,
+                                      C0.buf, C0.ld, rows, cols)
+        got = C.window()[rows, cols]
+        assert np.array_equal(got.astype(np.float64), ref), p.name
