@@ -117,6 +117,29 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": max(power)}
 
 
+def rank_info():
+    """(rank, world size, local rank) from the launcher's environment (torchrun); a plain run is rank 0 of 1."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (a job is as slow as its slowest replica).
+    Needs an initialised process group when the world size is above 1; returns the list unchanged otherwise."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def aggregate_throughput(flops_per_rank_step, step_ms_max, world):
+    """Whole-job TFLOP/s of `world` independent replicas that each did flops_per_rank_step in step_ms_max."""
+    return world * flops_per_rank_step / (step_ms_max * 1e-3) / 1e12
+
+
 def roofline_class(p, peaks):
     """(bound, peak, unit, algorithmic amount) of one problem: the slower of compute and HBM time decides."""
     t_hbm = p.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
@@ -149,8 +172,8 @@ def oracle_call(oracle, p, ops):
 
 
 def run_reference(args, problems, workload_name):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    rank, _, _ = rank_info()
+    if rank != 0:          # under torchrun only rank 0 runs the CPU oracle; the others leave quietly
         return 0
     import oracle
     sample = reference_sample(problems)
@@ -179,31 +202,24 @@ def run_reference(args, problems, workload_name):
     return 0
 
 
-def cpu_baseline(problems, budget_s=20.0):
-    """The oracle as it stands, on the host cores, on the largest members of the workload that fit the budget."""
+def cpu_baseline(problems, operands, budget_s=30.0):
+    """The oracle as it stands, on the host cores: one call each of the workload's members, smallest first,
+    for as long as the next one is predicted (from the rate just measured) to fit the time budget."""
     import oracle
-    probe = min(problems, key=lambda p: p.flops)
-    ops = probe.operands()
-    oracle_call(oracle, probe, ops)                      # builds / loads the library, warms the threads
-    t0 = time.perf_counter()
-    oracle_call(oracle, probe, ops)
-    rate = probe.flops / max(time.perf_counter() - t0, 1e-6)
-    chosen, spent = [], 0.0
-    for p in sorted(problems, key=lambda p: p.flops):
-        cost = p.flops / rate
-        if spent + cost > budget_s and chosen:
+    order = sorted(range(len(problems)), key=lambda i: problems[i].flops)
+    oracle_call(oracle, problems[order[0]], operands[order[0]])      # builds / loads the library, warms the threads
+    chosen, flops, secs, rate = [], 0.0, 0.0, None
+    for i in order:
+        p = problems[i]
+        if rate is not None and secs + p.flops / rate > budget_s:
             break
-        chosen.append(p)
-        spent += cost
-        if spent > budget_s:
-            break
-    flops, secs = 0.0, 0.0
-    for p in chosen:
-        o = ops if p is probe else p.operands()
         t0 = time.perf_counter()
-        oracle_call(oracle, p, o)
-        secs += time.perf_counter() - t0
+        oracle_call(oracle, p, operands[i])
+        dt = time.perf_counter() - t0
+        chosen.append(p)
         flops += p.flops
+        secs += dt
+        rate = p.flops / max(dt, 1e-9)
     blk = oracle.DEFAULT_BLOCKING
     return {"value": flops / secs / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"one call each of {', '.join(p.name for p in chosen)} ({flops / 1e9:.1f} GFLOP, {secs:.1f} s); "
@@ -216,9 +232,7 @@ def run_cuda(args, problems, workload_name):
     import torch
     import paper_2310_17408_b200 as g
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = rank_info()
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
@@ -226,16 +240,16 @@ def run_cuda(args, problems, workload_name):
     peaks = load_peaks()
     stream = torch.cuda.current_stream().cuda_stream
 
-    # CPU baseline first (rank 0, N = 1 only), before the GPU is busy
+    # operands: generated on the host (seeded); the CPU baseline runs first (rank 0, N = 1 only), before the GPU is busy
+    operands = [p.operands() for p in problems]
     base = None
     if world == 1 and not args.no_cpu_baseline:
-        base = cpu_baseline(problems, args.cpu_budget)
+        base = cpu_baseline(problems, operands, args.cpu_budget)
 
-    # operands: generated on the host (seeded), kept pinned for the end-to-end leg, resident copies for `value`
+    # pinned host copies for the end-to-end leg, resident device copies for `value`
     host, dev = [], []
     ws_need = 0
-    for p in problems:
-        A, B, C0 = p.operands()
+    for p, (A, B, C0) in zip(problems, operands):
         view = (lambda x: x.view(np.int16)) if p.dtype != DTYPE_F32 else (lambda x: x)
         hA, hB, hC = (torch.from_numpy(view(A.buf)).pin_memory(), torch.from_numpy(view(B.buf)).pin_memory(),
                       torch.from_numpy(C0.buf).pin_memory())
@@ -361,12 +375,9 @@ def run_cuda(args, problems, workload_name):
     # ---- reduce over ranks (max time), report on rank 0
     step_ms = total_ms / args.steps
     e2e_ms = e2e[0] * 1e3 if e2e else 0.0
-    if world > 1:
-        t = torch.tensor([step_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_ms, e2e_ms = float(t[0]), float(t[1])
+    step_ms, e2e_ms = max_over_ranks([step_ms, e2e_ms], device="cuda")
     flops_step = sum(p.flops for p in problems)
-    value = world * flops_step / (step_ms * 1e-3) / 1e12
+    value = aggregate_throughput(flops_step, step_ms, world)
 
     shapes, dominant, dom_ms = [], None, -1.0
     for i, p in enumerate(problems):
@@ -403,7 +414,7 @@ def run_cuda(args, problems, workload_name):
                            "parallelism": "replicas only" if world > 1 else "single GPU"},
                 "roofline": roof, "clocks": clocks, "gpu_launches": timed_launches, "shapes": shapes}
         if e2e:
-            line["e2e"] = {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            line["e2e"] = {"value": aggregate_throughput(flops_step, e2e_ms, world), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3],
                            "api": "gemm_host (pinned host buffers, copies inside the timed region)"}
         if base:
@@ -430,7 +441,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    ap.add_argument("--cpu-budget", type=float, default=30.0)
     args = ap.parse_args()
     problems = WORKLOADS[args.workload]()
     if args.shape:

@@ -157,6 +157,10 @@ int gemm_force_tile(int tile_m, int tile_n, int split_k);
  */
 int gemm_poll_status(void);
 uint32_t gemm_status_detail(void);
+/* Exercises the give-up path without a fault: enqueues a one-warp kernel that waits, with a limit of well under a
+ * millisecond, on a barrier nothing arrives at.  The wait expires, the kernel exits normally, and the next
+ * gemm_poll_status() returns GEMM_ERR_DEVICE with detail 0xE57F01xx; the context stays usable. */
+int gemm_selftest_wait_expiry(void* stream);
 const char* gemm_status_string(int code);
 int gemm_last_cuda_error(void);   /* cudaError_t of the last failed launch, 0 if none */
 

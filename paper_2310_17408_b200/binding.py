@@ -19,7 +19,8 @@ GEMM_KERNEL_SCALE_ONLY = 6
 
 EXPORTS = ("gemm", "gemm_host", "gemm_workspace_bytes", "gemm_set_workspace", "gemm_last_config",
            "gemm_force_kernel", "gemm_force_tile", "gemm_poll_status", "gemm_status_detail",
-           "gemm_status_string", "gemm_last_cuda_error", "gemm_f32_splitk_static")
+           "gemm_status_string", "gemm_last_cuda_error", "gemm_f32_splitk_static",
+           "gemm_selftest_wait_expiry")
 GEMM_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -61,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.gemm_status_string.argtypes = [ci]
     lib.gemm_last_cuda_error.restype = ci
     lib.gemm_last_cuda_error.argtypes = []
+    lib.gemm_selftest_wait_expiry.restype = ci
+    lib.gemm_selftest_wait_expiry.argtypes = [vp]
     lib.gemm_f32_splitk_static.restype = ci
     lib.gemm_f32_splitk_static.argtypes = [cc, cc, i64, i64, i64, cf, vp, i64, vp, i64, cf, vp, i64, ci, vp]
     return lib
@@ -131,3 +134,8 @@ def gemm_f32_splitk_static(transA, transB, m, n, k, alpha, A, lda, B, ldb, beta,
     Meant for callers that cannot allocate device memory or register a workspace (see include/b200_gemm.h)."""
     return _lib.gemm_f32_splitk_static(_c(transA), _c(transB), m, n, k, alpha, A, lda, B, ldb, beta, C, ldc,
                                        split_k, stream)
+
+
+def gemm_selftest_wait_expiry(stream=0) -> int:
+    """Enqueue the kernel whose bounded wait is certain to expire; gemm_poll_status() then reports GEMM_ERR_DEVICE."""
+    return _lib.gemm_selftest_wait_expiry(stream)

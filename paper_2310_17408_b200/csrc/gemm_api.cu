@@ -421,6 +421,14 @@ int gemm_poll_status(void) {
 
 uint32_t gemm_status_detail(void) { return g_last_detail; }
 
+int gemm_selftest_wait_expiry(void* stream) {
+    DeviceState* st = device_state();
+    if (!st) return GEMM_ERR_LAUNCH;
+    if (!st->arch_ok) return GEMM_ERR_ARCH;
+    cudaError_t e = launch_wait_expiry_probe(st->status, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+}
+
 int gemm_last_cuda_error(void) { return t_last_cuda_error; }
 
 const char* gemm_status_string(int code) {

@@ -55,6 +55,9 @@ cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* parti
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,
                             cudaStream_t stream);
 
+// launches a one-warp kernel whose bounded wait is certain to expire (nothing arrives at its barrier)
+cudaError_t launch_wait_expiry_probe(uint32_t* status, cudaStream_t stream);
+
 int sm_count();
 
 }  // namespace b200gemm

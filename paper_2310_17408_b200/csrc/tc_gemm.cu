@@ -24,7 +24,7 @@ constexpr int UMMA_K = 16;          // k extent of one tcgen05.mma for 16-bit in
 constexpr uint32_t SPIN_FAST = 4096;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;   // then ~128 ns sleeps: gives up after a few seconds
 
-enum Role : uint32_t { ROLE_TMA = 1, ROLE_MMA = 2, ROLE_EPI = 3 };
+enum Role : uint32_t { ROLE_TMA = 1, ROLE_MMA = 2, ROLE_EPI = 3, ROLE_SELFTEST = 0x7F };
 enum Bar : uint32_t { BAR_FULL = 1, BAR_EMPTY = 2, BAR_TMEM_FULL = 3, BAR_TMEM_EMPTY = 4 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -50,8 +50,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait.  Returns false if the wait expired or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status, uint32_t code) {
-    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+                                          uint32_t* status, uint32_t code, uint32_t limit = SPIN_LIMIT) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it >= SPIN_FAST) {
             if (*abort_flag) return false;
@@ -355,6 +355,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::TMEM_COLS) : "memory");
     }
+}
+
+// Self-test of the give-up path: one thread waits, with a short limit, on a barrier that nothing ever arrives at.
+// The wait expires, the code lands in the status word and the kernel returns normally.
+__global__ void __launch_bounds__(32) wait_expiry_probe_kernel(uint32_t* status, uint32_t limit) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(smem_u32(&bar), 0, &abort_flag, status, STATUS_MARK | (ROLE_SELFTEST << 16) | (BAR_FULL << 8), limit);
+    }
+    __syncthreads();
+}
+
+cudaError_t launch_wait_expiry_probe(uint32_t* status, cudaStream_t stream) {
+    wait_expiry_probe_kernel<<<1, 32, 0, stream>>>(status, SPIN_FAST + 2048);     // a few hundred microseconds
+    return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- host side

@@ -184,3 +184,20 @@ def test_invalid_arguments_launch_nothing():
         assert g.gemm_status_string(want).startswith("invalid argument")
     torch.cuda.synchronize()
     assert torch.all(C == 7.0)
+
+
+def test_bounded_wait_expiry_is_reported_and_context_survives():
+    # a wait that can never be satisfied gives up after its limit: status word set, kernel exits, nothing faults
+    s = torch.cuda.current_stream().cuda_stream
+    assert g.gemm_poll_status() == 0
+    assert g.gemm_selftest_wait_expiry(s) == 0
+    assert g.gemm_poll_status() == g.GEMM_ERR_DEVICE
+    detail = g.gemm_status_detail()
+    assert detail >> 24 == 0xE5 and (detail >> 16) & 0xFF == 0x7F, hex(detail)
+    assert g.gemm_status_string(g.GEMM_ERR_DEVICE) == "a bounded device-side wait expired"
+    assert g.gemm_poll_status() == 0                      # cleared by the poll
+    # the context is still usable: a tensor-core GEMM right after it is correct
+    p = problem(DTYPE_BF16, 200, 300, 150, "N", "N", 1.0, 0.0, "int", (0, 0, 0))
+    A, B, C0 = p.operands()
+    C, cfg = run_problem(p, A, B, C0)
+    check_against_oracle(p, A, B, C0, C, integer=True)
