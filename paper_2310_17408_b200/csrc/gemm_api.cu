@@ -1,6 +1,7 @@
 // C ABI of the GEMM library: argument validation, quick returns, the shape selector (tile shape, split-k,
 // fast-path eligibility — the role the paper gives to choosing the (mr, nr) micro-kernel and the cache
 // parameters per problem, Sections I and IV) and dispatch to the kernels.
+#include <algorithm>
 #include <mutex>
 #include <new>
 
@@ -135,26 +136,48 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
     if (p->repack_b) ws_repack += (size_t)round_up(p->ldb_p * b_cols * 2, 256);
     if (ws_repack > ws_avail) { p->kernel = GEMM_KERNEL_SIMT_GENERIC; return; }
 
-    // tile_n: the widest tile that still gives every SM work; narrower tiles when the tile count is small
-    int bn = 256;
-    if (g_force_tile_n == 64 || g_force_tile_n == 128 || g_force_tile_n == 256) bn = g_force_tile_n;
-    else {
-        const int64_t tm = ceil_div(a.m, 128);
-        if (tm * ceil_div(a.n, 256) < sms) bn = 128;
-        if (tm * ceil_div(a.n, 128) < sms) bn = 64;
-        if (a.n <= 64) bn = 64;
-        else if (a.n <= 128 && bn > 128) bn = 128;
+    // Tile width and split-k by a small cost model (microseconds) with constants measured on B200:
+    //   - a kernel costs ~7 us before any tile work shows (launch, TMEM/barrier set-up, first loads, last stores)
+    //   - one 64-wide k block takes max(tensor time 0.27 us * bn/256, stage bytes / 146 GB/s per-SM fill rate)
+    //   - all SMs together fill shared memory from L2 at ~10 TB/s; HBM moves 6.5 TB/s
+    //   - the epilogue moves 32 columns of a tile in ~0.45 us
+    //   - splitting k adds a reduction pass: ~4 us + (splits + 1) * m * n * 4 bytes at ~5 TB/s
+    auto cost_us = [&](int bn, int splits) {
+        const double tiles = (double)ceil_div(a.m, 128) * (double)ceil_div(a.n, bn);
+        const double items = tiles * splits;
+        const double rounds = (double)ceil_div((int64_t)items, sms);
+        const double kb = (double)ceil_div(ceil_div(a.k, splits), 64);
+        const double stage = (128.0 + bn) * 128.0;
+        const double t_kb = std::max(0.27 * bn / 256.0, stage / 146e3);
+        const double main_us = rounds * kb * t_kb + rounds * (bn / 32) * 0.45;
+        const double fill_us = items * kb * stage / 1e7;
+        const double mn = (double)a.m * (double)a.n;
+        const double hbm_us = (2.0 * ((double)a.m * a.k + (double)a.k * a.n) + 4.0 * mn * splits) / 6.5e6;
+        double t = 7.0 + std::max(main_us, std::max(fill_us, hbm_us));
+        if (splits > 1) t += 4.0 + (splits + 1) * mn * 4.0 / 5e6;
+        return t;
+    };
+    int bn = 256, want = 1;
+    {
+        const int bn_lo = (g_force_tile_n == 64 || g_force_tile_n == 128 || g_force_tile_n == 256) ? g_force_tile_n
+                          : (a.n <= 64 ? 64 : 128);
+        const int bn_hi = (g_force_tile_n == 64 || g_force_tile_n == 128 || g_force_tile_n == 256) ? g_force_tile_n
+                          : (a.n <= 64 ? 64 : (a.n <= 128 ? 128 : 256));
+        const int split_opts[] = {1, 2, 3, 4, 6, 8};
+        double best = 1e300;
+        for (int cand = bn_lo; cand <= bn_hi; cand *= 2)
+            for (int so : split_opts) {
+                if (g_force_split > 0 && so != 1) continue;
+                const int sp = g_force_split > 0 ? g_force_split : so;
+                if (sp > 1 && g_force_split == 0) {
+                    if (a.k / sp < 256) continue;
+                    if (ws_repack + (size_t)sp * a.m * a.n * sizeof(float) > ws_avail) continue;
+                }
+                const double c = cost_us(cand, sp);
+                if (c < best) { best = c; bn = cand; want = sp; }
+            }
     }
     p->tile = bn;
-    const int64_t tiles = ceil_div(a.m, 128) * ceil_div(a.n, bn);
-    int want = 1;
-    if (g_force_split > 0) want = g_force_split;
-    else if (tiles * 2 <= sms && a.k >= 1024) {
-        want = (int)(sms / tiles);
-        const int64_t max_by_k = a.k / 512;
-        if (want > max_by_k) want = (int)max_by_k;
-        if (want > 32) want = 32;
-    }
     p->ks = make_split(a.k, want, 64);
     p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
     if (ws_repack + p->ws_partials > ws_avail) {

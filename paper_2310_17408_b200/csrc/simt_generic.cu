@@ -138,27 +138,49 @@ cudaError_t launch_scale(const GemmArgs& a) {
 
 // ---------------------------------------------------------------- split-k reduction + epilogue
 
-// partials: [split][n][m] fp32 (leading dimension m).  Summed in increasing split index.
+// partials: [split][n][m] fp32 (leading dimension m).  Summed in increasing split index (deterministic).
+// Thread block 32 x 8: x walks rows (V of them per thread), y walks columns.
+template <int V>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(int64_t m, int64_t n, int splits, const float* __restrict__ partials, float alpha, float beta,
                      float* __restrict__ C, int64_t ldc) {
-    const int64_t total = m * n;
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (int64_t)gridDim.x * blockDim.x) {
-        float s = partials[idx];
-        for (int z = 1; z < splits; ++z) s += partials[idx + (int64_t)z * total];
-        int64_t i = idx % m, j = idx / m;
-        float* c = C + i + j * ldc;
-        *c = epilogue(alpha, s, beta, c);
-    }
+    const int64_t plane = m * n;
+    const int64_t mv = m / V;
+    for (int64_t j = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; j < n; j += (int64_t)gridDim.y * blockDim.y)
+        for (int64_t iv = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; iv < mv; iv += (int64_t)gridDim.x * blockDim.x) {
+            const float* p = partials + iv * V + j * m;
+            float* c = C + iv * V + j * ldc;
+            if (V == 4) {
+                float4 s = *reinterpret_cast<const float4*>(p);
+                for (int z = 1; z < splits; ++z) {
+                    const float4 q = *reinterpret_cast<const float4*>(p + (int64_t)z * plane);
+                    s.x += q.x; s.y += q.y; s.z += q.z; s.w += q.w;
+                }
+                float4 r = make_float4(alpha * s.x, alpha * s.y, alpha * s.z, alpha * s.w);
+                if (beta != 0.0f) {
+                    const float4 c0 = *reinterpret_cast<const float4*>(c);
+                    r.x = fmaf(beta, c0.x, r.x); r.y = fmaf(beta, c0.y, r.y);
+                    r.z = fmaf(beta, c0.z, r.z); r.w = fmaf(beta, c0.w, r.w);
+                }
+                *reinterpret_cast<float4*>(c) = r;
+            } else {
+                float s = *p;
+                for (int z = 1; z < splits; ++z) s += p[(int64_t)z * plane];
+                *c = epilogue(alpha, s, beta, c);
+            }
+        }
 }
 
 cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* partials) {
-    int64_t total = a.m * a.n;
-    int64_t blocks = (total + 255) / 256;
-    int64_t cap = (int64_t)sm_count() * 16;
-    if (blocks > cap) blocks = cap;
-    splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc);
+    const bool vec = a.m % 4 == 0 && a.ldc % 4 == 0 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 &&
+                     (reinterpret_cast<uintptr_t>(a.C) & 15) == 0;
+    const int64_t mv = vec ? a.m / 4 : a.m;
+    int64_t gx = (mv + 31) / 32, gy = (a.n + 7) / 8;
+    if (gx > 1024) gx = 1024;
+    if (gy > 32768) gy = 32768;
+    dim3 grid((unsigned)gx, (unsigned)gy), block(32, 8);
+    if (vec) splitk_reduce_kernel<4><<<grid, block, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc);
+    else splitk_reduce_kernel<1><<<grid, block, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc);
     return cudaGetLastError();
 }
 

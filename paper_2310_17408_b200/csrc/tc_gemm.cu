@@ -74,6 +74,10 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(tm), "r"(src), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int32_t c0, int32_t c1, int32_t c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_read() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
@@ -295,7 +299,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool raw = splits > 1;
             float* out = raw ? partials + (int64_t)sp * m * n : C;
             const int64_t ldo = raw ? m : ldc;
-            const bool via_tma = store_via_tma && !raw;
+            // store_via_tma: 0 = direct stores, 1 = tmC maps C (2-D), 2 = tmC maps the split-k partials (3-D: m, n, split)
+            const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
             if (row0 < m) {
 #pragma unroll 1
                 for (int c = 0; c < BN / 32; ++c) {
@@ -329,7 +334,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         fence_async_smem();
                         __syncwarp();
                         if (lane == 0) {
-                            tma_store_2d(&tmC, smem_u32(st), (int32_t)row0, (int32_t)col0);
+                            if (raw) tma_store_3d(&tmC, smem_u32(st), (int32_t)row0, (int32_t)col0, sp);
+                            else tma_store_2d(&tmC, smem_u32(st), (int32_t)row0, (int32_t)col0);
                             bulk_commit();
                         }
                         sbuf ^= 1;
@@ -411,6 +417,20 @@ static bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows,
     return r == CUDA_SUCCESS;
 }
 
+// map over the split-k partial sums [split][n][m] (fp32, dense): 32 x 32 x 1 boxes
+static bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)m, (cuuint64_t)n, (cuuint64_t)splits};
+    cuuint64_t strides[2] = {(cuuint64_t)m * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
+    cuuint32_t box[3] = {32, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // map over the fp32 result for the epilogue's tile stores: 32 x 32 boxes, no swizzle
 static bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc) {
     EncodeTiledFn fn = encode_fn();
@@ -486,6 +506,9 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
     if (ks.splits == 1 && (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 && a.ldc % 4 == 0 &&
         a.ldc * 4 < (1LL << 40))
         store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc) ? 1 : 0;
+    if (ks.splits > 1 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && a.m % 4 == 0 &&
+        a.m * a.n * 4 < (1LL << 40))
+        store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
     switch (tile_n) {
         case 256: return launch_tc<256, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
         case 128: return launch_tc<128, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
