@@ -44,6 +44,32 @@ WORKLOADS = {
 }
 
 
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture, see profiles/), keyed by
+# kernel and problem, with the hash of the kernel's source file at capture time: a changed kernel reports null.
+TRAFFIC = {
+    ("simt_fast_kernel", "8192x8192x8192", "f32"): {
+        "bytes": 3197775360 + 259812352, "source": "paper_2310_17408_b200/csrc/simt_fast.cu",
+        "sha256": "85a3f559eb1b818ddc5872644a50230a37e27f3fcffa529f4c08a57c9b244e23"},
+    ("tc_gemm_kernel", "8192x8192x8192", "bf16"): {
+        "bytes": 1038049000 + 250858496, "source": "paper_2310_17408_b200/csrc/tc_gemm.cu",
+        "sha256": "1d18e3ed44c38bfc16185719c7ad841fdafaea0cbf211289395eb17856d23194"},
+}
+
+
+def recorded_traffic(kernel, p):
+    import hashlib
+    rec = TRAFFIC.get((kernel, f"{p.m}x{p.n}x{p.k}", DTYPE_NAMES[p.dtype]))
+    if not rec:
+        return None
+    try:
+        with open(os.path.join(ROOT, rec["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != rec["sha256"]:
+                return None
+    except OSError:
+        return None
+    return rec["bytes"]
+
+
 def load_peaks():
     """Roofline denominators: measured on this machine (MEASURED_PEAKS.json) or the stated fallback."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -398,7 +424,8 @@ def run_cuda(args, problems, workload_name):
         p, bound, peak, unit, achieved, cfg = dominant
         kernel_names = {1: "simt_generic_kernel", 2: "simt_fast_kernel", 3: "tc_gemm_kernel", 6: "scale_kernel"}
         roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": None, "kernel": kernel_names.get(cfg["kernel"], "?"), "problem": p.name,
+                "traffic": recorded_traffic(kernel_names.get(cfg["kernel"], "?"), p),
+                "kernel": kernel_names.get(cfg["kernel"], "?"), "problem": p.name,
                 "peak_source": (f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz (max SM clock)"
                                 if bound == "alu" else f"{peaks['source']} ({'MEASURED_PEAKS.json' if peaks['source'] == 'measured' else 'recipe fallback'})")}
         if bound == "alu" and clocks.get("sm_mhz"):
@@ -437,6 +464,8 @@ def main():
     ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS))
     ap.add_argument("--shape", default=None, help="M,N,K: time this single problem instead of a workload (alpha=1, beta=0)")
     ap.add_argument("--dtype", default="f32", choices=["f32", "f16", "bf16"], help="operand type for --shape")
+    ap.add_argument("--alpha", type=float, default=1.0, help="alpha for --shape")
+    ap.add_argument("--beta", type=float, default=0.0, help="beta for --shape")
     ap.add_argument("--table", default=None, help="also write the JSON (indented, with per-shape rows) to this file")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -449,7 +478,7 @@ def main():
         m, n, k = (int(t) for t in args.shape.split(","))
         dt = {"f32": DTYPE_F32, "f16": DTYPE_F16, "bf16": DTYPE_BF16}[args.dtype]
         kind = "uniform" if dt == DTYPE_F32 else "normal"
-        problems = [Problem(f"{args.dtype}_{m}x{n}x{k}", dt, m, n, k, 1.0, 0.0, kindA=kind, kindB=kind, seed=0)]
+        problems = [Problem(f"{args.dtype}_{m}x{n}x{k}", dt, m, n, k, args.alpha, args.beta, kindA=kind, kindB=kind, seed=0)]
         args.workload = f"single:{args.dtype}:{m}x{n}x{k}"
     if args.impl == "reference":
         return run_reference(args, problems, args.workload)
