@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-from workloads import DTYPE_BF16, DTYPE_F16, DTYPE_F32, DTYPE_NAMES, config_problems  # noqa: E402
+from workloads import DTYPE_BF16, DTYPE_F16, DTYPE_F32, DTYPE_NAMES, config_problems, im2row_problems  # noqa: E402
 
 SM_COUNT = 148
 FP32_LANES_PER_SM = 128
@@ -41,6 +41,12 @@ WORKLOADS = {
     "cfg5_bf16": lambda: config_problems(5, dtype=DTYPE_BF16),
     "cfg5_f16_squares": lambda: config_problems(5, dtype=DTYPE_F16)[:3],
     "cfg5_bf16_squares": lambda: config_problems(5, dtype=DTYPE_BF16)[:3],
+    # second workload (VGG16, batch 32) and the paper's own orientation (m = batch*pixels, n = channels)
+    "vgg16_fp32": lambda: im2row_problems("vgg16"),
+    "vgg16_bf16": lambda: im2row_problems("vgg16", dtype=DTYPE_BF16),
+    "vgg16_fp32_paper_orientation": lambda: im2row_problems("vgg16", weights_as_A=False),
+    "resnet50_fp32_paper_orientation": lambda: im2row_problems("resnet50", weights_as_A=False),
+    "resnet50_bf16_paper_orientation": lambda: im2row_problems("resnet50", weights_as_A=False, dtype=DTYPE_BF16),
 }
 
 

@@ -88,3 +88,13 @@ def test_integer_valued_large_shapes_bit_exact_on_samples():
                                       C0.buf, C0.ld, rows, cols)
         got = C.window()[rows, cols]
         assert np.array_equal(got.astype(np.float64), ref), p.name
+
+
+def test_vgg16_and_paper_orientation_shapes():
+    # second workload (VGG16 at batch 32, includes k = 27) and the tall-and-skinny orientation the paper's tables use
+    from workloads import im2row_problems
+    cases = im2row_problems("vgg16")[:3] + im2row_problems("vgg16", dtype=DTYPE_BF16)[:2] + \
+        im2row_problems("resnet50", weights_as_A=False)[:4] + im2row_problems("resnet50", weights_as_A=False, dtype=DTYPE_F16)[:3] + \
+        im2row_problems("vgg16", weights_as_A=False)[-2:]
+    for i, p in enumerate(cases):
+        run_and_check(p, seed=i)

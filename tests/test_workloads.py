@@ -49,3 +49,13 @@ def test_config_lists():
     c5 = config_problems(5, dtype=DTYPE_BF16)
     assert len(c5) == 23 and c5[0].dtype == DTYPE_BF16 and c5[2].m == 16384
     assert len({p.seed for p in c5}) == 23
+
+
+def test_second_workload_and_paper_orientation():
+    from workloads import im2row_problems
+    v = im2row_problems("vgg16")
+    assert len(v) == 9 and (v[0].m, v[0].n, v[0].k) == (64, 32 * 224 * 224, 27)
+    px = im2row_problems("resnet50", weights_as_A=False)
+    assert len(px) == 20 and (px[0].m, px[0].n, px[0].k) == (32 * 112 * 112, 64, 147)
+    assert px[0].kindA == "absnormal" and px[0].kindB == "normal" and abs(px[0].scaleB ** 2 - 2 / 147) < 1e-15
+    assert len({p.seed for p in v + px}) == 29

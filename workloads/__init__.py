@@ -24,4 +24,5 @@ from .shapes import (  # noqa: F401
     square_half_sweep,
     Problem,
     config_problems,
+    im2row_problems,
 )

@@ -187,3 +187,26 @@ def config_problems(config: int, *, integer: bool = False, dtype: int | None = N
     else:
         raise ValueError("config must be 1..5")
     return probs
+
+
+def im2row_problems(network: str = "vgg16", *, batch: int = 32, weights_as_A: bool = True,
+                    dtype: int = DTYPE_F32) -> list[Problem]:
+    """The second workload and the paper's own orientation of both networks.
+
+    network: 'resnet50' or 'vgg16' (Tables "resnet50" / "vgg16").  weights_as_A=False keeps the paper's roles
+    (m = batch*pixels, n = output channels: activations are operand A, weights operand B), the tall-and-skinny
+    mirror of the config-3 problems.  Seeds 6000 + index (vgg16) / 7000 + index (resnet50), +500 in the paper's
+    orientation.
+    """
+    layers = {"vgg16": VGG16_BATCH1, "resnet50": RESNET50_V15_BATCH1}[network]
+    base = (6000 if network == "vgg16" else 7000) + (0 if weights_as_A else 500)
+    tag = ("h" if dtype == DTYPE_F16 else "b" if dtype == DTYPE_BF16 else "") + network[:3] + ("" if weights_as_A else "_px")
+    probs = []
+    for i, (m, n, k) in enumerate(im2row_shapes(layers, batch, weights_as_A)):
+        w_std = (2.0 / k) ** 0.5
+        if weights_as_A:
+            kinds = dict(kindA="normal", kindB="absnormal", scaleA=w_std)
+        else:
+            kinds = dict(kindA="absnormal", kindB="normal", scaleB=w_std)
+        probs.append(Problem(f"{tag}_{i + 1:02d}", dtype, m, n, k, 1.0, 0.0, seed=base + i, **kinds))
+    return probs
