@@ -186,32 +186,36 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 
 // ---------------------------------------------------------------- 16-bit operand repack (aligned leading dimension)
 
-// one thread per 8 destination elements (one 16-byte store); the source column is read with scalar loads
+// One warp per column segment of up to 2048 elements: lanes walk it two elements at a time (two 2-byte loads, one
+// 4-byte store), so both the unaligned source column and the aligned destination column are touched in contiguous
+// 64 / 128-byte pieces.  Rows rows..ld_out-1 of the copy are zero.
+constexpr int REPACK_SEG = 2048;
+
 __global__ void __launch_bounds__(256)
 repack16_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld, uint16_t* __restrict__ dst,
                 int64_t ld_out) {
-    const int64_t vec_per_col = ld_out / 8;
-    const int64_t total = vec_per_col * cols;
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t j = idx / vec_per_col, i = (idx % vec_per_col) * 8;
-        const uint16_t* sp = src + i + j * ld;
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const uint32_t lo = (i + 2 * e < rows) ? sp[2 * e] : 0u;
-            const uint32_t hi = (i + 2 * e + 1 < rows) ? sp[2 * e + 1] : 0u;
-            w[e] = lo | (hi << 16);
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t segs = (ld_out + REPACK_SEG - 1) / REPACK_SEG;
+    for (int64_t u = warp; u < cols * segs; u += nwarps) {
+        const int64_t j = u / segs, i0 = (u % segs) * REPACK_SEG;
+        const int64_t i1 = min(ld_out, i0 + REPACK_SEG);
+        const uint16_t* sp = src + j * ld;
+        uint32_t* dp = reinterpret_cast<uint32_t*>(dst + j * ld_out);      // ld_out is a multiple of 8 elements
+        for (int64_t i = i0 + 2 * lane; i < i1; i += 64) {
+            const uint32_t lo = (i < rows) ? sp[i] : 0u;
+            const uint32_t hi = (i + 1 < rows) ? sp[i + 1] : 0u;
+            dp[i >> 1] = lo | (hi << 16);
         }
-        *reinterpret_cast<uint4*>(dst + i + j * ld_out) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,
                             cudaStream_t stream) {
-    const int64_t total = (ld_out / 8) * cols;
-    int64_t blocks = (total + 255) / 256;
-    const int64_t cap = (int64_t)sm_count() * 32;
+    const int64_t units = cols * ((ld_out + REPACK_SEG - 1) / REPACK_SEG);
+    int64_t blocks = (units + 7) / 8;                   // 8 warps per block
+    const int64_t cap = (int64_t)sm_count() * 64;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     repack16_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint16_t*)src, rows, cols, ld, (uint16_t*)dst, ld_out);

@@ -9,8 +9,9 @@
 //   loops L4/L5 + L6       -> tcgen05.mma 128 x BN x 16, issued by one thread; the C block lives in tensor
 //                             memory (TMEM) for the whole k loop, as the paper's C block lives in registers
 //   alpha / beta (Fig. 3)  -> epilogue warps read TMEM (tcgen05.ld), scale, and store column-major C
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2..5 = epilogue (one TMEM lane
-// quarter each).  Two accumulators in TMEM let the epilogue of one tile overlap the main loop of the next.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2..9 = epilogue (two per TMEM lane
+// quarter, alternating 32-column chunks).  Two to four accumulators in TMEM let the epilogue of one tile overlap the
+// main loops of the next ones.
 // Every mbarrier wait is bounded: on expiry the role records a code in the status word and all roles drain.
 #include <cuda.h>
 
@@ -21,6 +22,8 @@ namespace b200gemm {
 constexpr int TBM = 128;            // MMA M (TMEM lanes)
 constexpr int TBK = 64;             // k block: 64 x 2 bytes = one 128-byte swizzle row
 constexpr int UMMA_K = 16;          // k extent of one tcgen05.mma for 16-bit inputs
+constexpr int EPI_WARPS = 8;        // two epilogue warps per TMEM lane quarter, each taking every other 32-column chunk
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
 constexpr uint32_t SPIN_FAST = 4096;
 constexpr uint32_t SPIN_LIMIT = 1u << 24;   // then ~128 ns sleeps: gives up after a few seconds
 
@@ -126,15 +129,18 @@ template <int BN> struct TcCfg {
     static constexpr int A_BYTES = TBM * TBK * 2;
     static constexpr int B_BYTES = BN * TBK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int TMEM_COLS = 2 * BN;                       // two accumulators
-    static constexpr int STORE_BYTES = 4 * 2 * 32 * 32 * 4;       // per epilogue warp: two 32 x 32 fp32 staging tiles
+    // 227 KB of shared memory hold the operand ring plus the epilogue's staging tiles (one or two per warp)
+    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 5 : 6);
+    static constexpr int STORE_BUFS = (BN == 256) ? 1 : 2;
+    static constexpr int NACC = (BN == 256) ? 2 : 4;               // accumulators in flight between MMA and epilogue
+    static constexpr int TMEM_COLS = NACC * BN;                    // 512 columns per SM
+    static constexpr int STORE_BYTES = EPI_WARPS * STORE_BUFS * 32 * 32 * 4;   // per epilogue warp: STORE_BUFS 32 x 32 fp32 tiles
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STORE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 // A_MN: op(A) is contiguous along m in memory (transA = N); B_MN: op(B) contiguous along n (transB = T).
 template <int BN, bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
@@ -147,20 +153,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // layout: [stages][C staging tiles of the epilogue warps][barriers]
     float* store_stage = reinterpret_cast<float*>(smem_al + STAGES * Cfg::STAGE_BYTES);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + STAGES * Cfg::STAGE_BYTES + Cfg::STORE_BYTES);
-    // barrier slots: [0,S) full, [S,2S) empty, 2S+{0,1} tmem_full, 2S+{2,3} tmem_empty, then 2 words
+    // barrier slots: [0,S) full, [S,2S) empty, then NACC tmem_full, NACC tmem_empty, then 2 words
     const uint32_t bar0 = smem_base + STAGES * Cfg::STAGE_BYTES + Cfg::STORE_BYTES;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    constexpr int NACC = Cfg::NACC;
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 4);
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + NACC + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * STAGES + 2 * NACC);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        for (int a = 0; a < NACC; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -247,7 +254,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 decode(item, tm, tn, sp);
                 int64_t kbeg;
                 const int kb_n = kblocks_of(sp, kbeg);
-                const uint32_t acc = it & 1, aph = (it >> 1) & 1;
+                const uint32_t acc = it % NACC, aph = (it / NACC) & 1;
                 if (!mbar_wait(tempty_bar(acc), aph ^ 1, abort_flag, status,
                                STATUS_MARK | (ROLE_MMA << 16) | (BAR_TMEM_EMPTY << 8) | acc)) { ok = false; break; }
                 tc_fence_after();
@@ -277,19 +284,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
         }
     } else {
-        // ------------------------------------------------ epilogue (warps 2..5), TMEM lanes 32q .. 32q+31
+        // ------------------------------------------------ epilogue (warps 2..9), TMEM lanes 32q .. 32q+31
         // Lane = row of C.  Each 32-column chunk is read from TMEM, scaled, and then either written straight to
         // global memory (a warp stores 32 consecutive floats of one column per instruction) or, when C can be
         // addressed by TMA, transposed through a 32 x 32 staging tile in shared memory and written by an
         // asynchronous bulk tensor store, which also clips the tile at the matrix edge.
-        const int q = warp & 3;
-        float* stage = store_stage + (warp - 2) * (2 * 32 * 32);
+        const int q = warp & 3;                       // a warp may touch TMEM lanes 32*(warp % 4) .. +31 only
+        const int half = (warp - 2) >> 2;             // which of the two warps of this lane quarter
+        float* stage = store_stage + (warp - 2) * (Cfg::STORE_BUFS * 32 * 32);
         uint32_t it = 0, sbuf = 0;
         bool ok = true;
         for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
             int tm, tn, sp;
             decode(item, tm, tn, sp);
-            const uint32_t acc = it & 1, aph = (it >> 1) & 1;
+            const uint32_t acc = it % NACC, aph = (it / NACC) & 1;
             if (!mbar_wait(tfull_bar(acc), aph, abort_flag, status,
                            STATUS_MARK | (ROLE_EPI << 16) | (BAR_TMEM_FULL << 8) | acc)) { ok = false; break; }
             tc_fence_after();
@@ -301,11 +309,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int64_t ldo = raw ? m : ldc;
             // store_via_tma: 0 = direct stores, 1 = tmC maps C (2-D), 2 = tmC maps the split-k partials (3-D: m, n, split)
             const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
+            // this warp's chunks: c = half, half + 2, ... while the chunk starts inside the matrix
+            bool released = false;
+            auto release_acc = [&]() {      // the accumulator may be overwritten once this warp has read its last chunk
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+                released = true;
+            };
             if (row0 < m) {
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int c = half; c < BN / 32; c += 2) {
                     const int64_t col0 = n0 + c * 32;
                     if (col0 >= n) break;
+                    const bool last_chunk = (c + 2 >= BN / 32) || (col0 + 64 >= n);
                     uint32_t v[32];
                     tmem_ld32(tmem_base + acc * BN + c * 32 + ((uint32_t)(q * 32) << 16), v);
                     float* cp = out + row + col0 * ldo;
@@ -316,17 +333,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int j = 0; j < 32; ++j) c0[j] = (row < m && col0 + j < n) ? cp[j * ldo] : 0.0f;
                     }
                     tmem_ld_wait();
-                    float r[32];
+                    if (last_chunk) release_acc();
+                    float* r = reinterpret_cast<float*>(v);       // scaled in place
+                    if (!raw) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        r[j] = __uint_as_float(v[j]);
-                        if (!raw) {
+                        for (int j = 0; j < 32; ++j) {
                             r[j] *= alpha;
                             if (need_c0) r[j] = fmaf(beta, c0[j], r[j]);
                         }
                     }
                     if (via_tma) {
-                        if (lane == 0) bulk_wait_read<1>();      // the store that last used this staging tile has read it
+                        if (lane == 0) bulk_wait_read<Cfg::STORE_BUFS - 1>();   // the store that last used this staging tile has read it
                         __syncwarp();
                         float* st = stage + sbuf * (32 * 32);
 #pragma unroll
@@ -338,7 +355,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             else tma_store_2d(&tmC, smem_u32(st), (int32_t)row0, (int32_t)col0);
                             bulk_commit();
                         }
-                        sbuf ^= 1;
+                        sbuf = (sbuf + 1 == (uint32_t)Cfg::STORE_BUFS) ? 0 : sbuf + 1;
                     } else if (row < m) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
@@ -346,9 +363,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (!released) release_acc();
         }
         if (lane == 0) bulk_wait_all();       // staging tiles must outlive the stores that read them
     }
@@ -483,7 +498,7 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     const int64_t items = tiles_m * tiles_n * ks.splits;
     const int grid = (int)(items < sm_count() ? items : sm_count());
     cfg->tile_m = TBM; cfg->tile_n = BN; cfg->tile_k = TBK; cfg->stages = Cfg::STAGES; cfg->grid = grid;
-    kern<<<grid, 192, Cfg::SMEM_BYTES, a.stream>>>(tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc, (int)tiles_m,
+    kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, a.stream>>>(tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc, (int)tiles_m,
                                                    (int)tiles_n, ks.splits, ks.chunk,
                                                    ks.splits > 1 ? partials : nullptr,
                                                    instr_desc(a.dtype, A_MN, B_MN, BN), a.status);
