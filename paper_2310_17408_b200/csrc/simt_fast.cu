@@ -274,8 +274,8 @@ bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb) {
 template <int BM, int BN, int WM, int WN, int MINB, bool AK, bool BKC, int VA, int VB>
 static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg) {
     int64_t tiles_m = (a.m + BM - 1) / BM, tiles_n = (a.n + BN - 1) / BN;
-    if (tiles_m * tiles_n > 0x7FFFFFFFLL || tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF)
-        return cudaErrorInvalidConfiguration;
+    if (tiles_m * tiles_n > 0x7FFFFFFFLL || tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF / 16)
+        return cudaErrorInvalidConfiguration;       // tile indices are 32-bit in the kernel (groups of 16 tile rows)
     dim3 grid((unsigned)(tiles_m * tiles_n), 1, (unsigned)ks.splits);
     cfg->tile_m = BM; cfg->tile_n = BN; cfg->tile_k = BK; cfg->stages = 2;
     cfg->grid = (int32_t)(tiles_m * tiles_n * ks.splits);

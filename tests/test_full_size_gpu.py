@@ -98,3 +98,29 @@ def test_vgg16_and_paper_orientation_shapes():
         im2row_problems("vgg16", weights_as_A=False)[-2:]
     for i, p in enumerate(cases):
         run_and_check(p, seed=i)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_BF16])
+def test_result_with_more_than_2_31_entries(dtype):
+    # C has 32768 x 65600 = 2.15e9 entries (8.6 GB): every index into C must be 64-bit.  beta = 0, so C is
+    # allocated on the device only; sampled columns (first, last, around the 2^31-entry mark) are checked exactly.
+    import torch
+    from workloads import make_matrix
+    from gpu_util import to_device
+    m, n, k = 32768, 65600, 32
+    A = make_matrix(m, k, kind="int", seed=77, matrix_id=0, dtype=dtype)
+    B = make_matrix(k, n, kind="int", seed=77, matrix_id=1, dtype=dtype)
+    dA, dB = to_device(A), to_device(B)
+    dC = torch.full((m * n,), float("nan"), dtype=torch.float32, device="cuda")
+    rc = g.gemm(dtype, "N", "N", m, n, k, 1.0, dA.data_ptr(), m, dB.data_ptr(), k, 0.0, dC.data_ptr(), m,
+                torch.cuda.current_stream().cuda_stream)
+    assert rc == 0, g.gemm_status_string(rc)
+    assert g.gemm_poll_status() == 0
+    cols = [0, 1, 255, 256, 65535, 65536, 65537, n - 257, n - 2, n - 1]       # 65536 * 32768 = 2^31 entries
+    ref = A.as_f64() @ B.as_f64()[:, cols]
+    got = torch.stack([dC[j * m:(j + 1) * m] for j in cols], dim=1).cpu().numpy().astype(np.float64)
+    assert np.array_equal(got, ref)
+    # nothing left unwritten anywhere: no NaN survives in the whole result
+    assert not bool(torch.isnan(dC).any())
+    del dC
+    torch.cuda.empty_cache()
