@@ -429,7 +429,8 @@ def run_cuda(args, problems, workload_name):
             host_step()
         barrier()
         e2e_s = time.perf_counter() - t0
-        h2d = sum(h[0].numel() * h[0].element_size() + h[1].numel() * h[1].element_size() + h[2].numel() * 4 for h in host)
+        h2d = sum(h[0].numel() * h[0].element_size() + h[1].numel() * h[1].element_size() +
+                  (h[2].numel() * 4 if p.beta != 0.0 else 0) for h, p in zip(host, problems))   # C goes in only when beta != 0
         d2h = sum(h[2].numel() * 4 for h in host)
         e2e = (e2e_s / e2e_steps, h2d, d2h, e2e_steps)
 

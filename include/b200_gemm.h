@@ -91,9 +91,12 @@ int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k,
          float beta, void* C, int64_t ldc, void* stream);
 
 /*
- * gemm_host — the same operation on HOST buffers (pageable or pinned): allocates device buffers
- * from the stream-ordered pool, copies A, B (and C if beta != 0) to the device, runs gemm(), copies
- * C back and synchronises `stream` before returning.  Leading dimensions and layout as for gemm().
+ * gemm_host — the same operation on HOST buffers (pinned memory for full speed; pageable works but serialises).
+ * Allocates device buffers from the stream-ordered pool, then moves column panels of op(B) and C through a
+ * three-stream pipeline (copy in / multiply on `stream` / copy out), so that transfers overlap the arithmetic,
+ * and synchronises `stream` before returning.  Only the m x n window of C is transferred: C is copied in only when
+ * beta != 0, and rows m..ldc-1 of the host array are never touched.  Leading dimensions and layout as for gemm().
+ * Calls from several host threads on one device share the copy streams and are therefore serialised by them.
  */
 int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k,
               float alpha, const void* A_host, int64_t lda, const void* B_host, int64_t ldb,

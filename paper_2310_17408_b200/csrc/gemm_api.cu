@@ -331,6 +331,20 @@ int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, f
     return run_gemm(a, st);
 }
 
+// copy a rows x cols window of a column-major matrix (element size es, leading dimension ld on both sides)
+static cudaError_t copy_window(void* dst, const void* src, int64_t rows, int64_t cols, int64_t ld, int es,
+                               cudaMemcpyKind kind, cudaStream_t s) {
+    if (rows == 0 || cols == 0) return cudaSuccess;
+    if (rows == ld) return cudaMemcpyAsync(dst, src, (size_t)rows * cols * es, kind, s);
+    return cudaMemcpy2DAsync(dst, (size_t)ld * es, src, (size_t)ld * es, (size_t)rows * es, (size_t)cols, kind, s);
+}
+
+struct HostPipe {          // per device: the two copy streams of gemm_host
+    bool init = false;
+    cudaStream_t in = nullptr, out = nullptr;
+};
+static HostPipe g_pipe[MAX_DEVICES];
+
 int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha, const void* A_host,
               int64_t lda, const void* B_host, int64_t ldb, float beta, void* C_host, int64_t ldc, void* stream) {
     bool ta = false, tb = false;
@@ -338,42 +352,105 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     if (bad) return bad;
     if (m == 0 || n == 0) return GEMM_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    {   // keep freed staging buffers in the stream-ordered pool instead of returning them at every synchronise
-        static thread_local int pool_tuned_dev = -1;
-        int dev = 0;
-        cudaMemPool_t pool;
-        if (cudaGetDevice(&dev) == cudaSuccess && dev != pool_tuned_dev &&
-            cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
-            uint64_t keep = ~0ull;
-            cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
-            pool_tuned_dev = dev;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return GEMM_ERR_LAUNCH;
+    HostPipe* pipe = &g_pipe[dev];
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!pipe->init) {
+            // keep freed staging buffers in the stream-ordered pool instead of returning them at every synchronise
+            cudaMemPool_t pool;
+            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+                uint64_t keep = ~0ull;
+                cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+            }
+            if (cudaStreamCreateWithFlags(&pipe->in, cudaStreamNonBlocking) != cudaSuccess ||
+                cudaStreamCreateWithFlags(&pipe->out, cudaStreamNonBlocking) != cudaSuccess)
+                return fail_launch(cudaGetLastError());
+            pipe->init = true;
         }
     }
     const int es = elem_size(dtype);
     const bool needs_ab = (k > 0 && alpha != 0.0f);
-    const size_t a_bytes = needs_ab ? (size_t)lda * (ta ? m : k) * es : 0;
+    const int64_t a_rows = ta ? k : m, a_cols = ta ? m : k;
+    const size_t a_bytes = needs_ab ? (size_t)lda * a_cols * es : 0;
     const size_t b_bytes = needs_ab ? (size_t)ldb * (tb ? k : n) * es : 0;
     const size_t c_bytes = (size_t)ldc * n * sizeof(float);
+
+    // Column panels of C (and of op(B)) flow through a three-stream pipeline: panel p+1 is copied in while panel p
+    // is multiplied and panel p-1 is copied out.  Small problems use one panel.
+    const double traffic = (double)b_bytes + (double)m * n * 4.0 * (beta != 0.0f ? 2.0 : 1.0);
+    int64_t panel = n;
+    if (traffic > 32e6 && n >= 1024) {
+        int64_t panels = (int64_t)(traffic / 48e6) + 1;
+        if (panels > 16) panels = 16;
+        panel = round_up(ceil_div(n, panels), 256);
+    }
+    const int np = (int)ceil_div(n, panel);
+
     void *dA = nullptr, *dB = nullptr, *dC = nullptr;
     cudaError_t e = cudaSuccess;
     int rc = GEMM_OK;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess && r != cudaSuccess) e = r; return r == cudaSuccess; };
-    if (a_bytes) chk(cudaMallocAsync(&dA, a_bytes, s));
-    if (b_bytes) chk(cudaMallocAsync(&dB, b_bytes, s));
-    chk(cudaMallocAsync(&dC, c_bytes, s));
+    const int nev = 2 * np + 3;
+    cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[nev];
+    if (!ev) return GEMM_ERR_LAUNCH;
+    int made = 0;
+    for (; made < nev; ++made)
+        if (!chk(cudaEventCreateWithFlags(&ev[made], cudaEventDisableTiming))) break;
+    cudaEvent_t ev_alloc = ev[0], ev_a = ev[1], ev_done = ev[2];
+
     if (e == cudaSuccess) {
-        if (a_bytes) chk(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, s));
-        if (b_bytes) chk(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, s));
-        // C travels whole (padding rows included) so that the copy back leaves the host padding as it was
-        chk(cudaMemcpyAsync(dC, C_host, c_bytes, cudaMemcpyHostToDevice, s));
+        if (a_bytes) chk(cudaMallocAsync(&dA, a_bytes, s));
+        if (b_bytes) chk(cudaMallocAsync(&dB, b_bytes, s));
+        chk(cudaMallocAsync(&dC, c_bytes, s));
     }
-    if (e == cudaSuccess)
-        rc = gemm(dtype, transA, transB, m, n, k, alpha, dA, lda, dB, ldb, beta, dC, ldc, stream);
-    if (e == cudaSuccess && rc == GEMM_OK) chk(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, s));
+    if (e == cudaSuccess) {
+        chk(cudaEventRecord(ev_alloc, s));                       // the copy streams start after the allocations
+        chk(cudaStreamWaitEvent(pipe->in, ev_alloc, 0));
+        chk(cudaStreamWaitEvent(pipe->out, ev_alloc, 0));
+        if (a_bytes) chk(copy_window(dA, A_host, a_rows, a_cols, lda, es, cudaMemcpyHostToDevice, pipe->in));
+        chk(cudaEventRecord(ev_a, pipe->in));
+        chk(cudaStreamWaitEvent(s, ev_a, 0));
+    }
+    for (int p = 0; p < np && e == cudaSuccess && rc == GEMM_OK; ++p) {
+        const int64_t j0 = (int64_t)p * panel, cols = (n - j0 < panel) ? n - j0 : panel;
+        cudaEvent_t ev_in = ev[3 + 2 * p], ev_mul = ev[4 + 2 * p];
+        const char* hB = static_cast<const char*>(B_host);
+        char* dBp = static_cast<char*>(dB);
+        const size_t b_off = needs_ab ? (tb ? (size_t)j0 * es : (size_t)j0 * ldb * es) : 0;
+        if (needs_ab) {
+            if (tb) chk(copy_window(dBp + b_off, hB + b_off, cols, k, ldb, es, cudaMemcpyHostToDevice, pipe->in));
+            else chk(copy_window(dBp + b_off, hB + b_off, k, cols, ldb, es, cudaMemcpyHostToDevice, pipe->in));
+        }
+        const size_t c_off = (size_t)j0 * ldc * sizeof(float);
+        // only the m x cols window of C travels: the host's padding rows are never touched
+        if (beta != 0.0f)
+            chk(copy_window(static_cast<char*>(dC) + c_off, static_cast<const char*>(C_host) + c_off, m, cols, ldc, 4,
+                            cudaMemcpyHostToDevice, pipe->in));
+        chk(cudaEventRecord(ev_in, pipe->in));
+        chk(cudaStreamWaitEvent(s, ev_in, 0));
+        if (e != cudaSuccess) break;
+        rc = gemm(dtype, transA, transB, m, cols, k, alpha, dA, lda, needs_ab ? dBp + b_off : nullptr, ldb, beta,
+                  static_cast<char*>(dC) + c_off, ldc, stream);
+        if (rc != GEMM_OK) break;
+        chk(cudaEventRecord(ev_mul, s));
+        chk(cudaStreamWaitEvent(pipe->out, ev_mul, 0));
+        chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols, ldc, 4,
+                        cudaMemcpyDeviceToHost, pipe->out));
+    }
+    if (made > 2) {
+        cudaEventRecord(ev_done, pipe->out);                     // the caller's stream rejoins both copy streams
+        cudaStreamWaitEvent(s, ev_done, 0);
+        cudaEventRecord(ev_a, pipe->in);
+        cudaStreamWaitEvent(s, ev_a, 0);
+    }
     if (dA) cudaFreeAsync(dA, s);
     if (dB) cudaFreeAsync(dB, s);
     if (dC) cudaFreeAsync(dC, s);
     chk(cudaStreamSynchronize(s));
+    for (int i = 0; i < made; ++i) cudaEventDestroy(ev[i]);
+    delete[] ev;
     if (e != cudaSuccess) return fail_launch(e);
     return rc;
 }

@@ -201,3 +201,23 @@ def test_bounded_wait_expiry_is_reported_and_context_survives():
     A, B, C0 = p.operands()
     C, cfg = run_problem(p, A, B, C0)
     check_against_oracle(p, A, B, C0, C, integer=True)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_BF16])
+def test_gemm_host_pipelined_panels_match_oracle(dtype):
+    # host-buffer entry point: several column panels in flight (large n), padded leading dimensions, both B layouts
+    kind = "uniform" if dtype == DTYPE_F32 else "normal"
+    cases = [(300, 9000, 700, "N", "N", 1.5, 0.5, (4, 8, 4)),      # multi-panel, C read and written
+             (260, 8200, 1100, "T", "T", 1.0, 0.0, (8, 8, 2)),     # multi-panel, strided panels of B, C write-only
+             (100, 90, 70, "N", "T", -1.0, 1.0, (1, 3, 1))]        # single panel
+    for (m, n, k, ta, tb, alpha, beta, pad) in cases:
+        p = problem(dtype, m, n, k, ta, tb, alpha, beta, kind, pad, seed=m)
+        A, B, C0 = p.operands()
+        C = C0.copy()
+        if beta == 0.0:
+            C.window()[:] = np.nan                                  # must be overwritten, never read
+        rc = g.gemm_host(dtype, ta, tb, m, n, k, alpha, A.buf.ctypes.data, A.ld, B.buf.ctypes.data, B.ld, beta,
+                         C.buf.ctypes.data, C.ld, torch.cuda.current_stream().cuda_stream)
+        assert rc == 0, g.gemm_status_string(rc)
+        assert C.padding_intact()
+        check_against_oracle(p, A, B, C0, C)
