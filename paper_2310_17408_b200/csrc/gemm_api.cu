@@ -387,12 +387,21 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
         panel = round_up(ceil_div(n, panels), 256);
     }
     const int np = (int)ceil_div(n, panel);
+    // While A itself is still arriving, the first column panel is computed in row panels of op(A): each needs
+    // only its own rows of A, so the multiplication starts long before the whole of A is on the device.
+    int64_t rpanel = m;
+    if (np > 1 && needs_ab && (double)a_bytes > 32e6 && m >= 1024) {
+        int64_t rp = (int64_t)((double)a_bytes / 32e6) + 1;
+        if (rp > 8) rp = 8;
+        rpanel = round_up(ceil_div(m, rp), 256);
+    }
+    const int nr = (int)ceil_div(m, rpanel);
 
     void *dA = nullptr, *dB = nullptr, *dC = nullptr;
     cudaError_t e = cudaSuccess;
     int rc = GEMM_OK;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess && r != cudaSuccess) e = r; return r == cudaSuccess; };
-    const int nev = 2 * np + 3;
+    const int nev = 2 * np + 3 + nr;
     cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[nev];
     if (!ev) return GEMM_ERR_LAUNCH;
     int made = 0;
@@ -409,9 +418,11 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
         chk(cudaEventRecord(ev_alloc, s));                       // the copy streams start after the allocations
         chk(cudaStreamWaitEvent(pipe->in, ev_alloc, 0));
         chk(cudaStreamWaitEvent(pipe->out, ev_alloc, 0));
-        if (a_bytes) chk(copy_window(dA, A_host, a_rows, a_cols, lda, es, cudaMemcpyHostToDevice, pipe->in));
-        chk(cudaEventRecord(ev_a, pipe->in));
-        chk(cudaStreamWaitEvent(s, ev_a, 0));
+        if (a_bytes && nr == 1) {
+            chk(copy_window(dA, A_host, a_rows, a_cols, lda, es, cudaMemcpyHostToDevice, pipe->in));
+            chk(cudaEventRecord(ev_a, pipe->in));
+            chk(cudaStreamWaitEvent(s, ev_a, 0));
+        }
     }
     for (int p = 0; p < np && e == cudaSuccess && rc == GEMM_OK; ++p) {
         const int64_t j0 = (int64_t)p * panel, cols = (n - j0 < panel) ? n - j0 : panel;
@@ -431,9 +442,27 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
         chk(cudaEventRecord(ev_in, pipe->in));
         chk(cudaStreamWaitEvent(s, ev_in, 0));
         if (e != cudaSuccess) break;
-        rc = gemm(dtype, transA, transB, m, cols, k, alpha, dA, lda, needs_ab ? dBp + b_off : nullptr, ldb, beta,
-                  static_cast<char*>(dC) + c_off, ldc, stream);
-        if (rc != GEMM_OK) break;
+        if (p == 0 && nr > 1) {
+            for (int r = 0; r < nr && e == cudaSuccess && rc == GEMM_OK; ++r) {
+                const int64_t i0 = (int64_t)r * rpanel, rows = (m - i0 < rpanel) ? m - i0 : rpanel;
+                // rows i0.. of op(A): a row window of the stored matrix (transA = N) or whole columns of it (T)
+                const size_t a_off = ta ? (size_t)i0 * lda * es : (size_t)i0 * es;
+                char* dAp = static_cast<char*>(dA) + a_off;
+                const char* hAp = static_cast<const char*>(A_host) + a_off;
+                if (ta) chk(copy_window(dAp, hAp, k, rows, lda, es, cudaMemcpyHostToDevice, pipe->in));
+                else chk(copy_window(dAp, hAp, rows, k, lda, es, cudaMemcpyHostToDevice, pipe->in));
+                cudaEvent_t ev_row = ev[3 + 2 * np + r];
+                chk(cudaEventRecord(ev_row, pipe->in));
+                chk(cudaStreamWaitEvent(s, ev_row, 0));
+                if (e != cudaSuccess) break;
+                rc = gemm(dtype, transA, transB, rows, cols, k, alpha, dAp, lda, dBp + b_off, ldb, beta,
+                          static_cast<char*>(dC) + c_off + (size_t)i0 * sizeof(float), ldc, stream);
+            }
+        } else {
+            rc = gemm(dtype, transA, transB, m, cols, k, alpha, dA, lda, needs_ab ? dBp + b_off : nullptr, ldb, beta,
+                      static_cast<char*>(dC) + c_off, ldc, stream);
+        }
+        if (rc != GEMM_OK || e != cudaSuccess) break;
         chk(cudaEventRecord(ev_mul, s));
         chk(cudaStreamWaitEvent(pipe->out, ev_mul, 0));
         chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols, ldc, 4,

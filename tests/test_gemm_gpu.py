@@ -209,7 +209,9 @@ def test_gemm_host_pipelined_panels_match_oracle(dtype):
     kind = "uniform" if dtype == DTYPE_F32 else "normal"
     cases = [(300, 9000, 700, "N", "N", 1.5, 0.5, (4, 8, 4)),      # multi-panel, C read and written
              (260, 8200, 1100, "T", "T", 1.0, 0.0, (8, 8, 2)),     # multi-panel, strided panels of B, C write-only
-             (100, 90, 70, "N", "T", -1.0, 1.0, (1, 3, 1))]        # single panel
+             (100, 90, 70, "N", "T", -1.0, 1.0, (1, 3, 1)),        # single panel
+             (4500, 3000, 2100, "N", "N", 1.0, 0.5, (4, 0, 4)),    # A large enough to arrive in row panels
+             (4400, 2900, 2050, "T", "N", 1.0, 0.0, (8, 8, 0))]    # same with A stored transposed
     for (m, n, k, ta, tb, alpha, beta, pad) in cases:
         p = problem(dtype, m, n, k, ta, tb, alpha, beta, kind, pad, seed=m)
         A, B, C0 = p.operands()
