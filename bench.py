@@ -95,8 +95,10 @@ def fp32_alu_peak_tflops(sm_mhz: float) -> float:
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only queries)."""
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """Samples nvidia-smi clocks and throttle reasons (read-only queries).  It is started well before the timed
+    region, because nvidia-smi takes a moment to produce its first line; only samples whose timestamp falls
+    inside the timed window are used."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -109,7 +111,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -117,9 +119,9 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -129,7 +131,10 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in self.lines:
+        for seen, line in self.lines:
+            # a sample is attributed to the moment its line arrived (nvidia-smi prints as it samples)
+            if t_begin is not None and not (t_begin <= seen <= t_end + 0.05):
+                continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
                 continue
@@ -141,12 +146,9 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        # samples under load: the upper half of the power readings
-        cut = statistics.median(power)
-        loaded = [c for c, p in zip(sm, power) if p >= cut] or sm
-        return {"sm_mhz": statistics.median(loaded), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm), "power_w_max": max(power)}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples inside the timed region"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_median": statistics.median(power), "power_w_max": max(power)}
 
 
 def rank_info():
@@ -317,22 +319,33 @@ def run_cuda(args, problems, workload_name):
             launches += g.gemm_last_config()["launches"]
 
     # ---- device-resident timing
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         one_step()
     barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     events = [[] for _ in problems]
     launches = 0
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    wall_begin = time.time()
     t_begin.record()
     for _ in range(args.steps):
         one_step(events)
     t_end.record()
     barrier()
+    wall_end = time.time()
     total_ms = t_begin.elapsed_time(t_end)
-    clocks = sampler.stop()
+    if wall_end - wall_begin >= 0.4:
+        clocks = sampler.stop(wall_begin, wall_end)
+    else:
+        # a timed region this short sees no nvidia-smi sample: keep running the same steps for 0.6 s and sample there
+        w0 = time.time()
+        while time.time() - w0 < 0.6:
+            one_step()
+        torch.cuda.synchronize()
+        clocks = sampler.stop(w0, time.time())
+        clocks["window"] = "0.6 s of the same steps run right after the (shorter) timed region"
     timed_launches = launches
     if g.gemm_poll_status() != 0:
         raise RuntimeError(f"device status {hex(g.gemm_status_detail())}")
@@ -495,7 +508,7 @@ def run_cuda(args, problems, workload_name):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS))
