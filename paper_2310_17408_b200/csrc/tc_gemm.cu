@@ -165,6 +165,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    // let the next kernel of the stream start its own set-up as soon as SMs free up (it waits before touching memory)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < NACC; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), EPI_WARPS); }
@@ -181,6 +183,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: everything above (barrier and TMEM set-up) may overlap the tail of the
+    // previous kernel in the stream; nothing below touches global memory before that kernel has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int64_t items = (int64_t)tiles_m * tiles_n * splits;
     constexpr int GROUP = 16;
@@ -501,11 +506,21 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     const int64_t items = tiles_m * tiles_n * ks.splits;
     const int grid = (int)(items < sm_count() ? items : sm_count());
     cfg->tile_m = TBM; cfg->tile_n = BN; cfg->tile_k = TBK; cfg->stages = Cfg::STAGES; cfg->grid = grid;
-    kern<<<grid, TC_THREADS, Cfg::SMEM_BYTES, a.stream>>>(tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc, (int)tiles_m,
-                                                   (int)tiles_n, ks.splits, ks.chunk,
-                                                   ks.splits > 1 ? partials : nullptr,
-                                                   instr_desc(a.dtype, A_MN, B_MN, BN), a.status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)grid);
+    lc.blockDim = dim3(TC_THREADS);
+    lc.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    lc.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // pairs with griddepcontrol.wait in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
+                                        (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
+                                        ks.splits > 1 ? partials : (float*)nullptr,
+                                        instr_desc(a.dtype, A_MN, B_MN, BN), a.status);
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <bool A_MN, bool B_MN>
