@@ -151,6 +151,9 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
     __shared__ __align__(16) float As[2][BK * (BM + PAD)];
     __shared__ __align__(16) float Bs[2][BK * (BN + PAD)];
 
+    // programmatic dependent launch: the next kernel of the stream may be scheduled once every CTA of this one
+    // has started; it waits (griddepcontrol.wait) before it touches global memory, as this kernel does below
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int t = threadIdx.x;
     const int warp = t >> 5, lane = t & 31;
     const int wm = warp % WARPS_M, wn = warp / WARPS_M;
@@ -202,6 +205,7 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
         }
     };
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the previous kernel's results are visible from here on
     if (ktiles > 0) {
         gload(0);
         LA::store(ra, As[0], t);
@@ -279,10 +283,20 @@ static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gem
     dim3 grid((unsigned)(tiles_m * tiles_n), 1, (unsigned)ks.splits);
     cfg->tile_m = BM; cfg->tile_n = BN; cfg->tile_k = BK; cfg->stages = 2;
     cfg->grid = (int32_t)(tiles_m * tiles_n * ks.splits);
-    simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB><<<grid, WM * WN * 32, 0, a.stream>>>(
-        a.m, a.n, a.k, a.alpha, (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
-        (int)tiles_m, (int)tiles_n, ks.chunk, ks.splits > 1 ? partials : nullptr);
-    return cudaGetLastError();
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = dim3(WM * WN * 32);
+    lc.stream = a.stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // pairs with griddepcontrol.wait in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    cudaError_t le = cudaLaunchKernelEx(&lc, simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB>, a.m, a.n, a.k, a.alpha,
+                                        (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
+                                        (int)tiles_m, (int)tiles_n, ks.chunk,
+                                        ks.splits > 1 ? partials : (float*)nullptr);
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <bool AK, bool BKC, int VA, int VB>
