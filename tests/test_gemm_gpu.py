@@ -223,3 +223,85 @@ def test_gemm_host_pipelined_panels_match_oracle(dtype):
         assert rc == 0, g.gemm_status_string(rc)
         assert C.padding_intact()
         check_against_oracle(p, A, B, C0, C)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_BF16])
+def test_concurrent_host_threads_on_their_own_streams(dtype):
+    # calls from different host threads on different streams are independent when no workspace is registered
+    import threading
+    drop_workspace()
+    kind = "uniform" if dtype == DTYPE_F32 else "normal"
+    results, errors = {}, []
+
+    def worker(idx):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            p = problem(dtype, 260 + 64 * idx, 390, 700 + 100 * idx, "N", "T" if idx % 2 else "N", 1.5, 0.5, kind, (0, 0, 0),
+                        seed=50 + idx)
+            A, B, C0 = p.operands()
+            from gpu_util import to_device
+            with torch.cuda.stream(stream):
+                dA, dB, dC = to_device(A), to_device(B), to_device(C0)
+                for _ in range(20):                      # keep both streams busy at the same time
+                    dC.copy_(torch.from_numpy(C0.buf), non_blocking=False)
+                    rc = g.gemm(dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), A.ld, dB.data_ptr(),
+                                B.ld, p.beta, dC.data_ptr(), C0.ld, stream.cuda_stream)
+                    assert rc == 0
+                stream.synchronize()
+                from workloads import Matrix
+                results[idx] = (p, A, B, C0, Matrix(dC.cpu().numpy(), p.m, p.n, C0.ld, DTYPE_F32))
+        except Exception as exc:      # surfaced in the main thread
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(3)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert g.gemm_poll_status() == 0
+    for idx, (p, A, B, C0, C) in results.items():
+        check_against_oracle(p, A, B, C0, C)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_F16, DTYPE_BF16])
+def test_nan_and_inf_in_operands_stay_in_their_rows_and_columns(dtype):
+    # a NaN in row 5 of A poisons row 5 of C, an Inf in column 7 of B makes column 7 of C non-finite; nothing else changes
+    from gpu_util import to_device
+    from workloads import Matrix, encode_bf16, encode_f16
+    m, n, k = 200, 300, 130
+    p = problem(dtype, m, n, k, "N", "N", 1.0, 0.0, "int", (0, 0, 0), seed=4)
+    A, B, C0 = p.operands()
+    clean, _ = run_problem(p, A, B, C0)
+    A2, B2 = A.copy(), B.copy()
+    nan = {DTYPE_F32: np.float32("nan"), DTYPE_F16: encode_f16(np.array([np.nan]))[0], DTYPE_BF16: encode_bf16(np.array([np.nan]))[0]}[dtype]
+    inf = {DTYPE_F32: np.float32("inf"), DTYPE_F16: encode_f16(np.array([np.inf]))[0], DTYPE_BF16: encode_bf16(np.array([np.inf]))[0]}[dtype]
+    A2.window()[5, 17] = nan
+    B2.window()[40, 7] = inf
+    dirty, _ = run_problem(p, A2, B2, C0)
+    d, c = dirty.window(), clean.window()
+    assert np.all(np.isnan(d[5, :]))
+    assert not np.any(np.isfinite(d[:, 7]))
+    mask = np.ones((m, n), dtype=bool)
+    mask[5, :] = False
+    mask[:, 7] = False
+    assert np.array_equal(d[mask], c[mask])
+
+
+def test_fp16_subnormal_inputs_are_not_flushed():
+    # binary16 subnormals (multiples of 2^-24 below 2^-14) times small integers: every product and sum is exact in
+    # fp32, so the tensor-core result must equal the fp64 oracle exactly if subnormal inputs are honoured
+    from workloads import Matrix, encode_f16
+    m, n, k = 128, 128, 64
+    rng = np.random.default_rng(3)
+    a = rng.integers(1, 1000, (m, k)).astype(np.float64) * 2.0 ** -24          # all subnormal in binary16
+    b = rng.integers(-4, 5, (k, n)).astype(np.float64)
+    A = Matrix(encode_f16(a.T.ravel()).copy(), m, k, m, DTYPE_F16)              # column-major buffers
+    B = Matrix(encode_f16(b.T.ravel()).copy(), k, n, k, DTYPE_F16)
+    assert np.array_equal(A.as_f64(), a) and np.all(np.abs(a) < 2.0 ** -14)
+    C0 = make_matrix(m, n, kind="zeros", seed=0, matrix_id=2)
+    p = Problem("sub", DTYPE_F16, m, n, k, 1.0, 0.0)
+    C, cfg = run_problem(p, A, B, C0)
+    assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
+    assert np.array_equal(C.window().astype(np.float64), a @ b)
