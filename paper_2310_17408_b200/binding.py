@@ -35,7 +35,7 @@ class GemmConfig(ctypes.Structure):
 
 def _load() -> ctypes.CDLL:
     if not _LIB_PATH.exists():
-        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2310_17408_b200.build` "
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python paper_2310_17408_b200/build.py` "
                           "(nvcc, sm_100a); this package has no CPU or library fallback")
     lib = ctypes.CDLL(str(_LIB_PATH), mode=ctypes.RTLD_LOCAL)
     i64, vp, ci, cf, cc = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_char

@@ -10,6 +10,14 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200, sm_100a)")
+    # a fresh checkout has no built library yet: build it (nvcc cross-compiles without a GPU) before collection
+    lib = os.path.join(ROOT, "paper_2310_17408_b200", "libb200gemm.so")
+    if not os.path.exists(lib):
+        import importlib.util
+        spec = importlib.util.spec_from_file_location("b200gemm_build", os.path.join(ROOT, "paper_2310_17408_b200", "build.py"))
+        mod = importlib.util.module_from_spec(spec)
+        spec.loader.exec_module(mod)
+        mod.build()
 
 
 def pytest_collection_modifyitems(config, items):
