@@ -466,7 +466,7 @@ def run_cuda(args, problems, workload_name):
                        "bound": bound, "frac": amount / (cold_ms * 1e-3) / peak, "frac_in_step": achieved / peak,
                        "ms_graph": graph_ms, "frac_graph": (amount / (graph_ms * 1e-3) / peak) if graph_ms else None,
                        "host_us_per_call": host_us, "operand_sets": nsets, "calls": reps, "kernel": configs[i]["kernel"],
-                       "tile": [configs[i]["tile_m"], configs[i]["tile_n"]], "split_k": configs[i]["split_k"],
+                       "tile": [configs[i]["tile_m"], configs[i]["tile_n"]], "split_k": configs[i]["split_k"], "tail_split": configs[i].get("tail_split", 0),
                        "launches": configs[i]["launches"]})
         if avg > dom_ms:
             dom_ms, dominant = avg, (p, bound, peak, unit, achieved, configs[i])

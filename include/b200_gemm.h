@@ -59,7 +59,7 @@ typedef struct {
     int32_t vector_b;
     int32_t launches;      /* kernels enqueued by the call (main + reduction / scaling)      */
     int32_t repacked;      /* bit 0: A was copied to an aligned layout first, bit 1: B       */
-    int32_t reserved;
+    int32_t tail_split;    /* fp32: k ranges each tile of the last, partly filled wave was cut into (0 = not used) */
 } gemm_config_t;
 
 /*
@@ -148,7 +148,7 @@ int gemm_last_config(gemm_config_t* out);
 
 /* tests / benchmarks: force a kernel family (GEMM_KERNEL_AUTO restores the selector).  A forced family
  * that cannot run the problem (wrong dtype, alignment) falls back to the selector's choice.
- * gemm_force_tile: force tile_n (0 = auto) and split_k (0 = auto) of the chosen family. */
+ * gemm_force_tile: force the tile (0 = auto) and split_k (0 = auto; 1 = no split of any kind) of the chosen family. */
 int gemm_force_kernel(int kernel);
 int gemm_force_tile(int tile_m, int tile_n, int split_k);
 

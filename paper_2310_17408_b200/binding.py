@@ -27,10 +27,10 @@ GEMM_STATIC_SCRATCH_BYTES = 8 << 20
 class GemmConfig(ctypes.Structure):
     _fields_ = [(name, ctypes.c_int32) for name in
                 ("kernel", "tile_m", "tile_n", "tile_k", "split_k", "stages", "grid", "vector_a", "vector_b",
-                 "launches", "repacked", "reserved")]
+                 "launches", "repacked", "tail_split")]
 
     def as_dict(self):
-        return {name: getattr(self, name) for name, _ in self._fields_ if name != "reserved"}
+        return {name: getattr(self, name) for name, _ in self._fields_}
 
 
 def _load() -> ctypes.CDLL:

@@ -28,6 +28,7 @@ static thread_local gemm_config_t t_last_cfg = {};
 static thread_local int t_last_cuda_error = 0;
 static int g_force_kernel = GEMM_KERNEL_AUTO;
 static int g_force_tile_m = 0, g_force_tile_n = 0, g_force_split = 0;
+static bool g_no_tail_split = false;   // gemm_force_tile(.., split_k = 1) also switches the tail split off
 static uint32_t g_last_detail = 0;
 
 static DeviceState* device_state() {
@@ -66,6 +67,8 @@ struct Plan {
     int64_t lda_p, ldb_p;     // leading dimensions of the repacked operands
     size_t ws_partials;       // bytes
     size_t ws_total;
+    int tail_first, tail_splits;   // fp32 tail split (tail_splits <= 1: off)
+    int64_t tail_chunk;
 };
 
 // k partition: `want` splits of a multiple of `quantum`, no empty split
@@ -96,7 +99,16 @@ static void plan_simt(const GemmArgs& a, int sms, size_t ws_avail, Plan* p) {
         const double tiles = (double)tm * tn;
         const double slots = sms * ctas_per_sm[t];
         const double waves = tiles / slots;
-        const double full = (double)ceil_div((int64_t)tiles, (int64_t)slots);
+        double full = (double)ceil_div((int64_t)tiles, (int64_t)slots);
+        {   // a partly filled last wave that can be cut along k (see the tail split below) costs 1 / splits of a wave
+            const int64_t r = (int64_t)tiles % (int64_t)slots;
+            int64_t sp = r > 0 ? (int64_t)slots / r : 1;
+            if (sp > a.k / 256) sp = a.k / 256;
+            if (sp > 8) sp = 8;
+            if (tiles > slots && r > 0 && 2 * r <= (int64_t)slots && sp >= 2 && g_force_split == 0 && !g_no_tail_split &&
+                (size_t)(r * sp) * kSimtTileM[t] * kSimtTileN[t] * sizeof(float) <= ws_avail)
+                full = full - 1.0 + 1.0 / (double)sp;
+        }
         const double util = waves / full;                                           // tail effect
         const double useful = ((double)a.m * a.n) / (tiles * kSimtTileM[t] * kSimtTileN[t]);   // edge waste
         const double score = util * useful * eff[t];
@@ -121,6 +133,30 @@ static void plan_simt(const GemmArgs& a, int sms, size_t ws_avail, Plan* p) {
         p->ws_partials = 0;
     }
     p->ws_total = p->ws_partials;
+
+    // Tail split: with more tiles than CTA slots the last wave is only partly filled.  Its r tiles are cut into
+    // floor(slots / r) k ranges each, so that the last wave fills the machine and takes 1 / splits of a full one;
+    // a reduction over those tiles only (tile-local fp32 slots in the workspace) finishes them.
+    p->tail_splits = 1;
+    p->tail_first = 0x7FFFFFFF;
+    if (p->ks.splits == 1 && g_force_split == 0 && !g_no_tail_split && tiles > slots) {
+        const int64_t r = tiles % slots;
+        if (r > 0 && 2 * r <= slots) {
+            int64_t s = slots / r;
+            if (s > a.k / 256) s = a.k / 256;
+            if (s > 8) s = 8;
+            const size_t need = (size_t)(r * s) * kSimtTileM[best] * kSimtTileN[best] * sizeof(float);
+            if (s >= 2 && need <= ws_avail) {
+                p->tail_first = (int)(tiles - r);
+                p->tail_splits = (int)s;
+                p->tail_chunk = round_up(ceil_div(a.k, s), 16);
+                p->tail_splits = (int)ceil_div(a.k, p->tail_chunk);
+                p->ws_partials = (size_t)(r * p->tail_splits) * kSimtTileM[best] * kSimtTileN[best] * sizeof(float);
+                p->ws_total = p->ws_partials;
+                if (p->tail_splits < 2) { p->tail_splits = 1; p->tail_first = 0x7FFFFFFF; p->ws_partials = p->ws_total = 0; }
+            }
+        }
+    }
 }
 
 static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, bool b_ok, Plan* p) {
@@ -296,8 +332,17 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st) {
         }
     }
     float* partials = p.ks.splits > 1 ? reinterpret_cast<float*>(wsp) : nullptr;
-    if (p.kernel == GEMM_KERNEL_TENSOR) e = launch_tensor(a, p.tile, p.ks, partials, &cfg);
-    else e = launch_simt_fast(a, p.tile, p.ks, partials, &cfg);
+    if (p.kernel == GEMM_KERNEL_TENSOR) {
+        e = launch_tensor(a, p.tile, p.ks, partials, &cfg);
+    } else if (p.tail_splits > 1) {
+        TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
+        e = launch_simt_fast(a, p.tile, p.ks, nullptr, &cfg, tail);
+        if (e == cudaSuccess) e = launch_tail_reduce(a, p.tile, tail);
+        cfg.launches++;
+        cfg.tail_split = p.tail_splits;
+    } else {
+        e = launch_simt_fast(a, p.tile, p.ks, partials, &cfg);
+    }
     if (e == cudaSuccess && p.ks.splits > 1) {
         e = launch_splitk_reduce(a, p.ks.splits, partials);
         cfg.launches++;
@@ -528,6 +573,7 @@ int gemm_force_tile(int tile_m, int tile_n, int split_k) {
     g_force_tile_m = tile_m;
     g_force_tile_n = tile_n;
     g_force_split = split_k;
+    g_no_tail_split = (split_k == 1);
     return GEMM_OK;
 }
 

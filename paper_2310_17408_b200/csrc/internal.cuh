@@ -31,6 +31,27 @@ struct KSplit {
 // device status word layout: bits 31..24 = 0xE5 marker, 23..16 = role, 15..8 = barrier id, 7..0 = stage
 constexpr uint32_t STATUS_MARK = 0xE5000000u;
 
+// Tail split of the fp32 SIMT path: tiles first .. are cut into `splits` k ranges of `chunk` each
+// (first = INT_MAX: off).  Item i >= first writes its raw block to partials + (i - first) * tile_m * tile_n.
+struct TailSplit {
+    int first;
+    int splits;
+    int64_t chunk;
+    float* partials;
+};
+
+// Tile order of the fp32 SIMT path: groups of SIMT_GROUP tile rows, all tile columns inside a group, rows fastest,
+// so that the CTAs resident at one time share their A and B panels in L2.
+constexpr int SIMT_GROUP = 16;
+__host__ __device__ inline void decode_tile(int tile, int tiles_m, int tiles_n, int* tm, int* tn) {
+    const int per_group = SIMT_GROUP * tiles_n;
+    const int g = tile / per_group;
+    const int rest = tiles_m - g * SIMT_GROUP;
+    const int gsz = rest < SIMT_GROUP ? rest : SIMT_GROUP;
+    *tm = g * SIMT_GROUP + (tile % per_group) % gsz;
+    *tn = (tile % per_group) / gsz;
+}
+
 inline int elem_size(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }
 
 // C <- beta*C  (beta == 0: store +0 without reading)
@@ -42,7 +63,10 @@ cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg);
 // fast fp32 SIMT kernel.  tile: 0 = 128x128, 1 = 128x64, 2 = 64x128, 3 = 64x64.
 // ks.splits > 1: raw partial sums go to `partials` ([split][n][m], fp32), no epilogue.
 bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb);
-cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg);
+cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg,
+                             TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
+// finishes the tail tiles: C <- alpha * sum_z slot[(t - first) * splits + z] + beta*C for tiles t >= first
+cudaError_t launch_tail_reduce(const GemmArgs& a, int tile, TailSplit tail);
 
 // C <- alpha * sum_s partials[s] + beta*C, summed in increasing s (deterministic)
 cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* partials);

@@ -142,7 +142,7 @@ template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool
 __global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
 simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
                  const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
-                 int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials) {
+                 int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, TailSplit tail) {
     constexpr int NT = WARPS_M * WARPS_N * 32;
     static_assert(BM == WARPS_M * 64 && BN == WARPS_N * 32, "warp tile is 64 x 32");
     using LA = Loader<BM, NT, A_KCONT, VA>;
@@ -161,18 +161,25 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
     const int am = wm * 64 + lm * 4;                  // thread rows: am..am+3 and am+32..am+35
     const int bn = wn * 32 + ln * 4;                  // thread cols: bn..bn+3 and bn+16..bn+19
 
-    // grouped tile order: GROUP tile rows at a time, all tile columns inside a group
-    constexpr int GROUP = 16;
-    const int tile = blockIdx.x;
-    const int per_group = GROUP * tiles_n;
-    const int g = tile / per_group;
-    const int gsz = min(GROUP, tiles_m - g * GROUP);
-    const int tm = g * GROUP + (tile % per_group) % gsz;
-    const int tn = (tile % per_group) / gsz;
+    // Work items: blockIdx.x < tail.first is one whole tile.  The tiles of the last, partly filled wave
+    // (tail.first and up) are cut into tail.splits k ranges each, so that the wave still fills the machine;
+    // their raw partial sums go to tile-local slots of tail.partials and a small reduction pass finishes them.
+    int tile = blockIdx.x, ksplit = blockIdx.z;
+    int64_t kc = kchunk;
+    float* tail_out = nullptr;
+    if (tile >= tail.first) {
+        const int item = tile - tail.first;
+        tile = tail.first + item / tail.splits;
+        ksplit = item % tail.splits;
+        kc = tail.chunk;
+        tail_out = tail.partials + (int64_t)item * (BM * BN);
+    }
+    int tm, tn;
+    decode_tile(tile, tiles_m, tiles_n, &tm, &tn);
     const int64_t i0 = (int64_t)tm * BM, j0 = (int64_t)tn * BN;
 
-    const int64_t kbeg = (int64_t)blockIdx.z * kchunk;
-    const int64_t kend = min(k, kbeg + kchunk);
+    const int64_t kbeg = (int64_t)ksplit * kc;
+    const int64_t kend = min(k, kbeg + kc);
     const int64_t ktiles = (kend - kbeg + BK - 1) / BK;
 
     float acc[8][8];
@@ -224,6 +231,19 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
     }
 
     // ---- store: alpha*acc + beta*C, or raw partial sums for split-k
+    if (tail_out != nullptr) {      // tile-local slot [BN][BM]: whole register blocks, no bounds (edge entries are zero)
+#pragma unroll
+        for (int jh = 0; jh < 2; ++jh)
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                for (int ih = 0; ih < 2; ++ih) {
+                    const float* v = &acc[jh * 4 + jj][ih * 4];
+                    *reinterpret_cast<float4*>(tail_out + (am + ih * 32) + (bn + jh * 16 + jj) * BM) =
+                        make_float4(v[0], v[1], v[2], v[3]);
+                }
+        return;
+    }
     const bool raw = partials != nullptr;
     float* out = raw ? partials + (int64_t)blockIdx.z * m * n : C;
     const int64_t ldo = raw ? m : ldc;
@@ -276,13 +296,16 @@ bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb) {
 }
 
 template <int BM, int BN, int WM, int WN, int MINB, bool AK, bool BKC, int VA, int VB>
-static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg) {
+static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
     int64_t tiles_m = (a.m + BM - 1) / BM, tiles_n = (a.n + BN - 1) / BN;
     if (tiles_m * tiles_n > 0x7FFFFFFFLL || tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF / 16)
         return cudaErrorInvalidConfiguration;       // tile indices are 32-bit in the kernel (groups of 16 tile rows)
-    dim3 grid((unsigned)(tiles_m * tiles_n), 1, (unsigned)ks.splits);
+    int64_t items = tiles_m * tiles_n;
+    if (tail.first < items) items = tail.first + (items - tail.first) * tail.splits;      // tail tiles count once per k range
+    if (items > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)items, 1, (unsigned)ks.splits);
     cfg->tile_m = BM; cfg->tile_n = BN; cfg->tile_k = BK; cfg->stages = 2;
-    cfg->grid = (int32_t)(tiles_m * tiles_n * ks.splits);
+    cfg->grid = (int32_t)(items * ks.splits);
     cudaLaunchConfig_t lc = {};
     lc.gridDim = grid;
     lc.blockDim = dim3(WM * WN * 32);
@@ -295,40 +318,87 @@ static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gem
     cudaError_t le = cudaLaunchKernelEx(&lc, simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB>, a.m, a.n, a.k, a.alpha,
                                         (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.chunk,
-                                        ks.splits > 1 ? partials : (float*)nullptr);
+                                        ks.splits > 1 ? partials : (float*)nullptr, tail);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <bool AK, bool BKC, int VA, int VB>
-static cudaError_t launch_tile(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg) {
+static cudaError_t launch_tile(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
     switch (tile) {
-        case 0: return launch_one<128, 128, 2, 4, 2, AK, BKC, VA, VB>(a, ks, partials, cfg);
-        case 1: return launch_one<128, 64, 2, 2, 3, AK, BKC, VA, VB>(a, ks, partials, cfg);
-        case 2: return launch_one<64, 128, 1, 4, 3, AK, BKC, VA, VB>(a, ks, partials, cfg);
-        default: return launch_one<64, 64, 1, 2, 6, AK, BKC, VA, VB>(a, ks, partials, cfg);
+        case 0: return launch_one<128, 128, 2, 4, 2, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
+        case 1: return launch_one<128, 64, 2, 2, 3, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
+        case 2: return launch_one<64, 128, 1, 4, 3, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
+        default: return launch_one<64, 64, 1, 2, 6, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
     }
 }
 
 template <bool AK, bool BKC>
 static cudaError_t launch_vec(const GemmArgs& a, int va, int vb, int tile, KSplit ks, float* partials,
-                              gemm_config_t* cfg) {
-    if (va == 4 && vb == 4) return launch_tile<AK, BKC, 4, 4>(a, tile, ks, partials, cfg);
-    if (va == 4) return launch_tile<AK, BKC, 4, 1>(a, tile, ks, partials, cfg);
-    if (vb == 4) return launch_tile<AK, BKC, 1, 4>(a, tile, ks, partials, cfg);
-    return launch_tile<AK, BKC, 1, 1>(a, tile, ks, partials, cfg);
+                              gemm_config_t* cfg, TailSplit tail) {
+    if (va == 4 && vb == 4) return launch_tile<AK, BKC, 4, 4>(a, tile, ks, partials, cfg, tail);
+    if (va == 4) return launch_tile<AK, BKC, 4, 1>(a, tile, ks, partials, cfg, tail);
+    if (vb == 4) return launch_tile<AK, BKC, 1, 4>(a, tile, ks, partials, cfg, tail);
+    return launch_tile<AK, BKC, 1, 1>(a, tile, ks, partials, cfg, tail);
 }
 
-cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg) {
+cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
     int va, vb;
     simt_fast_eligible(a, &va, &vb);
     cfg->kernel = GEMM_KERNEL_SIMT_FAST;
     cfg->split_k = ks.splits;
     cfg->vector_a = va; cfg->vector_b = vb;
     // A is contiguous along k when transposed; B is contiguous along k when not transposed
-    if (!a.ta && !a.tb) return launch_vec<false, true>(a, va, vb, tile, ks, partials, cfg);
-    if (a.ta && !a.tb) return launch_vec<true, true>(a, va, vb, tile, ks, partials, cfg);
-    if (!a.ta && a.tb) return launch_vec<false, false>(a, va, vb, tile, ks, partials, cfg);
-    return launch_vec<true, false>(a, va, vb, tile, ks, partials, cfg);
+    if (!a.ta && !a.tb) return launch_vec<false, true>(a, va, vb, tile, ks, partials, cfg, tail);
+    if (a.ta && !a.tb) return launch_vec<true, true>(a, va, vb, tile, ks, partials, cfg, tail);
+    if (!a.ta && a.tb) return launch_vec<false, false>(a, va, vb, tile, ks, partials, cfg, tail);
+    return launch_vec<true, false>(a, va, vb, tile, ks, partials, cfg, tail);
+}
+
+// ---------------------------------------------------------------- tail reduction
+
+// One block row per tail tile (blockIdx.x) and a quarter of its entries per blockIdx.y: sums the tile's k ranges in
+// increasing order (deterministic) and applies alpha / beta once.
+__global__ void __launch_bounds__(256)
+tail_reduce_kernel(int64_t m, int64_t n, float alpha, float beta, float* __restrict__ C, int64_t ldc, int tiles_m,
+                   int tiles_n, int bm, int bn, TailSplit tail) {
+    const int tl = blockIdx.x;
+    int tm, tn;
+    decode_tile(tail.first + tl, tiles_m, tiles_n, &tm, &tn);
+    const int64_t i0 = (int64_t)tm * bm, j0 = (int64_t)tn * bn;
+    const int tile_elems = bm * bn;
+    const float* slot = tail.partials + (int64_t)tl * tail.splits * tile_elems;
+    const int vecs = tile_elems / 4, per_y = (vecs + gridDim.y - 1) / gridDim.y;
+    const int v_end = min(vecs, (int)(blockIdx.y + 1) * per_y);
+    for (int v = blockIdx.y * per_y + threadIdx.x; v < v_end; v += blockDim.x) {
+        const int e = v * 4, r = e % bm, c = e / bm;
+        float4 s4 = *reinterpret_cast<const float4*>(slot + e);
+        for (int z = 1; z < tail.splits; ++z) {
+            const float4 q = *reinterpret_cast<const float4*>(slot + (int64_t)z * tile_elems + e);
+            s4.x += q.x; s4.y += q.y; s4.z += q.z; s4.w += q.w;
+        }
+        const int64_t gi = i0 + r, gj = j0 + c;
+        if (gj >= n) continue;
+        const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+        float* cp = C + gi + gj * ldc;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (gi + q < m) {
+                float o = alpha * sv[q];
+                if (beta != 0.0f) o = fmaf(beta, cp[q], o);
+                cp[q] = o;
+            }
+    }
+}
+
+cudaError_t launch_tail_reduce(const GemmArgs& a, int tile, TailSplit tail) {
+    static const int bm_of[4] = {128, 128, 64, 64}, bn_of[4] = {128, 64, 128, 64};
+    const int bm = bm_of[tile], bn = bn_of[tile];
+    const int64_t tiles_m = (a.m + bm - 1) / bm, tiles_n = (a.n + bn - 1) / bn;
+    const int64_t tail_tiles = tiles_m * tiles_n - tail.first;
+    if (tail_tiles <= 0) return cudaSuccess;
+    tail_reduce_kernel<<<dim3((unsigned)tail_tiles, 4), 256, 0, a.stream>>>(a.m, a.n, a.alpha, a.beta, a.C, a.ldc,
+                                                                           (int)tiles_m, (int)tiles_n, bm, bn, tail);
+    return cudaGetLastError();
 }
 
 }  // namespace b200gemm

@@ -305,3 +305,28 @@ def test_fp16_subnormal_inputs_are_not_flushed():
     C, cfg = run_problem(p, A, B, C0)
     assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
     assert np.array_equal(C.window().astype(np.float64), a @ b)
+
+
+def test_fp32_tail_split_of_the_last_wave():
+    # more tiles than CTA slots with a small remainder: the tiles of the last wave are cut along k and finished by
+    # the tail reduction; ragged edges, all transpose combinations, integer-exact and random data
+    ensure_workspace(64 << 20)
+    for ta, tb in TRANS:
+        for (m, n, k) in [(2048, 2560, 2100), (2000, 2590, 1030), (4100, 1300, 777)]:
+            p = problem(DTYPE_F32, m, n, k, ta, tb, 1.5, 0.5, "uniform", (0, 4, 0), seed=m)
+            A, B, C0 = p.operands()
+            C, cfg = run_problem(p, A, B, C0)
+            assert cfg["tail_split"] >= 2 and cfg["split_k"] == 1 and cfg["launches"] == 2, cfg
+            check_against_oracle(p, A, B, C0, C)
+        p = problem(DTYPE_F32, 2000, 2590, 1030, ta, tb, -1.0, 1.0, "int", (4, 0, 4), seed=9)
+        A, B, C0 = p.operands()
+        C, cfg = run_problem(p, A, B, C0)
+        assert cfg["tail_split"] >= 2
+        check_against_oracle(p, A, B, C0, C, integer=True)
+    # without a workspace the same problem runs unsplit
+    drop_workspace()
+    p = problem(DTYPE_F32, 2048, 2560, 2100, "N", "N", 1.0, 0.0, "uniform", (0, 0, 0), seed=1)
+    A, B, C0 = p.operands()
+    C, cfg = run_problem(p, A, B, C0, workspace=False)
+    assert cfg["tail_split"] == 0
+    check_against_oracle(p, A, B, C0, C)
