@@ -62,6 +62,7 @@ static inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b
 struct Plan {
     int kernel;        // GEMM_KERNEL_*
     int tile;          // SIMT fast: tile id 0..3; tensor: tile_n
+    bool pair;         // tensor: 256 x 256 tiles on CTA pairs
     KSplit ks;
     bool repack_a, repack_b;
     int64_t lda_p, ldb_p;     // leading dimensions of the repacked operands
@@ -214,6 +215,18 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
             }
     }
     p->tile = bn;
+    // CTA pairs (256 x 256 tiles) fill a third less shared memory per flop, which is what limits the 128 x 256
+    // kernel: measured 9 % faster main loops (4096^3, 8192^3, the large VGG16 shapes), but ~2.5 us more fixed
+    // cost per launch (cluster set-up, cross-CTA barriers).  Taken when every pair has work and the main loops
+    // of the 128 x 256 kernel would run for 30 us or more.
+    {
+        const int64_t pair_tiles = ceil_div(a.m, 256) * ceil_div(a.n, 256);
+        const double rounds = (double)ceil_div(ceil_div(a.m, 128) * ceil_div(a.n, 256), sms);
+        const double main_us = rounds * (double)ceil_div(a.k, 64) * 0.27;
+        p->pair = bn == 256 && want == 1 && a.m > 128 && pair_tiles >= sms / 2 && main_us >= 30.0;
+    }
+    if (g_force_tile_m == 256) p->pair = bn == 256;
+    if (g_force_tile_m == 128) p->pair = false;
     p->ks = make_split(a.k, want, 64);
     p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
     if (ws_repack + p->ws_partials > ws_avail) {
@@ -333,7 +346,7 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st) {
     }
     float* partials = p.ks.splits > 1 ? reinterpret_cast<float*>(wsp) : nullptr;
     if (p.kernel == GEMM_KERNEL_TENSOR) {
-        e = launch_tensor(a, p.tile, p.ks, partials, &cfg);
+        e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg) : launch_tensor(a, p.tile, p.ks, partials, &cfg);
     } else if (p.tail_splits > 1) {
         TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
         e = launch_simt_fast(a, p.tile, p.ks, nullptr, &cfg, tail);

@@ -74,6 +74,8 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 // tcgen05 tensor-core kernel (fp16 / bf16).  tile_n in {64, 128, 256}; tile_m is 128.
 bool tensor_eligible(const GemmArgs& a);
 cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg);
+// the same on CTA pairs (tcgen05 cta_group::2): 256 x 256 tiles, two SMs per tile
+cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg);
 
 // copy op-independent stored matrix (rows x cols, ld) of 16-bit elements into an aligned layout (ld_out)
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,

@@ -1,0 +1,192 @@
+// Device-side building blocks shared by the tcgen05 kernels: bounded mbarrier waits, TMA copies, shared-memory
+// matrix descriptors, MMA issue / commit, TMEM loads; and the host-side tensor-map builders.
+#pragma once
+#include <cuda.h>
+
+#include "internal.cuh"
+
+namespace b200gemm {
+
+constexpr int TBM = 128;            // MMA M (TMEM lanes)
+constexpr int TBK = 64;             // k block: 64 x 2 bytes = one 128-byte swizzle row
+constexpr int UMMA_K = 16;          // k extent of one tcgen05.mma for 16-bit inputs
+constexpr int EPI_WARPS = 8;        // two epilogue warps per TMEM lane quarter, each taking every other 32-column chunk
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
+constexpr uint32_t SPIN_FAST = 4096;
+constexpr uint32_t SPIN_LIMIT = 1u << 24;   // then ~128 ns sleeps: gives up after a few seconds
+
+enum Role : uint32_t { ROLE_TMA = 1, ROLE_MMA = 2, ROLE_EPI = 3, ROLE_SELFTEST = 0x7F };
+enum Bar : uint32_t { BAR_FULL = 1, BAR_EMPTY = 2, BAR_TMEM_FULL = 3, BAR_TMEM_EMPTY = 4 };
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the wait expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status, uint32_t code, uint32_t limit = SPIN_LIMIT) {
+    for (uint32_t it = 0; it < limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it >= SPIN_FAST) {
+            if (*abort_flag) return false;
+            __nanosleep(128);
+        }
+    }
+    atomicCAS(status, 0u, code);
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(const CUtensorMap* tm, uint32_t dst, uint32_t bar, int32_t c0, int32_t c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+// shared memory -> global tile store (bulk async group); out-of-range parts of the box are clipped by the hardware
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int32_t c0, int32_t c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int32_t c0, int32_t c1, int32_t c2) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// shared-memory matrix descriptor (128-byte swizzle): start address, leading / stride byte offsets in 16-byte units
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;      // descriptor version of the tcgen05 family
+    d |= (uint64_t)2 << 61;      // swizzle mode: 128 bytes
+    return d;
+}
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the mbarrier once all previously issued MMAs of this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Epilogue of one accumulator tile for one warp (lane = row of C, TMEM lanes 32q .. 32q+31 starting at row0).
+// The warp takes the 32-column chunks half, half + 2, ... of the BN-wide tile: each chunk is read from TMEM, scaled
+// (alpha, beta of Fig. 3; raw = split-k partial sums, stored unscaled) and then either written straight to global
+// memory (32 consecutive floats of one column per instruction) or, when the target can be addressed by TMA,
+// transposed through a 32 x 32 staging tile in shared memory and written by an asynchronous bulk tensor store,
+// which also clips the tile at the matrix edge.  release_acc() is called exactly once, as soon as the warp has
+// read its last chunk, so that the accumulator can be overwritten while the stores are still in flight.
+template <int BN, int STORE_BUFS, typename Release>
+__device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int64_t row0, int64_t n0, int half, int lane,
+                                              int64_t m, int64_t n, float alpha, float beta, float* out, int64_t ldo,
+                                              bool raw, bool via_tma, const CUtensorMap* tmC, int sp, float* stage,
+                                              uint32_t& sbuf, Release&& release_acc) {
+    const int64_t row = row0 + lane;
+    bool released = false;
+    if (row0 < m) {
+#pragma unroll 1
+        for (int c = half; c < BN / 32; c += 2) {
+            const int64_t col0 = n0 + c * 32;
+            if (col0 >= n) break;
+            const bool last_chunk = (c + 2 >= BN / 32) || (col0 + 64 >= n);
+            uint32_t v[32];
+            tmem_ld32(tmem_acc + c * 32, v);
+            float* cp = out + row + col0 * ldo;
+            float c0[32];
+            const bool need_c0 = !raw && beta != 0.0f;
+            if (need_c0) {      // issue all reads of C before waiting on anything
+#pragma unroll
+                for (int j = 0; j < 32; ++j) c0[j] = (row < m && col0 + j < n) ? cp[j * ldo] : 0.0f;
+            }
+            tmem_ld_wait();
+            if (last_chunk) { release_acc(); released = true; }
+            float* r = reinterpret_cast<float*>(v);       // scaled in place
+            if (!raw) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    r[j] *= alpha;
+                    if (need_c0) r[j] = fmaf(beta, c0[j], r[j]);
+                }
+            }
+            if (via_tma) {
+                if (lane == 0) bulk_wait_read<STORE_BUFS - 1>();   // the store that last used this staging tile has read it
+                __syncwarp();
+                float* st = stage + sbuf * (32 * 32);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) st[j * 32 + lane] = r[j];
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (raw) tma_store_3d(tmC, smem_u32(st), (int32_t)row0, (int32_t)col0, sp);
+                    else tma_store_2d(tmC, smem_u32(st), (int32_t)row0, (int32_t)col0);
+                    bulk_commit();
+                }
+                sbuf = (sbuf + 1 == (uint32_t)STORE_BUFS) ? 0 : sbuf + 1;
+            } else if (row < m) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (col0 + j < n) cp[j * ldo] = r[j];
+            }
+        }
+    }
+    if (!released) release_acc();
+}
+
+// ---------------------------------------------------------------- host side (defined in tc_gemm.cu)
+
+// 2-D map over a stored column-major matrix of 16-bit elements: dim0 = contiguous dimension (rows), dim1 = columns
+// (stride ld); 128-byte swizzle
+bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_t cols, int64_t ld,
+              uint32_t box_rows, uint32_t box_cols);
+// map over the split-k partial sums [split][n][m] (fp32, dense): 32 x 32 x 1 boxes
+bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits);
+// map over the fp32 result for the epilogue's tile stores: 32 x 32 boxes, no swizzle
+bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc);
+// instruction descriptor of tcgen05.mma kind::f16 with fp32 accumulation: mma_m x mma_n, operand majorness
+uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n);
+
+}  // namespace b200gemm

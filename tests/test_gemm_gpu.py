@@ -78,6 +78,35 @@ def test_every_tile_and_split_k(dtype):
             check_against_oracle(p, A, B, C0, C, integer=True)
 
 
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+def test_cta_pair_tiles(dtype):
+    """256 x 256 tiles on CTA pairs (two SMs per tile): every transpose combination, split-k, tiles whose second
+    half lies partly or wholly outside the matrix, and more tiles than pairs (each pair walks several tiles and
+    reuses both accumulators and every pipeline stage several times)."""
+    ensure_workspace(256 << 20)
+    shapes = [(300, 520, 777), (129, 300, 200), (100, 520, 130), (1000, 1100, 264)]
+    for split in (1, 2, 3):
+        g.gemm_force_tile(256, 256, split)
+        for (m, n, k), (ta, tb) in itertools.product(shapes, TRANS):
+            p = problem(dtype, m, n, k, ta, tb, 1.5, 0.5, "normal", (8, 0, 4), seed=m + split)
+            A, B, C0 = p.operands()
+            C, cfg = run_problem(p, A, B, C0)
+            assert (cfg["kernel"], cfg["tile_m"], cfg["tile_n"]) == (g.GEMM_KERNEL_TENSOR, 256, 256), cfg
+            assert cfg["split_k"] == split or (split > 1 and cfg["split_k"] > 1), cfg
+            check_against_oracle(p, A, B, C0, C)
+            p = problem(dtype, m, n, k, ta, tb, 1.5, 0.5, "int", (0, 8, 0), seed=5)
+            A, B, C0 = p.operands()
+            C, cfg = run_problem(p, A, B, C0)
+            check_against_oracle(p, A, B, C0, C, integer=True)
+    g.gemm_force_tile(256, 256, 1)
+    for ta, tb in (("N", "N"), ("T", "N")):
+        p = problem(dtype, 2400, 4000, 136, ta, tb, 1.0, 0.0, "int", (0, 0, 0), seed=11)     # 160 tiles
+        A, B, C0 = p.operands()
+        C, cfg = run_problem(p, A, B, C0)
+        assert (cfg["tile_m"], cfg["tile_n"]) == (256, 256) and cfg["grid"] % 2 == 0, cfg
+        check_against_oracle(p, A, B, C0, C, integer=True)
+
+
 @pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_F16, DTYPE_BF16])
 def test_results_are_deterministic(dtype):
     ensure_workspace(64 << 20)
