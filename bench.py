@@ -473,9 +473,12 @@ def run_cuda(args, problems, workload_name):
     if rank == 0:
         p, bound, peak, unit, achieved, cfg = dominant
         kernel_names = {1: "simt_generic_kernel", 2: "simt_fast_kernel", 3: "tc_gemm_kernel", 6: "scale_kernel"}
+        kname = kernel_names.get(cfg["kernel"], "?")
+        if cfg["kernel"] == 3 and cfg["tile_m"] == 256:
+            kname = "tc_gemm_pair_kernel"          # 256 x 256 tiles on CTA pairs
         roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": recorded_traffic(kernel_names.get(cfg["kernel"], "?"), p),
-                "kernel": kernel_names.get(cfg["kernel"], "?"), "problem": p.name,
+                "traffic": recorded_traffic(kname, p),
+                "kernel": kname, "problem": p.name,
                 "peak_source": (f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz (max SM clock)"
                                 if bound == "alu" else f"{peaks['source']} ({'MEASURED_PEAKS.json' if peaks['source'] == 'measured' else 'recipe fallback'})")}
         if bound == "alu" and clocks.get("sm_mhz"):

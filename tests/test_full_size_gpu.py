@@ -60,12 +60,14 @@ def test_config5_half_squares_4096_8192(dtype):
     for i, p in enumerate(config_problems(5, dtype=dtype)[:2]):
         cfg, _ = run_and_check(p, seed=i)
         assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
+        assert (cfg["tile_m"], cfg["tile_n"]) == (256, 256)      # large squares run on CTA pairs
 
 
 def test_config5_f16_square_16384():
     p = config_problems(5, dtype=DTYPE_F16)[2]
     cfg, _ = run_and_check(p)
     assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
+    assert (cfg["tile_m"], cfg["tile_n"]) == (256, 256)
 
 
 @pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
