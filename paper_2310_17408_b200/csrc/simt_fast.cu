@@ -110,11 +110,34 @@ struct Loader {
     }
 };
 
+// Packed fp32 arithmetic: one fma.rn.f32x2 performs two independent IEEE fp32 fused multiply-adds (round to nearest
+// even, no flush to zero), lo = a.lo*b.lo + c.lo and hi = a.hi*b.hi + c.hi, in one issue slot.  It halves the
+// instructions of the products (issue slots used: 83 % -> 49 %); the FMA pipes themselves then set the pace.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma2(uint64_t& c, uint64_t a, uint64_t b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(c) : "l"(a), "l"(b));
+}
+
+// The thread's 8 x 8 register block as 2 x 2 sub-blocks of packed pairs.  For rows (i, i+1) and columns (j, j+1):
+//   P[j/2][i/2] = ( acc(i, j),   acc(i+1, j+1) )   updated with (a_i, a_i+1) * (b_j,   b_j+1)
+//   Q[j/2][i/2] = ( acc(i, j+1), acc(i+1, j)   )   updated with (a_i, a_i+1) * (b_j+1, b_j)
+// so that the pairs of A come straight out of the 128-bit fragment load and B needs only its four swapped pairs.
+struct Acc2 {
+    uint64_t P[4][4], Q[4][4];
+};
+
 // one BK slice of outer products on the thread's 8 x 8 register block
 template <int BM, int BN>
-__device__ __forceinline__ void compute_stage(float (&acc)[8][8], const float* __restrict__ As,
+__device__ __forceinline__ void compute_stage(Acc2& acc, const float* __restrict__ As,
                                               const float* __restrict__ Bs, int am, int bn) {
-    float a[2][8], b[2][8];
+    uint64_t a[2][4], b[2][4], bs[2][4];
     auto frag = [&](int kk, int buf) {
         const float* ap = As + kk * (BM + PAD) + am;
         const float* bp = Bs + kk * (BN + PAD) + bn;
@@ -122,20 +145,44 @@ __device__ __forceinline__ void compute_stage(float (&acc)[8][8], const float* _
         float4 a1 = *reinterpret_cast<const float4*>(ap + 32);
         float4 b0 = *reinterpret_cast<const float4*>(bp);
         float4 b1 = *reinterpret_cast<const float4*>(bp + 16);
-        a[buf][0] = a0.x; a[buf][1] = a0.y; a[buf][2] = a0.z; a[buf][3] = a0.w;
-        a[buf][4] = a1.x; a[buf][5] = a1.y; a[buf][6] = a1.z; a[buf][7] = a1.w;
-        b[buf][0] = b0.x; b[buf][1] = b0.y; b[buf][2] = b0.z; b[buf][3] = b0.w;
-        b[buf][4] = b1.x; b[buf][5] = b1.y; b[buf][6] = b1.z; b[buf][7] = b1.w;
+        a[buf][0] = pack2(a0.x, a0.y); a[buf][1] = pack2(a0.z, a0.w);
+        a[buf][2] = pack2(a1.x, a1.y); a[buf][3] = pack2(a1.z, a1.w);
+        b[buf][0] = pack2(b0.x, b0.y); b[buf][1] = pack2(b0.z, b0.w);
+        b[buf][2] = pack2(b1.x, b1.y); b[buf][3] = pack2(b1.z, b1.w);
+        bs[buf][0] = pack2(b0.y, b0.x); bs[buf][1] = pack2(b0.w, b0.z);
+        bs[buf][2] = pack2(b1.y, b1.x); bs[buf][3] = pack2(b1.w, b1.z);
     };
     frag(0, 0);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
         if (kk + 1 < BK) frag(kk + 1, (kk + 1) & 1);
+        // boustrophedon order over the 4 x 4 pairs: consecutive instructions share the A pair, and across a turn
+        // also the B pair (measured 1 % faster than row-by-row order)
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
+        for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(a[kk & 1][i], b[kk & 1][j], acc[j][i]);
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = (i & 1) ? 3 - jj : jj;
+                if (i & 1) {
+                    fma2(acc.Q[j][i], a[kk & 1][i], bs[kk & 1][j]);
+                    fma2(acc.P[j][i], a[kk & 1][i], b[kk & 1][j]);
+                } else {
+                    fma2(acc.P[j][i], a[kk & 1][i], b[kk & 1][j]);
+                    fma2(acc.Q[j][i], a[kk & 1][i], bs[kk & 1][j]);
+                }
+            }
     }
+}
+
+// packed accumulators -> acc[column][row] of the 8 x 8 block
+__device__ __forceinline__ void unpack_block(const Acc2& p, float (&acc)[8][8]) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            unpack2(p.P[j][i], acc[2 * j][2 * i], acc[2 * j + 1][2 * i + 1]);
+            unpack2(p.Q[j][i], acc[2 * j + 1][2 * i], acc[2 * j][2 * i + 1]);
+        }
 }
 
 template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB>
@@ -182,11 +229,11 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
     const int64_t kend = min(k, kbeg + kc);
     const int64_t ktiles = (kend - kbeg + BK - 1) / BK;
 
-    float acc[8][8];
+    Acc2 acc2;
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
+    for (int j = 0; j < 4; ++j)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[j][i] = 0.0f;
+        for (int i = 0; i < 4; ++i) acc2.P[j][i] = acc2.Q[j][i] = 0ull;      // (+0.0f, +0.0f)
 
     float ra[LA::ELEMS], rb[LB::ELEMS];
     const bool interior = (i0 + BM <= m) && (j0 + BN <= n);
@@ -221,7 +268,7 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
         for (int64_t kt = 0; kt < ktiles; ++kt) {
             const int cur = (int)(kt & 1);
             if (kt + 1 < ktiles) gload(kt + 1);                 // in flight during the math below
-            compute_stage<BM, BN>(acc, As[cur], Bs[cur], am, bn);
+            compute_stage<BM, BN>(acc2, As[cur], Bs[cur], am, bn);
             if (kt + 1 < ktiles) {
                 LA::store(ra, As[cur ^ 1], t);
                 LB::store(rb, Bs[cur ^ 1], t);
@@ -231,6 +278,8 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
     }
 
     // ---- store: alpha*acc + beta*C, or raw partial sums for split-k
+    float acc[8][8];
+    unpack_block(acc2, acc);
     if (tail_out != nullptr) {      // tile-local slot [BN][BM]: whole register blocks, no bounds (edge entries are zero)
 #pragma unroll
         for (int jh = 0; jh < 2; ++jh)
