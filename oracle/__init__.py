@@ -18,7 +18,7 @@ import numpy as np
 
 _HERE = Path(__file__).resolve().parent
 _SO = _HERE / "liboracle.so"
-_SRC = [_HERE / "gemm_oracle.c", _HERE / "gemm_l1_body.inc"]
+_SRC = [_HERE / "gemm_oracle.c", _HERE / "gemm_l1_body.inc", _HERE / "conv_oracle.c"]
 
 OR_F32, OR_F16, OR_BF16 = 0, 1, 2
 ACC_F32, ACC_F32FMA, ACC_F64 = 0, 1, 2
@@ -33,9 +33,17 @@ def build(force: bool = False) -> Path:
     if not force and _SO.exists() and all(_SO.stat().st_mtime >= s.stat().st_mtime for s in _SRC):
         return _SO
     cmd = ["gcc", "-O3", "-march=x86-64-v3", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
-           "-shared", "-fPIC", "-o", str(_SO), str(_SRC[0]), "-lm"]
+           "-shared", "-fPIC", "-o", str(_SO), str(_SRC[0]), str(_SRC[2]), "-lm"]
     subprocess.run(cmd, check=True, cwd=str(_HERE))
     return _SO
+
+
+class ConvGeom(ctypes.Structure):
+    """Geometry of a convolution layer (conv_oracle.c): NHWC activations, kh x kw filters, strides, zero padding."""
+    _fields_ = [("batch", ctypes.c_int64), ("h", ctypes.c_int64), ("w", ctypes.c_int64), ("c_in", ctypes.c_int64),
+                ("c_out", ctypes.c_int64), ("kh", ctypes.c_int32), ("kw", ctypes.c_int32),
+                ("stride_h", ctypes.c_int32), ("stride_w", ctypes.c_int32), ("pad_h", ctypes.c_int32),
+                ("pad_w", ctypes.c_int32)]
 
 
 _lib = None
@@ -70,6 +78,17 @@ def lib() -> ctypes.CDLL:
         L.oracle_ukernel_f32.restype = ci
         L.oracle_ukernel_f32.argtypes = [ci, ci, i64, ctypes.c_float, vp, vp, ctypes.c_float, vp, ci]
         L.oracle_num_threads.restype = ci
+        gp = ctypes.POINTER(ConvGeom)
+        L.oracle_conv_out_h.restype = i64
+        L.oracle_conv_out_h.argtypes = [gp]
+        L.oracle_conv_out_w.restype = i64
+        L.oracle_conv_out_w.argtypes = [gp]
+        L.oracle_conv2d_direct.restype = ci
+        L.oracle_conv2d_direct.argtypes = [ci, gp, dbl, vp, vp, i64, dbl, vp, i64, vp, i64]
+        L.oracle_conv2d_samples_f64.restype = ci
+        L.oracle_conv2d_samples_f64.argtypes = [ci, gp, dbl, vp, vp, i64, dbl, vp, i64, i64, vp, vp, vp]
+        L.oracle_im2row.restype = ci
+        L.oracle_im2row.argtypes = [ci, gp, vp, vp, i64]
         _lib = L
     return _lib
 
@@ -208,3 +227,54 @@ def fp32_tolerance(k, alpha, beta, max_a, max_b, max_c0):
     """Absolute bound for fp32 GEMM results: 4 * 2^-24 * (k |alpha| max|A| max|B| + |beta| max|C0|).
     At alpha = 1, beta = 0 this is the bound 4 k 2^-24 max|A| max|B|."""
     return 4.0 * 2.0 ** -24 * (k * abs(alpha) * max_a * max_b + abs(beta) * max_c0)
+
+
+# ---------------------------------------------------------------- convolution layers lowered with im2row (conv_oracle.c)
+
+def conv_geom(batch, h, w, c_in, c_out, kh, kw, stride_h=1, stride_w=1, pad_h=0, pad_w=0) -> ConvGeom:
+    return ConvGeom(batch, h, w, c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w)
+
+
+def conv_out_hw(g: ConvGeom):
+    return int(lib().oracle_conv_out_h(ctypes.byref(g))), int(lib().oracle_conv_out_w(ctypes.byref(g)))
+
+
+def conv2d_direct(dtype, g: ConvGeom, alpha, X, Wt, ldw, beta=0.0, Y0=None, ldy0=0):
+    """Definition of the layer in fp64.  Returns a C_out x pixels float64 array (pixels in (b, ho, wo) order)."""
+    _check_buf(X, dtype), _check_buf(Wt, dtype)
+    ho, wo = conv_out_hw(g)
+    npix = g.batch * ho * wo
+    ldo = max(1, g.c_out)
+    out = np.zeros(ldo * npix, dtype=np.float64)
+    rc = lib().oracle_conv2d_direct(dtype, ctypes.byref(g), float(alpha), _ptr(X), _ptr(Wt), ldw, float(beta),
+                                    _ptr(Y0), ldy0, _ptr(out), ldo)
+    if rc != 0:
+        raise RuntimeError(f"oracle_conv2d_direct failed: {rc}")
+    return out.reshape(npix, ldo).T[:g.c_out, :]
+
+
+def conv2d_samples_f64(dtype, g: ConvGeom, alpha, X, Wt, ldw, beta, Y0, ldy0, rows, cols):
+    """fp64 values of the output entries (channel rows[t], pixel cols[t])."""
+    _check_buf(X, dtype), _check_buf(Wt, dtype)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    out = np.zeros(rows.size, dtype=np.float64)
+    rc = lib().oracle_conv2d_samples_f64(dtype, ctypes.byref(g), float(alpha), _ptr(X), _ptr(Wt), ldw, float(beta),
+                                         _ptr(Y0), ldy0, rows.size, _ptr(rows), _ptr(cols), _ptr(out))
+    if rc != 0:
+        raise RuntimeError(f"oracle_conv2d_samples_f64 failed: {rc}")
+    return out
+
+
+def im2row(dtype, g: ConvGeom, X, ld=None):
+    """The lowered activation matrix: buffer of the k x pixels column-major matrix (leading dimension ld >= k) in
+    the element type of X; column j is the patch of output pixel j in (r, s, c) order."""
+    _check_buf(X, dtype)
+    ho, wo = conv_out_hw(g)
+    k = g.kh * g.kw * g.c_in
+    ld = k if ld is None else ld
+    out = np.zeros(ld * g.batch * ho * wo, dtype=X.dtype)
+    rc = lib().oracle_im2row(dtype, ctypes.byref(g), _ptr(X), _ptr(out), ld)
+    if rc != 0:
+        raise RuntimeError(f"oracle_im2row failed: {rc}")
+    return out

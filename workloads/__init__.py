@@ -25,4 +25,6 @@ from .shapes import (  # noqa: F401
     Problem,
     config_problems,
     im2row_problems,
+    ConvProblem,
+    conv_layer_problems,
 )

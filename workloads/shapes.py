@@ -210,3 +210,82 @@ def im2row_problems(network: str = "vgg16", *, batch: int = 32, weights_as_A: bo
             kinds = dict(kindA="absnormal", kindB="normal", scaleB=w_std)
         probs.append(Problem(f"{tag}_{i + 1:02d}", dtype, m, n, k, 1.0, 0.0, seed=base + i, **kinds))
     return probs
+
+
+# ---------------------------------------------------------------- convolution layers (the step before the lowering)
+
+@dataclass(frozen=True)
+class ConvProblem:
+    """One convolution layer whose im2row lowering is a GEMM of the workloads: geometry, scalars and the recipe of
+    its synthetic tensors.  Activations are NHWC, filters a column-major C_out x (kh*kw*C_in) matrix with the k index
+    in (r, s, c) order, the result NHWC (as a column-major matrix: C_out x pixels)."""
+    name: str
+    dtype: int
+    batch: int
+    h: int
+    w: int
+    c_in: int
+    c_out: int
+    kh: int
+    kw: int
+    stride: int = 1
+    pad: int = 0
+    alpha: float = 1.0
+    beta: float = 0.0
+    kindX: str = "absnormal"
+    kindW: str = "normal"
+    kindY: str = "uniform"
+    seed: int = 0
+    ld_pad: tuple = field(default=(0, 0))     # extra leading-dimension rows for the filter matrix and for Y
+
+    @property
+    def out_hw(self):
+        return ((self.h + 2 * self.pad - self.kh) // self.stride + 1, (self.w + 2 * self.pad - self.kw) // self.stride + 1)
+
+    @property
+    def gemm_mnk(self):
+        """(m, n, k) of the lowered GEMM with the filters as operand A: m = C_out, n = batch*Ho*Wo, k = kh*kw*C_in."""
+        ho, wo = self.out_hw
+        return self.c_out, self.batch * ho * wo, self.kh * self.kw * self.c_in
+
+    @property
+    def flops(self) -> float:
+        m, n, k = self.gemm_mnk
+        return 2.0 * m * n * k
+
+    def algorithmic_bytes(self) -> float:
+        """Activations and filters read once, result written once (read once more if beta != 0): what a fused
+        lowering has to move.  The lowered matrix itself (k x pixels) is never counted."""
+        es = 4 if self.dtype == DTYPE_F32 else 2
+        m, n, k = self.gemm_mnk
+        return es * (self.batch * self.h * self.w * self.c_in + m * k) + 4.0 * m * n * (2 if self.beta != 0.0 else 1)
+
+    def operands(self) -> tuple[Matrix, Matrix, Matrix]:
+        """(X, W, Y0): X as the C_in x (batch*H*W) column-major matrix that an NHWC tensor is, W as C_out x k,
+        Y0 (fp32) as C_out x pixels."""
+        m, n, k = self.gemm_mnk
+        scale_w = 1.0 if self.kindW == "int" else (2.0 / k) ** 0.5
+        X = make_matrix(self.c_in, self.batch * self.h * self.w, kind=self.kindX, seed=self.seed, matrix_id=1, dtype=self.dtype)
+        W = make_matrix(m, k, kind=self.kindW, seed=self.seed, matrix_id=0, dtype=self.dtype, ld=m + self.ld_pad[0], scale=scale_w)
+        Y0 = make_matrix(m, n, kind=self.kindY, seed=self.seed, matrix_id=2, dtype=DTYPE_F32, ld=m + self.ld_pad[1])
+        return X, W, Y0
+
+
+def conv_layer_problems(network: str = "resnet50", *, batch: int = 32, dtype: int = DTYPE_F32, integer: bool = False) -> list[ConvProblem]:
+    """The convolution layers behind the rows of Tables "resnet50" / "vgg16", with the usual geometry of those
+    networks: 7 x 7 stride 2 pad 3 on a 224 x 224 image for the ResNet stem, 3 x 3 stride 1 pad 1 and 1 x 1 layers on
+    an input of the output's size.  Their lowered GEMM dimensions equal im2row_shapes(..., weights_as_A=True).
+    Seeds 8000 + index (resnet50) / 9000 + index (vgg16)."""
+    layers = {"vgg16": VGG16_BATCH1, "resnet50": RESNET50_V15_BATCH1}[network]
+    base = 8000 if network == "resnet50" else 9000
+    tag = ("h" if dtype == DTYPE_F16 else "b" if dtype == DTYPE_BF16 else "") + network[:3] + "_conv"
+    kinds = dict(kindX="int", kindW="int", kindY="int") if integer else {}
+    out = []
+    for i, L in enumerate(layers):
+        if L.ksize == 7:
+            geo = dict(h=2 * L.out_hw, w=2 * L.out_hw, stride=2, pad=3)
+        else:
+            geo = dict(h=L.out_hw, w=L.out_hw, stride=1, pad=L.ksize // 2)
+        out.append(ConvProblem(f"{tag}_{i + 1:02d}", dtype, batch, c_in=L.cin, c_out=L.cout, kh=L.ksize, kw=L.ksize,
+                               seed=base + i, **geo, **kinds))
+    return out
