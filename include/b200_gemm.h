@@ -60,6 +60,7 @@ typedef struct {
     int32_t launches;      /* kernels enqueued by the call (main + reduction / scaling)      */
     int32_t repacked;      /* bit 0: A was copied to an aligned layout first, bit 1: B       */
     int32_t tail_split;    /* fp32: k ranges each tile of the last, partly filled wave was cut into (0 = not used) */
+    int32_t lowering;      /* conv2d_im2row: one of CONV_LOWERING_* (0 for plain gemm calls)                        */
 } gemm_config_t;
 
 /*
@@ -142,6 +143,53 @@ int gemm_set_workspace(void* dev, size_t bytes, void* stream);
 int gemm_f32_splitk_static(char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha,
                            const float* A, int64_t lda, const float* B, int64_t ldb, float beta, float* C, int64_t ldc,
                            int split_k, void* stream);
+
+/*
+ * Convolution layers lowered to GEMM with the im2row transform (Section IV-C, "Rectangular Matrices": the GEMM
+ * dimensions of Tables "resnet50" and "vgg16" are m = batch*Ho*Wo output pixels, n = C_out, k = C_in*kh*kw).
+ *
+ *   conv2d_im2row   Y <- alpha * conv(X, W) + beta * Y, computed as the GEMM the lowering defines,
+ *                       Y[C_out x pixels] = W[C_out x k] * L[k x pixels],
+ *                   where column j = (b*Ho + ho)*Wo + wo of L is the receptive field of output pixel j:
+ *                   L(p, j) = X(b, ho*stride_h - pad_h + r, wo*stride_w - pad_w + s, c) with p = (r*kw + s)*C_in + c,
+ *                   and 0 where that position lies outside the image (zero padding).
+ *                   Ho = (H + 2*pad_h - kh)/stride_h + 1, Wo likewise.
+ *     X       device pointer, NHWC activations of `dtype`: element (b, h, w, c) at ((b*H + h)*W + w)*C_in + c
+ *     W, ldw  device pointer, the filters as a column-major C_out x k matrix of `dtype` (ldw >= C_out), i.e.
+ *             element (co; r, s, c) at co + ((r*kw + s)*C_in + c)*ldw
+ *     Y, ldy  device pointer to fp32, NHWC result: element (co; pixel j) at co + j*ldy, ldy >= C_out; read only if
+ *             beta != 0; rows C_out..ldy-1 are never touched
+ *   Where it can, the lowering is fused into the operand staging of the GEMM kernels and L never exists in memory:
+ *   fp32 reads X through the index map inside the SIMT kernel's loads; fp16/bf16 layers with C_in a multiple of
+ *   64, a 16-byte aligned X, square filters and the same stride and padding in both directions let TMA's im2col
+ *   mode deliver the swizzled tiles.  1 x 1 layers with stride 1 and no padding need no lowering (L is X).  All other
+ *   cases first write L into the registered workspace with im2row() and then run gemm() on it; they return
+ *   GEMM_ERR_WORKSPACE if the workspace is smaller than conv2d_workspace_bytes().
+ *   Returns GEMM_OK, -(position of the first invalid argument) (2 = a field of *shape), or a GEMM_ERR_* code.
+ *   Asynchronous on `stream`, like gemm().
+ *
+ *   im2row          the transform by itself: writes L (element type of X, leading dimension ld >= k, column-major,
+ *                   16-byte chunks when alignment allows) to `out`.  An HBM-bound copy: C_in*kh*kw*pixels elements.
+ */
+typedef struct {
+    int64_t batch, h, w, c_in, c_out;
+    int32_t kh, kw, stride_h, stride_w, pad_h, pad_w;
+} conv_shape_t;
+
+enum {
+    CONV_LOWERING_NONE     = 0,
+    CONV_LOWERING_FUSED    = 1,  /* index map / TMA im2col inside the GEMM kernel; L never materialised */
+    CONV_LOWERING_EXPLICIT = 2,  /* im2row() into the workspace, then gemm()                             */
+    CONV_LOWERING_IDENTITY = 3   /* 1 x 1, stride 1, no padding: L is X                                  */
+};
+
+int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void* X, const void* W, int64_t ldw,
+                  float beta, void* Y, int64_t ldy, void* stream);
+int im2row(int dtype, const conv_shape_t* shape, const void* X, void* out, int64_t ld, void* stream);
+/* workspace conv2d_im2row would like for this layer: the lowered matrix if it has to be written, plus what the GEMM asks for */
+size_t conv2d_workspace_bytes(int dtype, const conv_shape_t* shape);
+/* tests / benchmarks: 0 = choose, CONV_LOWERING_FUSED or CONV_LOWERING_EXPLICIT = take that route when it is possible */
+int conv2d_force_lowering(int how);
 
 /* configuration chosen by the most recent gemm() of the calling thread (for tests and reports) */
 int gemm_last_config(gemm_config_t* out);

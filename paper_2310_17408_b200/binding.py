@@ -20,17 +20,27 @@ GEMM_KERNEL_SCALE_ONLY = 6
 EXPORTS = ("gemm", "gemm_host", "gemm_workspace_bytes", "gemm_set_workspace", "gemm_last_config",
            "gemm_force_kernel", "gemm_force_tile", "gemm_poll_status", "gemm_status_detail",
            "gemm_status_string", "gemm_last_cuda_error", "gemm_f32_splitk_static",
-           "gemm_selftest_wait_expiry")
+           "gemm_selftest_wait_expiry", "conv2d_im2row", "im2row", "conv2d_workspace_bytes",
+           "conv2d_force_lowering")
+CONV_LOWERING_NONE, CONV_LOWERING_FUSED, CONV_LOWERING_EXPLICIT, CONV_LOWERING_IDENTITY = 0, 1, 2, 3
 GEMM_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class GemmConfig(ctypes.Structure):
     _fields_ = [(name, ctypes.c_int32) for name in
                 ("kernel", "tile_m", "tile_n", "tile_k", "split_k", "stages", "grid", "vector_a", "vector_b",
-                 "launches", "repacked", "tail_split")]
+                 "launches", "repacked", "tail_split", "lowering")]
 
     def as_dict(self):
         return {name: getattr(self, name) for name, _ in self._fields_}
+
+
+class ConvShape(ctypes.Structure):
+    """conv_shape_t of the header: NHWC activations batch x h x w x c_in, c_out filters of kh x kw, strides, zero padding."""
+    _fields_ = [("batch", ctypes.c_int64), ("h", ctypes.c_int64), ("w", ctypes.c_int64), ("c_in", ctypes.c_int64),
+                ("c_out", ctypes.c_int64), ("kh", ctypes.c_int32), ("kw", ctypes.c_int32),
+                ("stride_h", ctypes.c_int32), ("stride_w", ctypes.c_int32), ("pad_h", ctypes.c_int32),
+                ("pad_w", ctypes.c_int32)]
 
 
 def _load() -> ctypes.CDLL:
@@ -64,6 +74,15 @@ def _load() -> ctypes.CDLL:
     lib.gemm_last_cuda_error.argtypes = []
     lib.gemm_selftest_wait_expiry.restype = ci
     lib.gemm_selftest_wait_expiry.argtypes = [vp]
+    sp = ctypes.POINTER(ConvShape)
+    lib.conv2d_im2row.restype = ci
+    lib.conv2d_im2row.argtypes = [ci, sp, cf, vp, vp, i64, cf, vp, i64, vp]
+    lib.im2row.restype = ci
+    lib.im2row.argtypes = [ci, sp, vp, vp, i64, vp]
+    lib.conv2d_workspace_bytes.restype = ctypes.c_size_t
+    lib.conv2d_workspace_bytes.argtypes = [ci, sp]
+    lib.conv2d_force_lowering.restype = ci
+    lib.conv2d_force_lowering.argtypes = [ci]
     lib.gemm_f32_splitk_static.restype = ci
     lib.gemm_f32_splitk_static.argtypes = [cc, cc, i64, i64, i64, cf, vp, i64, vp, i64, cf, vp, i64, ci, vp]
     return lib
@@ -139,3 +158,23 @@ def gemm_f32_splitk_static(transA, transB, m, n, k, alpha, A, lda, B, ldb, beta,
 def gemm_selftest_wait_expiry(stream=0) -> int:
     """Enqueue the kernel whose bounded wait is certain to expire; gemm_poll_status() then reports GEMM_ERR_DEVICE."""
     return _lib.gemm_selftest_wait_expiry(stream)
+
+
+def conv_shape(batch, h, w, c_in, c_out, kh, kw, stride_h=1, stride_w=1, pad_h=0, pad_w=0) -> ConvShape:
+    return ConvShape(batch, h, w, c_in, c_out, kh, kw, stride_h, stride_w, pad_h, pad_w)
+
+
+def conv2d_im2row(dtype, shape: ConvShape, alpha, X, W, ldw, beta, Y, ldy, stream=0) -> int:
+    return _lib.conv2d_im2row(dtype, ctypes.byref(shape), alpha, X, W, ldw, beta, Y, ldy, stream)
+
+
+def im2row(dtype, shape: ConvShape, X, out, ld, stream=0) -> int:
+    return _lib.im2row(dtype, ctypes.byref(shape), X, out, ld, stream)
+
+
+def conv2d_workspace_bytes(dtype, shape: ConvShape) -> int:
+    return int(_lib.conv2d_workspace_bytes(dtype, ctypes.byref(shape)))
+
+
+def conv2d_force_lowering(how) -> int:
+    return _lib.conv2d_force_lowering(how)

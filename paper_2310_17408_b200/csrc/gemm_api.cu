@@ -241,7 +241,7 @@ static Plan make_plan(const GemmArgs& a, int sms, size_t ws_avail) {
     Plan p{};
     p.ks = KSplit{1, a.k > 0 ? a.k : 1};
     int forced = g_force_kernel;
-    if (forced == GEMM_KERNEL_SIMT_GENERIC) { p.kernel = GEMM_KERNEL_SIMT_GENERIC; return p; }
+    if (forced == GEMM_KERNEL_SIMT_GENERIC && !a.conv) { p.kernel = GEMM_KERNEL_SIMT_GENERIC; return p; }
     if (a.dtype == GEMM_F32) {
         plan_simt(a, sms, ws_avail, &p);
         return p;
@@ -249,7 +249,9 @@ static Plan make_plan(const GemmArgs& a, int sms, size_t ws_avail) {
     // 16-bit inputs: tensor path if the operands are (or can be made) addressable by TMA
     auto aligned = [](const void* ptr, int64_t ld) { return (reinterpret_cast<uintptr_t>(ptr) & 15) == 0 && ld % 8 == 0; };
     GemmArgs probe = a;
-    const bool a_ok = aligned(a.A, a.lda), b_ok = aligned(a.B, a.ldb);
+    // a lowered convolution operand is fetched by TMA from the activation tensor: nothing of B to align or repack
+    const bool a_ok = aligned(a.A, a.lda), b_ok = a.conv ? true : aligned(a.B, a.ldb);
+    if (a.conv) { probe.B = nullptr; probe.ldb = 8; }
     if (!a_ok) { probe.A = nullptr; probe.lda = 8; }      // judged on the repacked layout
     if (!b_ok) { probe.B = nullptr; probe.ldb = 8; }
     if (!tensor_eligible(probe)) { p.kernel = GEMM_KERNEL_SIMT_GENERIC; return p; }
@@ -294,7 +296,7 @@ static int fail_launch(cudaError_t e) {
     return GEMM_ERR_LAUNCH;
 }
 
-static int run_gemm(const GemmArgs& a0, DeviceState* st) {
+static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
     GemmArgs a = a0;
     gemm_config_t cfg{};
     cfg.split_k = 1;
@@ -315,6 +317,11 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st) {
         std::lock_guard<std::mutex> lock(g_mutex);
         ws = st->ws;
         ws_bytes = st->ws_bytes;
+    }
+    if (ws_skip > 0) {      // the head of the workspace is in use by the caller (a lowered activation matrix)
+        if (ws == nullptr || ws_bytes < ws_skip) return GEMM_ERR_WORKSPACE;
+        ws = static_cast<uint8_t*>(ws) + ws_skip;
+        ws_bytes -= ws_skip;
     }
     Plan p = make_plan(a, st->sms, ws_bytes);
     if (p.kernel < 0) return GEMM_ERR_WORKSPACE;
@@ -363,6 +370,28 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st) {
     t_last_cfg = cfg;
     return e == cudaSuccess ? GEMM_OK : fail_launch(e);
 }
+
+// entry for the convolution front end (conv_api.cu)
+int dispatch_gemm(const GemmArgs& a, size_t ws_skip) {
+    DeviceState* st = device_state();
+    if (!st) return GEMM_ERR_LAUNCH;
+    if (!st->arch_ok) return GEMM_ERR_ARCH;
+    GemmArgs b = a;
+    b.status = st->status;
+    return run_gemm(b, st, ws_skip);
+}
+
+bool registered_workspace(void** ws, size_t* bytes) {
+    DeviceState* st = device_state();
+    if (!st) return false;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    *ws = st->ws;
+    *bytes = st->ws_bytes;
+    return true;
+}
+
+void note_lowering(int how) { t_last_cfg.lowering = how; }
+void note_launch_error(cudaError_t e) { t_last_cuda_error = (int)e; }
 
 }  // namespace b200gemm
 
@@ -639,6 +668,7 @@ const char* gemm_status_string(int code) {
         case -11: return "invalid argument 11 (ldb)";
         case -13: return "invalid argument 13 (C)";
         case -14: return "invalid argument 14 (ldc)";
+        case -15: return "invalid argument 15";
         default: return "unknown status";
     }
 }

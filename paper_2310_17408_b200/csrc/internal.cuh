@@ -9,6 +9,15 @@
 
 namespace b200gemm {
 
+// Index map of the im2row lowering (Section IV-C): when a call carries one, op(B) is not read from memory as a
+// stored matrix; its element (p, j) is the activation X(b, ho*sh - ph + r, wo*sw - pw + s, c) of an NHWC tensor, with
+// j = (b*Ho + ho)*Wo + wo and p = (r*kw + s)*C_in + c, and zero where the receptive field leaves the image.
+struct ConvIndex {
+    const void* X;             // NHWC activations, element type of the call
+    int64_t h, w, c_in;
+    int32_t ho, wo, kh, kw, sh, sw, ph, pw;
+};
+
 struct GemmArgs {
     int dtype;
     bool ta, tb;           // op(X) = X^T ?
@@ -20,6 +29,7 @@ struct GemmArgs {
     int64_t lda, ldb, ldc;
     cudaStream_t stream;
     uint32_t* status;      // device status word (bounded waits report here)
+    const ConvIndex* conv = nullptr;   // non-null: op(B) is the lowered activation matrix of this layer (B, ldb, tb unused)
 };
 
 // k partition used by every split-k path: split s covers [s*chunk, min(k, (s+1)*chunk))
@@ -85,5 +95,14 @@ cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t
 cudaError_t launch_wait_expiry_probe(uint32_t* status, cudaStream_t stream);
 
 int sm_count();
+
+// runs one GEMM (possibly with an im2row index map in a.conv) through the selector on the current device;
+// the first ws_skip bytes of the registered workspace are left alone
+int dispatch_gemm(const GemmArgs& a, size_t ws_skip);
+bool registered_workspace(void** ws, size_t* bytes);
+void note_lowering(int how);             // recorded in the calling thread's last configuration
+void note_launch_error(cudaError_t e);
+// whether TMA's im2col mode can do the lowering of this layer (defined with the tensor kernels)
+bool conv_tma_eligible(int dtype, const ConvIndex& cv, int64_t batch);
 
 }  // namespace b200gemm

@@ -110,6 +110,61 @@ struct Loader {
     }
 };
 
+// ---- operand B read through the im2row index map (the lowering fused into Pack-B): the tile's BN columns are
+// output pixels, its k index runs over (r, s, c).  Register layout and shared-memory store are those of the
+// k-contiguous Loader, so the rest of the kernel does not change.  VEC = 4 needs C_in % 4 == 0 and a 16-byte
+// aligned tensor: four consecutive k are then four consecutive channels of one filter tap.
+template <int X_TILE, int NT, int VEC>
+struct ConvLoader {
+    using L = Loader<X_TILE, NT, true, VEC>;
+    static constexpr int ELEMS = L::ELEMS, NV = L::NV;
+
+    // per load of the thread: element offset of pixel (b, ho*sh - ph, wo*sw - pw) and those two coordinates;
+    // a column past the last pixel gets coordinates that fail every bounds check
+    struct Pixel {
+        int64_t off;
+        int h0, w0;
+    };
+    __device__ static __forceinline__ Pixel pixel(const ConvIndex& cv, int64_t j, int64_t n) {
+        Pixel px;
+        if (j >= n) { px.off = 0; px.h0 = px.w0 = -(1 << 29); return px; }
+        const int hw = cv.ho * cv.wo;
+        const int b = (int)(j / hw), rem = (int)(j - (int64_t)b * hw);
+        const int oh = rem / cv.wo, ow = rem - oh * cv.wo;
+        px.h0 = oh * cv.sh - cv.ph;
+        px.w0 = ow * cv.sw - cv.pw;
+        px.off = (((int64_t)b * cv.h + px.h0) * cv.w + px.w0) * cv.c_in;
+        return px;
+    }
+
+    __device__ static __forceinline__ void load(float (&r)[ELEMS], const ConvIndex& cv, const Pixel (&px)[VEC == 4 ? NV : 1],
+                                                int64_t j0, int64_t k0, int64_t n, int64_t kmax, int t) {
+        const float* __restrict__ X = static_cast<const float*>(cv.X);
+        int x, kk;
+        L::coord(t, 0, x, kk);                    // kk is the same for every load of a thread
+        const int64_t p = k0 + kk;
+        const int tap = (int)(p / cv.c_in), c = (int)(p - (int64_t)tap * cv.c_in);
+        const int fr = tap / cv.kw, fs = tap - fr * cv.kw;
+        const bool k_ok = p < kmax;               // VEC = 4: k is a multiple of 4 here, so the four elements share it
+        const int64_t tap_off = ((int64_t)fr * cv.w + fs) * cv.c_in + c;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            if (VEC == 4) {
+                const int hi = px[v].h0 + fr, wi = px[v].w0 + fs;
+                float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (k_ok && (unsigned)hi < (unsigned)cv.h && (unsigned)wi < (unsigned)cv.w)
+                    q = __ldg(reinterpret_cast<const float4*>(X + px[v].off + tap_off));
+                r[v * 4 + 0] = q.x; r[v * 4 + 1] = q.y; r[v * 4 + 2] = q.z; r[v * 4 + 3] = q.w;
+            } else {
+                L::coord(t, v, x, kk);
+                const Pixel one = pixel(cv, j0 + x, n);
+                const int hi = one.h0 + fr, wi = one.w0 + fs;
+                r[v] = (k_ok && (unsigned)hi < (unsigned)cv.h && (unsigned)wi < (unsigned)cv.w) ? __ldg(X + one.off + tap_off) : 0.0f;
+            }
+        }
+    }
+};
+
 // Packed fp32 arithmetic: one fma.rn.f32x2 performs two independent IEEE fp32 fused multiply-adds (round to nearest
 // even, no flush to zero), lo = a.lo*b.lo + c.lo and hi = a.hi*b.hi + c.hi, in one issue slot.  It halves the
 // instructions of the products (issue slots used: 83 % -> 49 %); the FMA pipes themselves then set the pace.
@@ -185,15 +240,17 @@ __device__ __forceinline__ void unpack_block(const Acc2& p, float (&acc)[8][8]) 
         }
 }
 
-template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB>
-__global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
-simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
-                 const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
-                 int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, TailSplit tail) {
+template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB, bool CONV>
+__device__ __forceinline__ void
+simt_fast_body(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
+               const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
+               int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, const TailSplit& tail,
+               const ConvIndex& cv) {
     constexpr int NT = WARPS_M * WARPS_N * 32;
     static_assert(BM == WARPS_M * 64 && BN == WARPS_N * 32, "warp tile is 64 x 32");
     using LA = Loader<BM, NT, A_KCONT, VA>;
     using LB = Loader<BN, NT, B_KCONT, VB>;
+    using LC = ConvLoader<BN, NT, VB>;
 
     __shared__ __align__(16) float As[2][BK * (BM + PAD)];
     __shared__ __align__(16) float Bs[2][BK * (BN + PAD)];
@@ -246,17 +303,31 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
     const int64_t step_b = B_KCONT ? (int64_t)BK : (int64_t)BK * ldb;
     const int64_t fast_tiles = interior ? (kend - kbeg) / BK : 0;
 
+    // im2row index map: the pixels of this thread's loads are fixed for the whole k loop
+    typename LC::Pixel px[VB == 4 ? LC::NV : 1];
+    if (CONV && VB == 4) {
+#pragma unroll
+        for (int v = 0; v < LC::NV; ++v) {
+            int x, kk;
+            LB::coord(t, v, x, kk);
+            px[v] = LC::pixel(cv, j0 + x, n);
+        }
+    }
+
     auto gload = [&](int64_t kt) {
         if (kt < fast_tiles) {
             LA::load_fast(ra, pa, va);
-            LB::load_fast(rb, pb, vb);
             pa += step_a;
-            pb += step_b;
+            if (!CONV) {
+                LB::load_fast(rb, pb, vb);
+                pb += step_b;
+            }
         } else {
             const int64_t k0 = kbeg + kt * BK;
             LA::template load<true>(ra, A, lda, i0, k0, m, kend, t);
-            LB::template load<true>(rb, B, ldb, j0, k0, n, kend, t);
+            if (!CONV) LB::template load<true>(rb, B, ldb, j0, k0, n, kend, t);
         }
+        if (CONV) LC::load(rb, cv, px, j0, kbeg + kt * BK, n, kend, t);
     };
 
     asm volatile("griddepcontrol.wait;" ::: "memory");     // the previous kernel's results are visible from here on
@@ -334,6 +405,25 @@ simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __re
         }
 }
 
+template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB>
+__global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
+simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
+                 const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
+                 int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, TailSplit tail) {
+    simt_fast_body<BM, BN, WARPS_M, WARPS_N, MINB, A_KCONT, B_KCONT, VA, VB, false>(
+        m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, tiles_m, tiles_n, kchunk, partials, tail, ConvIndex{});
+}
+
+// the same kernel with operand B read through the im2row index map (n = output pixels, k = kh*kw*C_in)
+template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, int VA, int VB>
+__global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
+simt_conv_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
+                 float beta, float* __restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int64_t kchunk,
+                 float* __restrict__ partials, TailSplit tail, const ConvIndex cv) {
+    simt_fast_body<BM, BN, WARPS_M, WARPS_N, MINB, A_KCONT, true, VA, VB, true>(
+        m, n, k, alpha, A, lda, nullptr, k, beta, C, ldc, tiles_m, tiles_n, kchunk, partials, tail, cv);
+}
+
 // ---------------------------------------------------------------- host side
 
 bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb) {
@@ -364,10 +454,19 @@ static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gem
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
-    cudaError_t le = cudaLaunchKernelEx(&lc, simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB>, a.m, a.n, a.k, a.alpha,
-                                        (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
-                                        (int)tiles_m, (int)tiles_n, ks.chunk,
-                                        ks.splits > 1 ? partials : (float*)nullptr, tail);
+    cudaError_t le;
+    if constexpr (BKC) {
+        if (a.conv != nullptr) {      // operand B through the im2row index map (its memory layout is k-contiguous by construction)
+            le = cudaLaunchKernelEx(&lc, simt_conv_kernel<BM, BN, WM, WN, MINB, AK, VA, VB>, a.m, a.n, a.k, a.alpha,
+                                    (const float*)a.A, a.lda, a.beta, a.C, a.ldc, (int)tiles_m, (int)tiles_n, ks.chunk,
+                                    ks.splits > 1 ? partials : (float*)nullptr, tail, *a.conv);
+            return le != cudaSuccess ? le : cudaGetLastError();
+        }
+    }
+    le = cudaLaunchKernelEx(&lc, simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB>, a.m, a.n, a.k, a.alpha,
+                            (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
+                            (int)tiles_m, (int)tiles_n, ks.chunk,
+                            ks.splits > 1 ? partials : (float*)nullptr, tail);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
@@ -393,12 +492,14 @@ static cudaError_t launch_vec(const GemmArgs& a, int va, int vb, int tile, KSpli
 cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
     int va, vb;
     simt_fast_eligible(a, &va, &vb);
+    if (a.conv != nullptr)      // 128-bit loads need whole groups of four channels on 16-byte boundaries
+        vb = ((reinterpret_cast<uintptr_t>(a.conv->X) & 15) == 0 && a.conv->c_in % 4 == 0) ? 4 : 1;
     cfg->kernel = GEMM_KERNEL_SIMT_FAST;
     cfg->split_k = ks.splits;
     cfg->vector_a = va; cfg->vector_b = vb;
     // A is contiguous along k when transposed; B is contiguous along k when not transposed
-    if (!a.ta && !a.tb) return launch_vec<false, true>(a, va, vb, tile, ks, partials, cfg, tail);
-    if (a.ta && !a.tb) return launch_vec<true, true>(a, va, vb, tile, ks, partials, cfg, tail);
+    if (!a.ta && (!a.tb || a.conv)) return launch_vec<false, true>(a, va, vb, tile, ks, partials, cfg, tail);
+    if (a.ta && (!a.tb || a.conv)) return launch_vec<true, true>(a, va, vb, tile, ks, partials, cfg, tail);
     if (!a.ta && a.tb) return launch_vec<false, false>(a, va, vb, tile, ks, partials, cfg, tail);
     return launch_vec<true, false>(a, va, vb, tile, ks, partials, cfg, tail);
 }

@@ -60,6 +60,34 @@ __device__ __forceinline__ void tma_load_2d(const CUtensorMap* tm, uint32_t dst,
         ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
+// TMA load in im2col mode from an NHWC tensor (tensor map dimensions C, W, H, N): the box holds `pixelsPerColumn`
+// consecutive output pixels starting at the one whose receptive field begins at (w, h) of image n, each with
+// `channelsPerPixel` channels from c on, read at filter-tap offset (off_w, off_h); positions outside the image are
+// zero-filled.  Rows of the box are pixels, so the stage is the K-major operand tile of the lowered matrix.
+__device__ __forceinline__ void tma_load_im2col(const CUtensorMap* tm, uint32_t dst, uint32_t bar, int32_t c, int32_t w,
+                                                int32_t h, int32_t n, uint16_t off_w, uint16_t off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+}
+
+// geometry the producer needs to turn (tile column, k block) into im2col coordinates
+struct ConvTma {
+    int32_t ho, wo;        // output extent
+    int32_t stride, pad;   // same in both directions
+    int32_t kw;            // filter width
+    int32_t chunks;        // C_in / 64: k blocks per filter tap
+};
+// first pixel j of a tile -> tensor coordinates of its receptive field's corner
+__device__ __forceinline__ void conv_tile_origin(const ConvTma& cv, int64_t j, int32_t& w, int32_t& h, int32_t& n) {
+    const int hw = cv.ho * cv.wo;
+    n = (int32_t)(j / hw);
+    const int rem = (int)(j - (int64_t)n * hw);
+    const int oh = rem / cv.wo, ow = rem - oh * cv.wo;
+    w = ow * cv.stride - cv.pad;
+    h = oh * cv.stride - cv.pad;
+}
+
 // shared memory -> global tile store (bulk async group); out-of-range parts of the box are clipped by the hardware
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int32_t c0, int32_t c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
@@ -186,6 +214,15 @@ bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_
 bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits);
 // map over the fp32 result for the epilogue's tile stores: 32 x 32 boxes, no swizzle
 bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc);
+// im2col-mode map over NHWC activations of a 16-bit type: boxes of `pixels` output pixels x 64 channels, 128-byte
+// swizzle; square filter ksize, the same stride and padding in both directions
+bool make_im2col_map(CUtensorMap* tm, int dtype, const ConvIndex& cv, int64_t batch, uint32_t pixels);
+// whether the lowering of this layer can be done by TMA (channel count, alignment, symmetric geometry, field ranges)
+bool conv_tma_eligible(int dtype, const ConvIndex& cv, int64_t batch);
+inline ConvTma conv_tma_params(const ConvIndex* cv) {
+    if (!cv) return ConvTma{1, 1, 1, 0, 1, 1};
+    return ConvTma{cv->ho, cv->wo, cv->sh, cv->ph, cv->kw, (int32_t)(cv->c_in / 64)};
+}
 // instruction descriptor of tcgen05.mma kind::f16 with fp32 accumulation: mma_m x mma_n, operand majorness
 uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n);
 

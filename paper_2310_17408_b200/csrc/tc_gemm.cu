@@ -31,12 +31,14 @@ template <int BN> struct TcCfg {
 };
 
 // A_MN: op(A) is contiguous along m in memory (transA = N); B_MN: op(B) contiguous along n (transB = T).
-template <int BN, bool A_MN, bool B_MN>
+// CONV: op(B) is the im2row-lowered activation matrix of a convolution layer, fetched by TMA in im2col mode
+// straight from the NHWC tensor (tmB is then an im2col map); the lowered matrix never exists in memory.
+template <int BN, bool A_MN, bool B_MN, bool CONV>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
-               uint32_t idesc, uint32_t* status) {
+               uint32_t idesc, uint32_t* status, const ConvTma conv) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -108,6 +110,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 int64_t kbeg;
                 const int kb_n = kblocks_of(sp, kbeg);
                 const int32_t m0 = tm * TBM, n0 = tn * BN;
+                int32_t cw = 0, ch = 0, cn = 0;
+                if (CONV) conv_tile_origin(conv, (int64_t)tn * BN, cw, ch, cn);
                 for (int kb = 0; kb < kb_n; ++kb, ++cnt) {
                     const int s = cnt % STAGES;
                     const uint32_t ph = (cnt / STAGES) & 1;
@@ -123,7 +127,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else {
                         tma_load_2d(&tmA, sa, full_bar(s), k0, m0);
                     }
-                    if (B_MN) {
+                    if (CONV) {
+                        const int kg = k0 / TBK;                     // k block -> filter tap and channel chunk
+                        const int tap = kg / conv.chunks, c0 = (kg - tap * conv.chunks) * TBK;
+                        const int fr = tap / conv.kw, fs = tap - fr * conv.kw;
+                        tma_load_im2col(&tmB, sb, full_bar(s), c0, cw, ch, cn, (uint16_t)fs, (uint16_t)fr);
+                    } else if (B_MN) {
 #pragma unroll
                         for (int c = 0; c < BN / 64; ++c) tma_load_2d(&tmB, sb + c * (64 * TBK * 2), full_bar(s), n0 + c * 64, k0);
                     } else {
@@ -307,6 +316,51 @@ bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_
     return r == CUDA_SUCCESS;
 }
 
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+static EncodeIm2colFn encode_im2col_fn() {
+    static EncodeIm2colFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeIm2colFn>(p);
+    }
+    return fn;
+}
+
+bool conv_tma_eligible(int dtype, const ConvIndex& cv, int64_t batch) {
+    if (dtype != GEMM_F16 && dtype != GEMM_BF16) return false;
+    if (cv.c_in % 64 != 0 || (reinterpret_cast<uintptr_t>(cv.X) & 15) != 0) return false;
+    if (cv.kh != cv.kw || cv.sh != cv.sw || cv.ph != cv.pw) return false;      // one corner / stride value serves both directions
+    if (cv.sh < 1 || cv.sh > 8 || cv.ph > 127 || cv.kh > 128 || cv.ph - (cv.kh - 1) < -128) return false;   // field ranges of the map
+    if (cv.kh > 255) return false;                                             // filter offsets travel as 16-bit values
+    if (cv.h > 0x7FFFFFFF || cv.w > 0x7FFFFFFF || batch > 0x7FFFFFFF) return false;
+    if (cv.w * cv.c_in * 2 >= (1LL << 40) || cv.h * cv.w * cv.c_in * 2 >= (1LL << 40)) return false;
+    return encode_im2col_fn() != nullptr;
+}
+
+bool make_im2col_map(CUtensorMap* tm, int dtype, const ConvIndex& cv, int64_t batch, uint32_t pixels) {
+    EncodeIm2colFn fn = encode_im2col_fn();
+    if (!fn) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)cv.c_in, (cuuint64_t)cv.w, (cuuint64_t)cv.h, (cuuint64_t)batch};
+    cuuint64_t strides[3] = {(cuuint64_t)cv.c_in * 2, (cuuint64_t)cv.w * cv.c_in * 2, (cuuint64_t)cv.h * cv.w * cv.c_in * 2};
+    // receptive-field corners may start at -pad and must stop where the last filter tap still touches image + pad
+    int lower[2] = {-cv.pw, -cv.ph};
+    int upper[2] = {cv.pw - (cv.kw - 1), cv.ph - (cv.kh - 1)};
+    cuuint32_t estr[4] = {1, (cuuint32_t)cv.sw, (cuuint32_t)cv.sh, 1};
+    CUresult r = fn(tm, dtype == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+                    const_cast<void*>(cv.X), dims, strides, lower, upper, 64, pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool tensor_eligible(const GemmArgs& a) {
     if (a.dtype != GEMM_F16 && a.dtype != GEMM_BF16) return false;
     auto ok = [](const void* p, int64_t ld) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0 && ld % 8 == 0; };
@@ -329,13 +383,13 @@ uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n) {
     return d;
 }
 
-template <int BN, bool A_MN, bool B_MN>
+template <int BN, bool A_MN, bool B_MN, bool CONV>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
                              const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
     static bool attr_set[64] = {};
-    auto kern = tc_gemm_kernel<BN, A_MN, B_MN>;
+    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
@@ -361,19 +415,23 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN), a.status);
+                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN), a.status, conv_tma_params(a.conv));
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool CONV>
 static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg) {
     CUtensorMap tmA, tmB;
     // stored A: (m x k) if transA = N [contiguous m], (k x m) otherwise [contiguous k]
     bool ok = A_MN ? make_map(&tmA, a.dtype, a.A, a.m, a.k, a.lda, 64, TBK)
                    : make_map(&tmA, a.dtype, a.A, a.k, a.m, a.lda, TBK, TBM);
     // stored B: (k x n) if transB = N [contiguous k], (n x k) otherwise [contiguous n]
-    ok = ok && (B_MN ? make_map(&tmB, a.dtype, a.B, a.n, a.k, a.ldb, 64, TBK)
-                     : make_map(&tmB, a.dtype, a.B, a.k, a.n, a.ldb, TBK, (uint32_t)tile_n));
+    if (CONV) {      // n = batch * Ho * Wo pixels
+        ok = ok && make_im2col_map(&tmB, a.dtype, *a.conv, a.n / ((int64_t)a.conv->ho * a.conv->wo), (uint32_t)tile_n);
+    } else {
+        ok = ok && (B_MN ? make_map(&tmB, a.dtype, a.B, a.n, a.k, a.ldb, 64, TBK)
+                         : make_map(&tmB, a.dtype, a.B, a.k, a.n, a.ldb, TBK, (uint32_t)tile_n));
+    }
     if (!ok) return cudaErrorInvalidValue;
     // the result goes out through TMA tile stores when C is 16-byte addressable and this is not a split-k pass
     CUtensorMap tmC = tmA;
@@ -385,9 +443,9 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
         a.m * a.n * 4 < (1LL << 40))
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
     switch (tile_n) {
-        case 256: return launch_tc<256, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        case 128: return launch_tc<128, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        default:  return launch_tc<64, A_MN, B_MN>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 256: return launch_tc<256, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 128: return launch_tc<128, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        default:  return launch_tc<64, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
     }
 }
 
@@ -396,10 +454,13 @@ cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* parti
     cfg->split_k = ks.splits;
     cfg->vector_a = cfg->vector_b = 1;
     const bool a_mn = !a.ta, b_mn = a.tb;
-    if (a_mn && b_mn) return launch_tc_bn<true, true>(a, tile_n, ks, partials, cfg);
-    if (a_mn && !b_mn) return launch_tc_bn<true, false>(a, tile_n, ks, partials, cfg);
-    if (!a_mn && b_mn) return launch_tc_bn<false, true>(a, tile_n, ks, partials, cfg);
-    return launch_tc_bn<false, false>(a, tile_n, ks, partials, cfg);
+    if (a.conv != nullptr)
+        return a_mn ? launch_tc_bn<true, false, true>(a, tile_n, ks, partials, cfg)
+                    : launch_tc_bn<false, false, true>(a, tile_n, ks, partials, cfg);
+    if (a_mn && b_mn) return launch_tc_bn<true, true, false>(a, tile_n, ks, partials, cfg);
+    if (a_mn && !b_mn) return launch_tc_bn<true, false, false>(a, tile_n, ks, partials, cfg);
+    if (!a_mn && b_mn) return launch_tc_bn<false, true, false>(a, tile_n, ks, partials, cfg);
+    return launch_tc_bn<false, false, false>(a, tile_n, ks, partials, cfg);
 }
 
 }  // namespace b200gemm

@@ -53,6 +53,12 @@ __device__ __forceinline__ void tma_load_2d_pair(const CUtensorMap* tm, uint32_t
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tm), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
 }
+__device__ __forceinline__ void tma_load_im2col_pair(const CUtensorMap* tm, uint32_t dst, uint32_t bar_cluster, int32_t c,
+                                                     int32_t w, int32_t h, int32_t n, uint16_t off_w, uint16_t off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(dst), "l"(tm), "r"(bar_cluster), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+}
 __device__ __forceinline__ void umma_f16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
@@ -66,12 +72,13 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t mask) {
                  ::"r"(bar), "h"(mask) : "memory");
 }
 
-template <bool A_MN, bool B_MN>
+// CONV: op(B) is the lowered activation matrix of a convolution layer, fetched in im2col mode (see tc_gemm.cu)
+template <bool A_MN, bool B_MN, bool CONV>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k,
                     float alpha, float beta, float* __restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int splits,
-                    int64_t kchunk, float* __restrict__ partials, uint32_t idesc, uint32_t* status) {
+                    int64_t kchunk, float* __restrict__ partials, uint32_t idesc, uint32_t* status, const ConvTma conv) {
     constexpr int STAGES = PAIR_STAGES, NACC = PAIR_NACC, BN = PAIR_BN;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -143,6 +150,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int kb_n = kblocks_of(sp, kbeg);
                 const int32_t m0 = tm * (2 * TBM) + (int32_t)rank * TBM;            // this CTA's rows of op(A)
                 const int32_t n0 = tn * BN + (int32_t)rank * PAIR_HALF_N;           // this CTA's columns of op(B)
+                int32_t cw = 0, ch = 0, cn = 0;
+                if (CONV) conv_tile_origin(conv, (int64_t)tn * BN + (int64_t)rank * PAIR_HALF_N, cw, ch, cn);
                 for (int kb = 0; kb < kb_n; ++kb, ++cnt) {
                     const int s = cnt % STAGES;
                     const uint32_t ph = (cnt / STAGES) & 1;
@@ -159,7 +168,12 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     } else {
                         tma_load_2d_pair(&tmA, sa, fb, k0, m0);
                     }
-                    if (B_MN) {
+                    if (CONV) {
+                        const int kg = k0 / TBK;
+                        const int tap = kg / conv.chunks, c0 = (kg - tap * conv.chunks) * TBK;
+                        const int fr = tap / conv.kw, fs = tap - fr * conv.kw;
+                        tma_load_im2col_pair(&tmB, sb, fb, c0, cw, ch, cn, (uint16_t)fs, (uint16_t)fr);
+                    } else if (B_MN) {
 #pragma unroll
                         for (int c = 0; c < PAIR_HALF_N / 64; ++c) tma_load_2d_pair(&tmB, sb + c * (64 * TBK * 2), fb, n0 + c * 64, k0);
                     } else {
@@ -260,13 +274,17 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool CONV>
 static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg) {
     CUtensorMap tmA, tmB;
     bool ok = A_MN ? make_map(&tmA, a.dtype, a.A, a.m, a.k, a.lda, 64, TBK)
                    : make_map(&tmA, a.dtype, a.A, a.k, a.m, a.lda, TBK, TBM);
-    ok = ok && (B_MN ? make_map(&tmB, a.dtype, a.B, a.n, a.k, a.ldb, 64, TBK)
-                     : make_map(&tmB, a.dtype, a.B, a.k, a.n, a.ldb, TBK, PAIR_HALF_N));
+    if (CONV) {
+        ok = ok && make_im2col_map(&tmB, a.dtype, *a.conv, a.n / ((int64_t)a.conv->ho * a.conv->wo), PAIR_HALF_N);
+    } else {
+        ok = ok && (B_MN ? make_map(&tmB, a.dtype, a.B, a.n, a.k, a.ldb, 64, TBK)
+                         : make_map(&tmB, a.dtype, a.B, a.k, a.n, a.ldb, TBK, PAIR_HALF_N));
+    }
     if (!ok) return cudaErrorInvalidValue;
     CUtensorMap tmC = tmA;
     int store_via_tma = 0;
@@ -276,7 +294,7 @@ static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, ge
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
 
     static bool attr_set[64] = {};
-    auto kern = tc_gemm_pair_kernel<A_MN, B_MN>;
+    auto kern = tc_gemm_pair_kernel<A_MN, B_MN, CONV>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
@@ -307,7 +325,7 @@ static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status);
+                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status, conv_tma_params(a.conv));
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
@@ -316,10 +334,12 @@ cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     cfg->split_k = ks.splits;
     cfg->vector_a = cfg->vector_b = 1;
     const bool a_mn = !a.ta, b_mn = a.tb;
-    if (a_mn && b_mn) return launch_pair<true, true>(a, ks, partials, cfg);
-    if (a_mn && !b_mn) return launch_pair<true, false>(a, ks, partials, cfg);
-    if (!a_mn && b_mn) return launch_pair<false, true>(a, ks, partials, cfg);
-    return launch_pair<false, false>(a, ks, partials, cfg);
+    if (a.conv != nullptr)
+        return a_mn ? launch_pair<true, false, true>(a, ks, partials, cfg) : launch_pair<false, false, true>(a, ks, partials, cfg);
+    if (a_mn && b_mn) return launch_pair<true, true, false>(a, ks, partials, cfg);
+    if (a_mn && !b_mn) return launch_pair<true, false, false>(a, ks, partials, cfg);
+    if (!a_mn && b_mn) return launch_pair<false, true, false>(a, ks, partials, cfg);
+    return launch_pair<false, false, false>(a, ks, partials, cfg);
 }
 
 }  // namespace b200gemm

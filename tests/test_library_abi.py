@@ -11,7 +11,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "b200_gemm.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = re.findall(r"^\s*(?:const\s+char\s*\*|int|size_t|uint32_t)\s+(gemm\w*)\s*\(", text, flags=re.M)
+    names = re.findall(r"^\s*(?:const\s+char\s*\*|int|size_t|uint32_t)\s+((?:gemm|conv2d|im2row)\w*)\s*\(", text, flags=re.M)
     return sorted(set(names))
 
 
@@ -32,6 +32,20 @@ def test_argument_checks_run_without_a_device():
     assert g.gemm(0, "N", "N", 0, 4, 4, 1.0, 0, 1, 0, 4, 0.0, 0, 1) == 0       # m == 0: nothing to do
     assert "lda" in g.gemm_status_string(-9)
     assert g.gemm_force_kernel(99) == -1 and g.gemm_force_kernel(0) == 0
+
+
+def test_convolution_argument_checks_run_without_a_device():
+    s = g.conv_shape(1, 4, 4, 4, 4, 5, 5, 1, 1, 0, 0)              # filter larger than the padded image
+    assert g.conv2d_im2row(0, s, 1.0, 16, 16, 4, 0.0, 16, 4) == -2
+    s = g.conv_shape(2, 8, 8, 4, 6, 3, 3, 1, 1, 1, 1)
+    assert g.conv2d_im2row(9, s, 1.0, 16, 16, 6, 0.0, 16, 6) == -1
+    assert g.conv2d_im2row(0, s, 1.0, 16, 16, 5, 0.0, 16, 6) == -6
+    assert g.im2row(0, s, 16, 16, 35) == -5                         # ld < k = 36
+    assert g.conv2d_force_lowering(7) == -1 and g.conv2d_force_lowering(0) == 0
+    # a layer whose lowered matrix must be written asks for room for it: k = 27 padded to 32 rows, 2 bytes each
+    s = g.conv_shape(4, 32, 32, 3, 64, 3, 3, 1, 1, 1, 1)
+    assert g.conv2d_workspace_bytes(2, s) >= 32 * 4 * 32 * 32 * 2
+    assert g.conv2d_workspace_bytes(0, s) == g.gemm_workspace_bytes(0, "N", "N", 64, 4 * 32 * 32, 27)   # fp32: fused
 
 
 def test_workspace_request_for_split_k_shapes():
