@@ -28,7 +28,8 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-from workloads import DTYPE_BF16, DTYPE_F16, DTYPE_F32, DTYPE_NAMES, config_problems, im2row_problems  # noqa: E402
+from workloads import (DTYPE_BF16, DTYPE_F16, DTYPE_F32, DTYPE_NAMES, config_problems, conv_layer_problems,  # noqa: E402
+                       im2row_problems)
 
 SM_COUNT = 148
 FP32_LANES_PER_SM = 128
@@ -47,6 +48,14 @@ WORKLOADS = {
     "vgg16_fp32_paper_orientation": lambda: im2row_problems("vgg16", weights_as_A=False),
     "resnet50_fp32_paper_orientation": lambda: im2row_problems("resnet50", weights_as_A=False),
     "resnet50_bf16_paper_orientation": lambda: im2row_problems("resnet50", weights_as_A=False, dtype=DTYPE_BF16),
+}
+# the convolution layers themselves (NHWC activations in, NHWC result out): lowering fused into the GEMM kernels,
+# timed beside the explicit route (im2row pass + gemm) and beside the GEMM alone on an already lowered matrix
+CONV_WORKLOADS = {
+    "resnet50_conv_fp32": lambda: conv_layer_problems("resnet50"),
+    "resnet50_conv_bf16": lambda: conv_layer_problems("resnet50", dtype=DTYPE_BF16),
+    "vgg16_conv_fp32": lambda: conv_layer_problems("vgg16"),
+    "vgg16_conv_bf16": lambda: conv_layer_problems("vgg16", dtype=DTYPE_BF16),
 }
 
 
@@ -508,13 +517,115 @@ def run_cuda(args, problems, workload_name):
     return 0
 
 
+# ------------------------------------------------------------------------------------------ convolution layers
+
+def run_conv_layers(args, layers, workload_name):
+    """One step = every layer of the network once through conv2d_im2row (the selector's route).  Per layer it also
+    times the explicit route (im2row pass + gemm) and gemm alone on a lowered matrix that is already in memory
+    (what the paper's experiment measures), all cold-cache: calls cycle through enough operand sets to exceed L2."""
+    import torch
+    import paper_2310_17408_b200 as g
+
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream().cuda_stream
+    shapes = [g.conv_shape(p.batch, p.h, p.w, p.c_in, p.c_out, p.kh, p.kw, p.stride, p.stride, p.pad, p.pad) for p in layers]
+    g.conv2d_force_lowering(g.CONV_LOWERING_EXPLICIT)
+    ws_need = max(g.conv2d_workspace_bytes(p.dtype, s) for p, s in zip(layers, shapes))
+    g.conv2d_force_lowering(0)
+    ws = torch.empty(ws_need + (64 << 20), dtype=torch.uint8, device="cuda")
+    assert g.gemm_set_workspace(ws.data_ptr(), ws.numel(), 0) == 0
+    rows, step_ms, step_flops, launches = [], 0.0, 0.0, 0
+    sampler = ClockSampler(0)
+    sampler.start()
+    wall_begin = time.time()
+    for p, shp in zip(layers, shapes):
+        X, W, Y0 = p.operands()
+        view = (lambda x: x.view(np.int16)) if p.dtype != DTYPE_F32 else (lambda x: x)
+        m, n, k = p.gemm_mnk
+        es = 4 if p.dtype == DTYPE_F32 else 2
+        nsets = int(min(16, max(1, -(-2 * 126e6 // p.algorithmic_bytes()))))
+        dX = [torch.from_numpy(view(X.buf)).cuda() for _ in range(nsets)]
+        dW = [torch.from_numpy(view(W.buf)).cuda() for _ in range(nsets)]
+        dY = [torch.from_numpy(Y0.buf).cuda() for _ in range(nsets)]
+
+        def timed(call, reps):
+            for r in range(3):
+                call(r)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for r in range(reps):
+                call(r)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        def conv_call(r):
+            i = r % nsets
+            rc = g.conv2d_im2row(p.dtype, shp, p.alpha, dX[i].data_ptr(), dW[i].data_ptr(), W.ld, p.beta, dY[i].data_ptr(), Y0.ld, stream)
+            if rc != 0:
+                raise RuntimeError(f"conv2d_im2row failed on {p.name}: {g.gemm_status_string(rc)}")
+
+        reps = max(args.steps, 10)
+        ms_auto = timed(conv_call, reps)
+        cfg = g.gemm_last_config()
+        launches += reps * (cfg["launches"] + (1 if cfg["lowering"] == g.CONV_LOWERING_EXPLICIT else 0))
+        g.conv2d_force_lowering(g.CONV_LOWERING_EXPLICIT)
+        ms_explicit = timed(conv_call, reps)
+        g.conv2d_force_lowering(0)
+        # gemm alone on a lowered matrix that already exists (one copy: k x pixels can be hundreds of MB)
+        ld = -(-k // 8) * 8
+        low = torch.empty(ld * n, dtype=dX[0].dtype, device="cuda")
+        assert g.im2row(p.dtype, shp, dX[0].data_ptr(), low.data_ptr(), ld, stream) == 0
+
+        def gemm_call(r):
+            i = r % nsets
+            rc = g.gemm(p.dtype, "N", "N", m, n, k, p.alpha, dW[i].data_ptr(), W.ld, low.data_ptr(), ld, p.beta, dY[i].data_ptr(), Y0.ld, stream)
+            if rc != 0:
+                raise RuntimeError(g.gemm_status_string(rc))
+        ms_gemm = timed(gemm_call, reps)
+        del low
+        bound, peak, unit, amount = roofline_class(p, peaks)
+        rows.append({"name": p.name, "layer": f"{p.c_in}->{p.c_out} {p.kh}x{p.kw}/{p.stride} on {p.h}x{p.w}", "m": m, "n": n, "k": k,
+                     "lowering": {1: "fused", 2: "explicit", 3: "identity"}.get(cfg["lowering"], "?"),
+                     "kernel": cfg["kernel"], "tile": [cfg["tile_m"], cfg["tile_n"]], "split_k": cfg["split_k"],
+                     "ms": ms_auto, "ms_explicit_route": ms_explicit, "ms_gemm_on_lowered": ms_gemm,
+                     "tflops": p.flops / (ms_auto * 1e-3) / 1e12, "gbs": p.algorithmic_bytes() / (ms_auto * 1e-3) / 1e9,
+                     "lowered_matrix_mb": ld * n * es / 1e6, "bound": bound, "frac": amount / (ms_auto * 1e-3) / peak})
+        step_ms += ms_auto
+        step_flops += p.flops
+        del dX, dW, dY
+        torch.cuda.empty_cache()
+    clocks = sampler.stop(wall_begin, time.time())
+    if g.gemm_poll_status() != 0:
+        raise RuntimeError(f"device status {hex(g.gemm_status_detail())}")
+    dom = max(rows, key=lambda r: r["ms"])
+    line = {"metric": "gemm_tflops", "value": step_flops / (step_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": 1,
+            "steps": max(args.steps, 10), "warmup": 3, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": DTYPE_NAMES[layers[0].dtype], "data": "synthetic",
+            "config": {"workload": workload_name, "batch": layers[0].batch, "layout": "NHWC activations, C_out x k filters",
+                       "l2": "calls cycle through operand sets larger than L2", "parallelism": "single GPU",
+                       "step": "sum over the layers of the per-layer cold-cache time"},
+            "roofline": {"bound": dom["bound"], "achieved": dom["tflops"] if dom["bound"] != "hbm" else dom["gbs"],
+                         "peak": roofline_class(layers[rows.index(dom)], peaks)[1],
+                         "unit": "GB/s" if dom["bound"] == "hbm" else "TFLOP/s", "frac": dom["frac"], "traffic": None,
+                         "kernel": "conv2d_im2row (" + dom["lowering"] + ")", "problem": dom["name"]},
+            "clocks": clocks, "gpu_launches": launches, "shapes": rows}
+    print(json.dumps(line))
+    if args.table:
+        with open(args.table, "w") as f:
+            json.dump(line, f, indent=1)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS) + sorted(CONV_WORKLOADS))
     ap.add_argument("--shape", default=None, help="M,N,K: time this single problem instead of a workload (alpha=1, beta=0)")
     ap.add_argument("--dtype", default="f32", choices=["f32", "f16", "bf16"], help="operand type for --shape")
     ap.add_argument("--alpha", type=float, default=1.0, help="alpha for --shape")
@@ -525,6 +636,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-budget", type=float, default=30.0)
     args = ap.parse_args()
+    if args.workload in CONV_WORKLOADS:
+        return run_conv_layers(args, CONV_WORKLOADS[args.workload](), args.workload)
     problems = WORKLOADS[args.workload]()
     if args.shape:
         from workloads import Problem

@@ -161,15 +161,19 @@ int gemm_f32_splitk_static(char transA, char transB, int64_t m, int64_t n, int64
  *             beta != 0; rows C_out..ldy-1 are never touched
  *   Where it can, the lowering is fused into the operand staging of the GEMM kernels and L never exists in memory:
  *   fp32 reads X through the index map inside the SIMT kernel's loads; fp16/bf16 layers with C_in a multiple of
- *   64, a 16-byte aligned X, square filters and the same stride and padding in both directions let TMA's im2col
- *   mode deliver the swizzled tiles.  1 x 1 layers with stride 1 and no padding need no lowering (L is X).  All other
- *   cases first write L into the registered workspace with im2row() and then run gemm() on it; they return
- *   GEMM_ERR_WORKSPACE if the workspace is smaller than conv2d_workspace_bytes().
+ *   64, a 16-byte aligned X, filters TMA can address (16-byte aligned W, ldw a multiple of 8), square filters and
+ *   the same stride and padding in both directions let TMA's im2col mode deliver the swizzled tiles.  1 x 1 layers
+ *   with stride 1 and no padding need no lowering (L is X).  All other fp16/bf16 layers first write L into the
+ *   registered workspace with im2row() and then run gemm() on it; they return GEMM_ERR_WORKSPACE if the workspace
+ *   is smaller than conv2d_workspace_bytes().  fp32 layers whose C_in is not a multiple of 4 (or whose X is not
+ *   16-byte aligned) take that explicit route too when the workspace has room, because the index map then needs
+ *   scalar loads; without room they stay fused.
  *   Returns GEMM_OK, -(position of the first invalid argument) (2 = a field of *shape), or a GEMM_ERR_* code.
  *   Asynchronous on `stream`, like gemm().
  *
  *   im2row          the transform by itself: writes L (element type of X, leading dimension ld >= k, column-major,
  *                   16-byte chunks when alignment allows) to `out`.  An HBM-bound copy: C_in*kh*kw*pixels elements.
+ *                   Rows k..ld-1 of a column are either left untouched or set to zero.
  */
 typedef struct {
     int64_t batch, h, w, c_in, c_out;

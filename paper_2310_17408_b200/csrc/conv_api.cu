@@ -11,33 +11,51 @@ static int g_force_lowering = 0;
 static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline int64_t rup(int64_t a, int64_t b) { return cdiv(a, b) * b; }
 
-// ---- the transform as a copy kernel: one thread per 16-byte chunk (CHUNK = true) or per element of L.
-// Column j of L is the patch of output pixel j; a (pixel, tap) pair is C_in contiguous elements of X or zeros.
-template <typename T, bool CHUNK>
+// ---- the transform as a copy kernel.  Column j of L is the patch of output pixel j: kh*kw runs of C_in contiguous
+// elements of X (or zeros).  Three forms, by what the alignment allows:
+//   MODE 0  one thread per 16-byte chunk, loaded and stored whole (C_in a multiple of the chunk, everything aligned)
+//   MODE 1  one thread per 16-byte chunk of L, gathered element by element and stored whole (any C_in; L aligned);
+//           rows k..ld-1 that fall into a chunk are written as zeros
+//   MODE 2  one thread per element (no alignment at all)
+template <typename T, int MODE>
 __global__ void __launch_bounds__(256)
-im2row_kernel(const ConvIndex cv, int64_t pixels, const T* __restrict__ X, T* __restrict__ out, int64_t ld) {
-    constexpr int PER = CHUNK ? (int)(16 / sizeof(T)) : 1;          // elements moved by one thread
-    const int64_t per_tap = cv.c_in / PER;                          // threads per (pixel, tap)
-    const int64_t taps = (int64_t)cv.kh * cv.kw;
-    const int64_t total = pixels * taps * per_tap;
-    const int hw = cv.ho * cv.wo;
+im2row_kernel(const ConvIndex cv, int64_t pixels, int k, const T* __restrict__ X, T* __restrict__ out, int64_t ld) {
+    constexpr int PER = MODE == 2 ? 1 : (int)(16 / sizeof(T));      // elements of L written by one thread
+    const uint32_t cin = (uint32_t)cv.c_in, kw = (uint32_t)cv.kw;
+    const uint32_t per_col = MODE == 1 ? (uint32_t)(ld / PER) : (uint32_t)(k / PER);     // threads per column of L
+    const int64_t total = pixels * per_col;
+    const uint32_t hw = (uint32_t)(cv.ho * cv.wo);
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t j = idx / (taps * per_tap);
-        const int64_t within = idx - j * (taps * per_tap);
-        const int tap = (int)(within / per_tap);
-        const int64_t c = (within - (int64_t)tap * per_tap) * PER;
-        const int fr = tap / cv.kw, fs = tap - fr * cv.kw;
-        const int b = (int)(j / hw), rem = (int)(j - (int64_t)b * hw);
-        const int oh = rem / cv.wo, ow = rem - oh * cv.wo;
-        const int hi = oh * cv.sh - cv.ph + fr, wi = ow * cv.sw - cv.pw + fs;
-        const bool inside = (unsigned)hi < (unsigned)cv.h && (unsigned)wi < (unsigned)cv.w;
-        const int64_t src = (((int64_t)b * cv.h + hi) * cv.w + wi) * cv.c_in + c;
-        const int64_t dst = j * ld + (int64_t)tap * cv.c_in + c;
-        if (CHUNK) {
-            const uint4 v = inside ? __ldg(reinterpret_cast<const uint4*>(X + src)) : make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4*>(out + dst) = v;
+        const int64_t j = idx / per_col;
+        const uint32_t p0 = (uint32_t)(idx - j * per_col) * PER;     // first row of L this thread writes
+        const uint32_t b = (uint32_t)(j / hw), rem = (uint32_t)(j - (int64_t)b * hw);
+        const int oh = (int)(rem / (uint32_t)cv.wo), ow = (int)(rem - (uint32_t)oh * (uint32_t)cv.wo);
+        const int h0 = oh * cv.sh - cv.ph, w0 = ow * cv.sw - cv.pw;
+        const int64_t base = (((int64_t)b * cv.h + h0) * cv.w + w0) * cv.c_in;
+        auto source = [&](uint32_t p, bool& inside) {      // element offset in X of row p of this column
+            const uint32_t tap = p / cin, c = p - tap * cin;
+            const int fr = (int)(tap / kw), fs = (int)(tap - (uint32_t)fr * kw);
+            inside = p < (uint32_t)k && (unsigned)(h0 + fr) < (unsigned)cv.h && (unsigned)(w0 + fs) < (unsigned)cv.w;
+            return base + ((int64_t)fr * cv.w + fs) * cv.c_in + c;
+        };
+        T* dst = out + j * ld + p0;
+        if (MODE == 0) {
+            bool inside;
+            const int64_t src = source(p0, inside);
+            *reinterpret_cast<uint4*>(dst) = inside ? __ldg(reinterpret_cast<const uint4*>(X + src)) : make_uint4(0, 0, 0, 0);
+        } else if (MODE == 1) {
+            union { uint4 q; T e[PER]; } v;
+#pragma unroll
+            for (int i = 0; i < PER; ++i) {
+                bool inside;
+                const int64_t src = source(p0 + i, inside);
+                v.e[i] = inside ? __ldg(X + src) : T(0);
+            }
+            *reinterpret_cast<uint4*>(dst) = v.q;
         } else {
-            out[dst] = inside ? X[src] : T(0);
+            bool inside;
+            const int64_t src = source(p0, inside);
+            *dst = inside ? __ldg(X + src) : T(0);
         }
     }
 }
@@ -45,16 +63,19 @@ im2row_kernel(const ConvIndex cv, int64_t pixels, const T* __restrict__ X, T* __
 template <typename T>
 static cudaError_t launch_im2row_t(const ConvIndex& cv, int64_t pixels, const void* X, void* out, int64_t ld, cudaStream_t s) {
     const int es = (int)sizeof(T);
-    const bool chunk = (cv.c_in * es) % 16 == 0 && (ld * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0 &&
-                       (reinterpret_cast<uintptr_t>(out) & 15) == 0;
-    const int64_t per = chunk ? 16 / es : 1;
-    const int64_t total = pixels * cv.kh * cv.kw * (cv.c_in / per);
+    const int64_t k = (int64_t)cv.kh * cv.kw * cv.c_in;
+    const bool out_ok = (ld * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(out) & 15) == 0;
+    const bool in_ok = (cv.c_in * es) % 16 == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0;
+    const int mode = out_ok ? (in_ok ? 0 : 1) : 2;
+    const int64_t per = mode == 2 ? 1 : 16 / es;
+    const int64_t total = pixels * (mode == 1 ? ld / per : k / per);
     if (total == 0) return cudaSuccess;
     int64_t blocks = cdiv(total, 256);
     const int64_t cap = (int64_t)sm_count() * 32;
     if (blocks > cap) blocks = cap;
-    if (chunk) im2row_kernel<T, true><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (const T*)X, (T*)out, ld);
-    else im2row_kernel<T, false><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (const T*)X, (T*)out, ld);
+    if (mode == 0) im2row_kernel<T, 0><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (int)k, (const T*)X, (T*)out, ld);
+    else if (mode == 1) im2row_kernel<T, 1><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (int)k, (const T*)X, (T*)out, ld);
+    else im2row_kernel<T, 2><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (int)k, (const T*)X, (T*)out, ld);
     return cudaGetLastError();
 }
 
@@ -77,7 +98,7 @@ static int conv_setup(int dtype, const conv_shape_t* sh, const void* X, ConvInde
     const int64_t wo = (sh->w + 2 * (int64_t)sh->pad_w - sh->kw) / sh->stride_w + 1;
     // 32-bit pixel arithmetic inside the kernels
     if (sh->h > 0x3FFFFFFF || sh->w > 0x3FFFFFFF || ho * wo > 0x7FFFFFFF || sh->batch > 0x7FFFFFFF ||
-        (int64_t)sh->kh * sh->kw > 0x7FFF)
+        (int64_t)sh->kh * sh->kw > 0x7FFF || (int64_t)sh->kh * sh->kw * sh->c_in > 0x7FFFFFFF)
         return -2;
     cv->X = X;
     cv->h = sh->h; cv->w = sh->w; cv->c_in = sh->c_in;
@@ -136,7 +157,9 @@ size_t conv2d_workspace_bytes(int dtype, const conv_shape_t* shape) {
     if (lowering_is_identity(cv)) return need;
     // judged for 16-byte aligned tensors and a filter matrix TMA can address
     const bool fused = fused_possible(dtype, cv, shape->batch, reinterpret_cast<const void*>(16), 8);
-    if (!fused || g_force_lowering == CONV_LOWERING_EXPLICIT) need += (size_t)rup(rup(k, 8) * n * elem_size(dtype), 256);
+    const bool scalar_map = dtype == GEMM_F32 && cv.c_in % 4 != 0;       // served faster by writing L first
+    if (!fused || scalar_map || g_force_lowering == CONV_LOWERING_EXPLICIT)
+        need += (size_t)rup(rup(k, 8) * n * elem_size(dtype), 256);
     return need;
 }
 
@@ -167,7 +190,17 @@ int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void*
 
     GemmArgs a{dtype, false, false, m, n, k, alpha, beta, W, nullptr, static_cast<float*>(Y), ldw, k, ldy, s, nullptr};
     const bool can_fuse = fused_possible(dtype, cv, shape->batch, W, ldw);
-    const bool fuse = can_fuse && g_force_lowering != CONV_LOWERING_EXPLICIT;
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    if (!registered_workspace(&ws, &ws_bytes)) return GEMM_ERR_LAUNCH;
+    const int64_t ld = rup(k, 8);
+    const size_t l_bytes = (size_t)rup(ld * n * es, 256);
+    const bool room = ws != nullptr && ws_bytes >= l_bytes;
+    // fp32 layers whose channel count rules out 128-bit loads (the 3-channel first layers) run the index map with
+    // scalar loads at about a third of the kernel's speed: writing L first is faster when there is room for it
+    const bool scalar_map = dtype == GEMM_F32 && (cv.c_in % 4 != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0);
+    bool fuse = can_fuse && g_force_lowering != CONV_LOWERING_EXPLICIT;
+    if (fuse && scalar_map && room && g_force_lowering != CONV_LOWERING_FUSED) fuse = false;
     if (fuse) {
         a.conv = &cv;
         const int rc = dispatch_gemm(a, 0);
@@ -177,12 +210,13 @@ int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void*
 
     // explicit route: L goes to the head of the workspace (leading dimension a multiple of 8 elements so that TMA
     // can address it), the GEMM uses what is left
-    void* ws = nullptr;
-    size_t ws_bytes = 0;
-    if (!registered_workspace(&ws, &ws_bytes)) return GEMM_ERR_LAUNCH;
-    const int64_t ld = rup(k, 8);
-    const size_t l_bytes = (size_t)rup(ld * n * es, 256);
-    if (ws == nullptr || ws_bytes < l_bytes) return GEMM_ERR_WORKSPACE;
+    if (!room) {
+        if (!can_fuse) return GEMM_ERR_WORKSPACE;
+        a.conv = &cv;                               // forced explicit but no room: the fused route still works
+        const int rc = dispatch_gemm(a, 0);
+        if (rc == GEMM_OK) note_lowering(CONV_LOWERING_FUSED);
+        return rc;
+    }
     const cudaError_t e = launch_im2row(dtype, cv, n, X, ws, ld, s);
     if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
     a.B = ws;

@@ -137,16 +137,41 @@ struct ConvLoader {
         return px;
     }
 
-    __device__ static __forceinline__ void load(float (&r)[ELEMS], const ConvIndex& cv, const Pixel (&px)[VEC == 4 ? NV : 1],
-                                                int64_t j0, int64_t k0, int64_t n, int64_t kmax, int t) {
-        const float* __restrict__ X = static_cast<const float*>(cv.X);
+    // Position of the thread's k index inside the filter: tap (fr, fs) and channel c.  All loads of a thread share
+    // it (their kk is the same), and it moves forward by one k slice per load() call, so it is kept as running
+    // state instead of being divided out of p every time.
+    struct Tap {
+        int fr, fs, c;
+        int64_t p;
+    };
+    __device__ static __forceinline__ Tap first_tap(const ConvIndex& cv, int64_t kbeg, int t) {
         int x, kk;
-        L::coord(t, 0, x, kk);                    // kk is the same for every load of a thread
-        const int64_t p = k0 + kk;
-        const int tap = (int)(p / cv.c_in), c = (int)(p - (int64_t)tap * cv.c_in);
-        const int fr = tap / cv.kw, fs = tap - fr * cv.kw;
-        const bool k_ok = p < kmax;               // VEC = 4: k is a multiple of 4 here, so the four elements share it
-        const int64_t tap_off = ((int64_t)fr * cv.w + fs) * cv.c_in + c;
+        L::coord(t, 0, x, kk);
+        Tap tp;
+        tp.p = kbeg + kk;
+        const uint32_t p32 = (uint32_t)tp.p, cin = (uint32_t)cv.c_in;       // k = kh*kw*C_in fits 31 bits (checked by the host)
+        const uint32_t tap = p32 / cin;
+        tp.c = (int)(p32 - tap * cin);
+        tp.fr = (int)(tap / (uint32_t)cv.kw);
+        tp.fs = (int)(tap - (uint32_t)tp.fr * (uint32_t)cv.kw);
+        return tp;
+    }
+    __device__ static __forceinline__ void advance(const ConvIndex& cv, Tap& tp) {
+        tp.p += BK;
+        tp.c += BK;
+        const int cin = (int)cv.c_in;
+        while (tp.c >= cin) {
+            tp.c -= cin;
+            if (++tp.fs == cv.kw) { tp.fs = 0; ++tp.fr; }
+        }
+    }
+
+    __device__ static __forceinline__ void load(float (&r)[ELEMS], const ConvIndex& cv, const Pixel (&px)[VEC == 4 ? NV : 1],
+                                                Tap& tp, int64_t j0, int64_t n, int64_t kmax, int t) {
+        const float* __restrict__ X = static_cast<const float*>(cv.X);
+        const bool k_ok = tp.p < kmax;            // VEC = 4: k is a multiple of 4 here, so the four elements share it
+        const int64_t tap_off = ((int64_t)tp.fr * cv.w + tp.fs) * cv.c_in + tp.c;
+        const int fr = tp.fr, fs = tp.fs;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             if (VEC == 4) {
@@ -156,12 +181,14 @@ struct ConvLoader {
                     q = __ldg(reinterpret_cast<const float4*>(X + px[v].off + tap_off));
                 r[v * 4 + 0] = q.x; r[v * 4 + 1] = q.y; r[v * 4 + 2] = q.z; r[v * 4 + 3] = q.w;
             } else {
+                int x, kk;
                 L::coord(t, v, x, kk);
                 const Pixel one = pixel(cv, j0 + x, n);
                 const int hi = one.h0 + fr, wi = one.w0 + fs;
                 r[v] = (k_ok && (unsigned)hi < (unsigned)cv.h && (unsigned)wi < (unsigned)cv.w) ? __ldg(X + one.off + tap_off) : 0.0f;
             }
         }
+        advance(cv, tp);
     }
 };
 
@@ -314,7 +341,10 @@ simt_fast_body(int64_t m, int64_t n, int64_t k, float alpha, const float* __rest
         }
     }
 
-    auto gload = [&](int64_t kt) {
+    typename LC::Tap tap{0, 0, 0, 0};
+    if (CONV) tap = LC::first_tap(cv, kbeg, t);
+
+    auto gload = [&](int64_t kt) {      // called for kt = 0, 1, 2, ... in order
         if (kt < fast_tiles) {
             LA::load_fast(ra, pa, va);
             pa += step_a;
@@ -327,7 +357,7 @@ simt_fast_body(int64_t m, int64_t n, int64_t k, float alpha, const float* __rest
             LA::template load<true>(ra, A, lda, i0, k0, m, kend, t);
             if (!CONV) LB::template load<true>(rb, B, ldb, j0, k0, n, kend, t);
         }
-        if (CONV) LC::load(rb, cv, px, j0, kbeg + kt * BK, n, kend, t);
+        if (CONV) LC::load(rb, cv, px, tap, j0, n, kend, t);
     };
 
     asm volatile("griddepcontrol.wait;" ::: "memory");     // the previous kernel's results are visible from here on

@@ -88,7 +88,10 @@ def expected_route(p, W):
         return g.CONV_LOWERING_IDENTITY
     # 16-bit layers are fused when TMA can fetch both operands: whole 64-channel chunks, and a filter matrix whose
     # columns start on 16-byte boundaries
-    if p.dtype == DTYPE_F32 or (p.c_in % 64 == 0 and W.ld % 8 == 0):
+    if p.dtype == DTYPE_F32:
+        # with room in the workspace, layers that would need scalar loads through the index map are lowered first
+        return g.CONV_LOWERING_FUSED if p.c_in % 4 == 0 else g.CONV_LOWERING_EXPLICIT
+    if p.c_in % 64 == 0 and W.ld % 8 == 0:
         return g.CONV_LOWERING_FUSED
     return g.CONV_LOWERING_EXPLICIT
 
@@ -154,6 +157,7 @@ def test_every_tensor_tile_with_the_im2col_producer(dtype):
 def test_every_fp32_tile_with_the_index_map():
     ensure_workspace(256 << 20)
     for gm in ((2, 14, 15, 16, 200, 3, 3, 1, 1), (2, 14, 15, 6, 200, 3, 3, 2, 1)):      # 128-bit and scalar loads
+        g.conv2d_force_lowering(g.CONV_LOWERING_FUSED)      # the scalar index map is otherwise taken only without a workspace
         for tile in ((128, 128), (128, 64), (64, 128), (64, 64)):
             for split in (1, 2):
                 g.gemm_force_tile(tile[0], tile[1], split)
@@ -163,6 +167,18 @@ def test_every_fp32_tile_with_the_index_map():
                 assert cfg["lowering"] == g.CONV_LOWERING_FUSED and cfg["kernel"] == g.GEMM_KERNEL_SIMT_FAST
                 assert (cfg["tile_m"], cfg["tile_n"]) == tile and cfg["vector_b"] == (4 if gm[3] % 4 == 0 else 1), cfg
                 check(p, X, W, Y0, Y, integer=True)
+
+
+def test_fp32_layer_with_three_channels_stays_fused_without_workspace():
+    drop_workspace()
+    p = make(SMALL[0], DTYPE_F32, alpha=1.5, beta=0.5)
+    X, W, Y0 = p.operands()
+    dX, dW, dY = to_device(X), to_device(W), to_device(Y0)
+    rc = g.conv2d_im2row(p.dtype, shape_of(p), p.alpha, dX.data_ptr(), dW.data_ptr(), W.ld, p.beta, dY.data_ptr(), Y0.ld, 0)
+    assert rc == 0 and g.gemm_poll_status() == 0
+    assert g.gemm_last_config()["lowering"] == g.CONV_LOWERING_FUSED and g.gemm_last_config()["vector_b"] == 1
+    from workloads import Matrix
+    check(p, X, W, Y0, Matrix(dY.cpu().numpy(), Y0.rows, Y0.cols, Y0.ld, DTYPE_F32))
 
 
 def test_sixteen_bit_layer_without_workspace_reports_it():

@@ -45,7 +45,9 @@ def test_convolution_argument_checks_run_without_a_device():
     # a layer whose lowered matrix must be written asks for room for it: k = 27 padded to 32 rows, 2 bytes each
     s = g.conv_shape(4, 32, 32, 3, 64, 3, 3, 1, 1, 1, 1)
     assert g.conv2d_workspace_bytes(2, s) >= 32 * 4 * 32 * 32 * 2
-    assert g.conv2d_workspace_bytes(0, s) == g.gemm_workspace_bytes(0, "N", "N", 64, 4 * 32 * 32, 27)   # fp32: fused
+    assert g.conv2d_workspace_bytes(0, s) >= 32 * 4 * 32 * 32 * 4         # fp32 with 3 channels: lowered first, too
+    s = g.conv_shape(4, 32, 32, 8, 64, 3, 3, 1, 1, 1, 1)
+    assert g.conv2d_workspace_bytes(0, s) == g.gemm_workspace_bytes(0, "N", "N", 64, 4 * 32 * 32, 72)   # fp32, C_in % 4 == 0: fused
 
 
 def test_workspace_request_for_split_k_shapes():
