@@ -63,11 +63,11 @@ CONV_WORKLOADS = {
 # kernel and problem, with the hash of the kernel's source file at capture time: a changed kernel reports null.
 TRAFFIC = {
     ("simt_fast_kernel", "8192x8192x8192", "f32"): {
-        "bytes": 3079800320 + 260572416, "source": "paper_2310_17408_b200/csrc/simt_fast.cu",
-        "sha256": "2649140bc88e0e9bef46889623085491c29671487eafd8f8efc6cd7dd809cc4d"},
-    ("tc_gemm_kernel", "8192x8192x8192", "bf16"): {
-        "bytes": 1011795000 + 254793984, "source": "paper_2310_17408_b200/csrc/tc_gemm.cu",
-        "sha256": "5e8699c24d9a9cc17e883bea3ff4edec258652ce4e58e9e35f5d899dcb167aa6"},
+        "bytes": 3461221120 + 266224128, "source": "paper_2310_17408_b200/csrc/simt_fast.cu",
+        "sha256": "7346a4ec45286843a6c0f99c4ae3de365cd5dfb708788e0ea79050818e694869"},
+    ("tc_gemm_pair_kernel", "8192x8192x8192", "bf16"): {
+        "bytes": 1106418944 + 261512192, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
+        "sha256": "7326017d17f3d14fc2bb12bf08772fed1165ae66a2d8fefe6f8cb4e05cadac8a"},
 }
 
 
@@ -630,15 +630,24 @@ def main():
     ap.add_argument("--dtype", default="f32", choices=["f32", "f16", "bf16"], help="operand type for --shape")
     ap.add_argument("--alpha", type=float, default=1.0, help="alpha for --shape")
     ap.add_argument("--beta", type=float, default=0.0, help="beta for --shape")
+    ap.add_argument("--only", default=None, help="comma-separated problem names: keep only these members of the workload")
     ap.add_argument("--table", default=None, help="also write the JSON (indented, with per-shape rows) to this file")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-budget", type=float, default=30.0)
     args = ap.parse_args()
+    def keep(items):
+        if not args.only:
+            return items
+        names = set(args.only.split(","))
+        kept = [p for p in items if p.name in names]
+        if not kept:
+            raise SystemExit(f"--only {args.only}: no such problem in {args.workload} ({', '.join(p.name for p in items)})")
+        return kept
     if args.workload in CONV_WORKLOADS:
-        return run_conv_layers(args, CONV_WORKLOADS[args.workload](), args.workload)
-    problems = WORKLOADS[args.workload]()
+        return run_conv_layers(args, keep(CONV_WORKLOADS[args.workload]()), args.workload)
+    problems = keep(WORKLOADS[args.workload]())
     if args.shape:
         from workloads import Problem
         m, n, k = (int(t) for t in args.shape.split(","))
