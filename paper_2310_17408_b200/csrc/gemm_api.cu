@@ -227,6 +227,31 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
     }
     if (g_force_tile_m == 256) p->pair = bn == 256;
     if (g_force_tile_m == 128) p->pair = false;
+    // Tail split of the pair kernel: with more tiles than pairs and a last round that is at most half full, the
+    // tiles of that round are cut into floor(pairs / r) k ranges (at least 8 k blocks each)
+    p->tail_splits = 1;
+    p->tail_first = 0x7FFFFFFF;
+    size_t tail_need = 0;
+    if (p->pair && want == 1 && g_force_split == 0 && !g_no_tail_split) {
+        const int64_t tiles = ceil_div(a.m, 256) * ceil_div(a.n, 256), pairs = sms / 2;
+        const int64_t r = tiles % pairs;
+        if (tiles > pairs && r > 0 && 2 * r <= pairs) {
+            int64_t s = pairs / r;
+            if (s > a.k / 512) s = a.k / 512;
+            if (s > 8) s = 8;
+            if (s >= 2) {
+                const int64_t chunk = round_up(ceil_div(a.k, s), 64);
+                const int64_t splits = ceil_div(a.k, chunk);
+                const size_t need = (size_t)(r * splits) * 256 * 256 * sizeof(float);
+                if (splits >= 2 && ws_repack + need <= ws_avail) {
+                    p->tail_first = (int)(tiles - r);
+                    p->tail_splits = (int)splits;
+                    p->tail_chunk = chunk;
+                    tail_need = need;
+                }
+            }
+        }
+    }
     p->ks = make_split(a.k, want, 64);
     p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
     if (ws_repack + p->ws_partials > ws_avail) {
@@ -234,6 +259,8 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         p->ks = make_split(a.k, 1, 64);
         p->ws_partials = 0;
     }
+    if (p->tail_splits > 1 && p->ks.splits == 1) p->ws_partials = tail_need;
+    else { p->tail_splits = 1; p->tail_first = 0x7FFFFFFF; }
     p->ws_total = ws_repack + p->ws_partials;
 }
 
@@ -353,11 +380,19 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
     }
     float* partials = p.ks.splits > 1 ? reinterpret_cast<float*>(wsp) : nullptr;
     if (p.kernel == GEMM_KERNEL_TENSOR) {
-        e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg) : launch_tensor(a, p.tile, p.ks, partials, &cfg);
+        if (p.pair && p.tail_splits > 1) {
+            TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
+            e = launch_tensor_pair(a, p.ks, nullptr, &cfg, tail);
+            if (e == cudaSuccess) e = launch_tail_reduce(a, 256, 256, PAIR_GROUP, tail);
+            cfg.launches++;
+            cfg.tail_split = p.tail_splits;
+        } else {
+            e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg) : launch_tensor(a, p.tile, p.ks, partials, &cfg);
+        }
     } else if (p.tail_splits > 1) {
         TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
         e = launch_simt_fast(a, p.tile, p.ks, nullptr, &cfg, tail);
-        if (e == cudaSuccess) e = launch_tail_reduce(a, p.tile, tail);
+        if (e == cudaSuccess) e = launch_tail_reduce(a, kSimtTileM[p.tile], kSimtTileN[p.tile], SIMT_GROUP, tail);
         cfg.launches++;
         cfg.tail_split = p.tail_splits;
     } else {

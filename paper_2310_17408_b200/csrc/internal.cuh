@@ -41,8 +41,8 @@ struct KSplit {
 // device status word layout: bits 31..24 = 0xE5 marker, 23..16 = role, 15..8 = barrier id, 7..0 = stage
 constexpr uint32_t STATUS_MARK = 0xE5000000u;
 
-// Tail split of the fp32 SIMT path: tiles first .. are cut into `splits` k ranges of `chunk` each
-// (first = INT_MAX: off).  Item i >= first writes its raw block to partials + (i - first) * tile_m * tile_n.
+// Tail split (fp32 SIMT kernel and the CTA-pair tensor kernel): tiles first .. are cut into `splits` k ranges of
+// `chunk` each (first = INT_MAX: off).  Item i >= first writes its raw block to partials + (i - first) * tile_m * tile_n.
 struct TailSplit {
     int first;
     int splits;
@@ -50,15 +50,15 @@ struct TailSplit {
     float* partials;
 };
 
-// Tile order of the fp32 SIMT path: groups of SIMT_GROUP tile rows, all tile columns inside a group, rows fastest,
+// Tile order shared by the kernels: groups of `group` tile rows, all tile columns inside a group, rows fastest,
 // so that the CTAs resident at one time share their A and B panels in L2.
 constexpr int SIMT_GROUP = 16;
-__host__ __device__ inline void decode_tile(int tile, int tiles_m, int tiles_n, int* tm, int* tn) {
-    const int per_group = SIMT_GROUP * tiles_n;
+__host__ __device__ inline void decode_tile(int tile, int tiles_m, int tiles_n, int* tm, int* tn, int group = SIMT_GROUP) {
+    const int per_group = group * tiles_n;
     const int g = tile / per_group;
-    const int rest = tiles_m - g * SIMT_GROUP;
-    const int gsz = rest < SIMT_GROUP ? rest : SIMT_GROUP;
-    *tm = g * SIMT_GROUP + (tile % per_group) % gsz;
+    const int rest = tiles_m - g * group;
+    const int gsz = rest < group ? rest : group;
+    *tm = g * group + (tile % per_group) % gsz;
     *tn = (tile % per_group) / gsz;
 }
 
@@ -75,8 +75,9 @@ cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg);
 bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb);
 cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg,
                              TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
-// finishes the tail tiles: C <- alpha * sum_z slot[(t - first) * splits + z] + beta*C for tiles t >= first
-cudaError_t launch_tail_reduce(const GemmArgs& a, int tile, TailSplit tail);
+// finishes the tail tiles (bm x bn, tile order with groups of `group` rows):
+// C <- alpha * sum_z slot[(t - first) * splits + z] + beta*C for tiles t >= first
+cudaError_t launch_tail_reduce(const GemmArgs& a, int bm, int bn, int group, TailSplit tail);
 
 // C <- alpha * sum_s partials[s] + beta*C, summed in increasing s (deterministic)
 cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* partials);
@@ -85,7 +86,9 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 bool tensor_eligible(const GemmArgs& a);
 cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg);
 // the same on CTA pairs (tcgen05 cta_group::2): 256 x 256 tiles, two SMs per tile
-cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg);
+cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
+                               TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
+constexpr int PAIR_GROUP = 8;      // tile rows (of 256) per group of the pair kernel's tile order
 
 // copy op-independent stored matrix (rows x cols, ld) of 16-bit elements into an aligned layout (ld_out)
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,

@@ -534,51 +534,4 @@ cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* part
     return launch_vec<true, false>(a, va, vb, tile, ks, partials, cfg, tail);
 }
 
-// ---------------------------------------------------------------- tail reduction
-
-// One block row per tail tile (blockIdx.x) and a quarter of its entries per blockIdx.y: sums the tile's k ranges in
-// increasing order (deterministic) and applies alpha / beta once.
-__global__ void __launch_bounds__(256)
-tail_reduce_kernel(int64_t m, int64_t n, float alpha, float beta, float* __restrict__ C, int64_t ldc, int tiles_m,
-                   int tiles_n, int bm, int bn, TailSplit tail) {
-    const int tl = blockIdx.x;
-    int tm, tn;
-    decode_tile(tail.first + tl, tiles_m, tiles_n, &tm, &tn);
-    const int64_t i0 = (int64_t)tm * bm, j0 = (int64_t)tn * bn;
-    const int tile_elems = bm * bn;
-    const float* slot = tail.partials + (int64_t)tl * tail.splits * tile_elems;
-    const int vecs = tile_elems / 4, per_y = (vecs + gridDim.y - 1) / gridDim.y;
-    const int v_end = min(vecs, (int)(blockIdx.y + 1) * per_y);
-    for (int v = blockIdx.y * per_y + threadIdx.x; v < v_end; v += blockDim.x) {
-        const int e = v * 4, r = e % bm, c = e / bm;
-        float4 s4 = *reinterpret_cast<const float4*>(slot + e);
-        for (int z = 1; z < tail.splits; ++z) {
-            const float4 q = *reinterpret_cast<const float4*>(slot + (int64_t)z * tile_elems + e);
-            s4.x += q.x; s4.y += q.y; s4.z += q.z; s4.w += q.w;
-        }
-        const int64_t gi = i0 + r, gj = j0 + c;
-        if (gj >= n) continue;
-        const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
-        float* cp = C + gi + gj * ldc;
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            if (gi + q < m) {
-                float o = alpha * sv[q];
-                if (beta != 0.0f) o = fmaf(beta, cp[q], o);
-                cp[q] = o;
-            }
-    }
-}
-
-cudaError_t launch_tail_reduce(const GemmArgs& a, int tile, TailSplit tail) {
-    static const int bm_of[4] = {128, 128, 64, 64}, bn_of[4] = {128, 64, 128, 64};
-    const int bm = bm_of[tile], bn = bn_of[tile];
-    const int64_t tiles_m = (a.m + bm - 1) / bm, tiles_n = (a.n + bn - 1) / bn;
-    const int64_t tail_tiles = tiles_m * tiles_n - tail.first;
-    if (tail_tiles <= 0) return cudaSuccess;
-    tail_reduce_kernel<<<dim3((unsigned)tail_tiles, 4), 256, 0, a.stream>>>(a.m, a.n, a.alpha, a.beta, a.C, a.ldc,
-                                                                           (int)tiles_m, (int)tiles_n, bm, bn, tail);
-    return cudaGetLastError();
-}
-
 }  // namespace b200gemm

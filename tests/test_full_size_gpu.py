@@ -63,6 +63,24 @@ def test_config5_half_squares_4096_8192(dtype):
         assert (cfg["tile_m"], cfg["tile_n"]) == (256, 256)      # large squares run on CTA pairs
 
 
+def test_pair_kernel_tail_split_of_the_last_round():
+    # 164 tiles of 256 x 256 on 74 pairs: the 16 tiles of the third round are cut into k ranges, finished by the
+    # tile-local reduction; 4096^3 (256 tiles, last round 34) takes the same path by the selector's own choice
+    from workloads import Problem
+    g.gemm_force_tile(256, 256, 0)
+    try:
+        for dtype, kind in ((DTYPE_BF16, "normal"), (DTYPE_F16, "int")):
+            p = Problem("tail", dtype, 1024 - 3, 10496 - 5, 1024 + 64, 1.5, 0.5, kindA=kind, kindB=kind,
+                        kindC="int" if kind == "int" else "uniform", seed=21)
+            cfg, _ = run_and_check(p, seed=3)
+            assert (cfg["tile_m"], cfg["tile_n"], cfg["split_k"]) == (256, 256, 1), cfg
+            assert cfg["tail_split"] >= 2 and cfg["launches"] >= 2, (cfg["tail_split"], cfg["launches"])     # + repacking passes
+    finally:
+        g.gemm_force_tile(0, 0, 0)
+    cfg, _ = run_and_check(config_problems(5, dtype=DTYPE_BF16)[0], seed=4)
+    assert cfg["tail_split"] == 2, cfg
+
+
 def test_config5_f16_square_16384():
     p = config_problems(5, dtype=DTYPE_F16)[2]
     cfg, _ = run_and_check(p)
