@@ -44,12 +44,18 @@ im2row_kernel(const ConvIndex cv, int64_t pixels, int k, const T* __restrict__ X
             const int64_t src = source(p0, inside);
             *reinterpret_cast<uint4*>(dst) = inside ? __ldg(reinterpret_cast<const uint4*>(X + src)) : make_uint4(0, 0, 0, 0);
         } else if (MODE == 1) {
+            // one division for the chunk's first row, then the (tap, channel) position walks forward element by element
             union { uint4 q; T e[PER]; } v;
+            uint32_t tap = p0 / cin, c = p0 - tap * cin;
+            int fr = (int)(tap / kw), fs = (int)(tap - (uint32_t)fr * kw);
 #pragma unroll
             for (int i = 0; i < PER; ++i) {
-                bool inside;
-                const int64_t src = source(p0 + i, inside);
-                v.e[i] = inside ? __ldg(X + src) : T(0);
+                const bool inside = p0 + i < (uint32_t)k && (unsigned)(h0 + fr) < (unsigned)cv.h && (unsigned)(w0 + fs) < (unsigned)cv.w;
+                v.e[i] = inside ? __ldg(X + base + ((int64_t)fr * cv.w + fs) * cv.c_in + c) : T(0);
+                if (++c == cin) {
+                    c = 0;
+                    if (++fs == (int)kw) { fs = 0; ++fr; }
+                }
             }
             *reinterpret_cast<uint4*>(dst) = v.q;
         } else {

@@ -84,7 +84,8 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 
 // tcgen05 tensor-core kernel (fp16 / bf16).  tile_n in {64, 128, 256}; tile_m is 128.
 bool tensor_eligible(const GemmArgs& a);
-cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg);
+cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg,
+                          TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
 // the same on CTA pairs (tcgen05 cta_group::2): 256 x 256 tiles, two SMs per tile
 cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
                                TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
