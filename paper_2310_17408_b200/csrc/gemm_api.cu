@@ -182,18 +182,7 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
     auto cost_us = [&](int bn, int splits) {
         const double tiles = (double)ceil_div(a.m, 128) * (double)ceil_div(a.n, bn);
         const double items = tiles * splits;
-        double rounds = (double)ceil_div((int64_t)items, sms);
-        double tail_us = 0.0;
-        if (splits == 1 && g_force_split == 0 && !g_no_tail_split) {      // the tail split below shortens a last round that is at most half full
-            const int64_t r = (int64_t)items % sms;
-            int64_t s = r > 0 ? sms / r : 1;
-            if (s > a.k / 512) s = a.k / 512;
-            if (s > 8) s = 8;
-            if (items > sms && r > 0 && 2 * r <= sms && s >= 2) {
-                rounds = rounds - 1.0 + 1.0 / (double)s;
-                tail_us = 4.0 + (double)(r * (s + 1)) * 128.0 * bn * 4.0 / 5e6;      // its reduction pass
-            }
-        }
+        const double rounds = (double)ceil_div((int64_t)items, sms);
         const double kb = (double)ceil_div(ceil_div(a.k, splits), 64);
         const double stage = (128.0 + bn) * 128.0;
         const double t_kb = std::max(0.27 * bn / 256.0, stage / 146e3);
@@ -201,7 +190,7 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         const double fill_us = items * kb * stage / 1e7;
         const double mn = (double)a.m * (double)a.n;
         const double hbm_us = (2.0 * ((double)a.m * a.k + (double)a.k * a.n) + 4.0 * mn * splits) / 6.5e6;
-        double t = 7.0 + tail_us + std::max(main_us, std::max(fill_us, hbm_us));
+        double t = 7.0 + std::max(main_us, std::max(fill_us, hbm_us));
         if (splits > 1) t += 4.0 + (splits + 1) * mn * 4.0 / 5e6;
         return t;
     };
@@ -229,41 +218,15 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
     // CTA pairs (256 x 256 tiles) fill a third less shared memory per flop, which is what limits the 128 x 256
     // kernel: measured 9 % faster main loops (4096^3, 8192^3, the large VGG16 shapes), but ~2.5 us more fixed
     // cost per launch (cluster set-up, cross-CTA barriers).  Taken when every pair has work and the main loops
-    // of the 128 x 256 kernel would run for 30 us or more.
+    // of the 128 x 256 kernel would run for 10 us or more (measured: ahead from ~14 us on, behind at ~4 us).
     {
         const int64_t pair_tiles = ceil_div(a.m, 256) * ceil_div(a.n, 256);
         const double rounds = (double)ceil_div(ceil_div(a.m, 128) * ceil_div(a.n, 256), sms);
         const double main_us = rounds * (double)ceil_div(a.k, 64) * 0.27;
-        p->pair = bn == 256 && want == 1 && a.m > 128 && pair_tiles >= sms / 2 && main_us >= 30.0;
+        p->pair = bn == 256 && want == 1 && a.m > 128 && pair_tiles >= sms / 2 && main_us >= 10.0;
     }
     if (g_force_tile_m == 256) p->pair = bn == 256;
     if (g_force_tile_m == 128) p->pair = false;
-    // Tail split of the tensor kernels: with more tiles than CTAs (or CTA pairs) and a last round that is at most
-    // half full, the tiles of that round are cut into floor(slots / r) k ranges of at least 8 k blocks each
-    p->tail_splits = 1;
-    p->tail_first = 0x7FFFFFFF;
-    size_t tail_need = 0;
-    if (want == 1 && g_force_split == 0 && !g_no_tail_split) {
-        const int64_t tm_ = p->pair ? 256 : 128;
-        const int64_t tiles = ceil_div(a.m, tm_) * ceil_div(a.n, bn), slots = p->pair ? sms / 2 : sms;
-        const int64_t r = tiles % slots;
-        if (tiles > slots && r > 0 && 2 * r <= slots) {
-            int64_t s = slots / r;
-            if (s > a.k / 512) s = a.k / 512;
-            if (s > 8) s = 8;
-            if (s >= 2) {
-                const int64_t chunk = round_up(ceil_div(a.k, s), 64);
-                const int64_t splits = ceil_div(a.k, chunk);
-                const size_t need = (size_t)(r * splits) * tm_ * bn * sizeof(float);
-                if (splits >= 2 && ws_repack + need <= ws_avail) {
-                    p->tail_first = (int)(tiles - r);
-                    p->tail_splits = (int)splits;
-                    p->tail_chunk = chunk;
-                    tail_need = need;
-                }
-            }
-        }
-    }
     p->ks = make_split(a.k, want, 64);
     p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
     if (ws_repack + p->ws_partials > ws_avail) {
@@ -271,8 +234,8 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         p->ks = make_split(a.k, 1, 64);
         p->ws_partials = 0;
     }
-    if (p->tail_splits > 1 && p->ks.splits == 1) p->ws_partials = tail_need;
-    else { p->tail_splits = 1; p->tail_first = 0x7FFFFFFF; }
+    p->tail_splits = 1;
+    p->tail_first = 0x7FFFFFFF;
     p->ws_total = ws_repack + p->ws_partials;
 }
 
@@ -392,16 +355,7 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
     }
     float* partials = p.ks.splits > 1 ? reinterpret_cast<float*>(wsp) : nullptr;
     if (p.kernel == GEMM_KERNEL_TENSOR) {
-        if (p.tail_splits > 1) {
-            TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
-            e = p.pair ? launch_tensor_pair(a, p.ks, nullptr, &cfg, tail) : launch_tensor(a, p.tile, p.ks, nullptr, &cfg, tail);
-            if (e == cudaSuccess)
-                e = p.pair ? launch_tail_reduce(a, 256, 256, PAIR_GROUP, tail) : launch_tail_reduce(a, 128, p.tile, SIMT_GROUP, tail);
-            cfg.launches++;
-            cfg.tail_split = p.tail_splits;
-        } else {
-            e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg) : launch_tensor(a, p.tile, p.ks, partials, &cfg);
-        }
+        e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg) : launch_tensor(a, p.tile, p.ks, partials, &cfg);
     } else if (p.tail_splits > 1) {
         TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
         e = launch_simt_fast(a, p.tile, p.ks, nullptr, &cfg, tail);

@@ -41,8 +41,8 @@ struct KSplit {
 // device status word layout: bits 31..24 = 0xE5 marker, 23..16 = role, 15..8 = barrier id, 7..0 = stage
 constexpr uint32_t STATUS_MARK = 0xE5000000u;
 
-// Tail split (fp32 SIMT kernel and the CTA-pair tensor kernel): tiles first .. are cut into `splits` k ranges of
-// `chunk` each (first = INT_MAX: off).  Item i >= first writes its raw block to partials + (i - first) * tile_m * tile_n.
+// Tail split of the fp32 SIMT path: tiles first .. are cut into `splits` k ranges of `chunk` each
+// (first = INT_MAX: off).  Item i >= first writes its raw block to partials + (i - first) * tile_m * tile_n.
 struct TailSplit {
     int first;
     int splits;
@@ -84,12 +84,9 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 
 // tcgen05 tensor-core kernel (fp16 / bf16).  tile_n in {64, 128, 256}; tile_m is 128.
 bool tensor_eligible(const GemmArgs& a);
-cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg,
-                          TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
+cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg);
 // the same on CTA pairs (tcgen05 cta_group::2): 256 x 256 tiles, two SMs per tile
-cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
-                               TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
-constexpr int PAIR_GROUP = 8;      // tile rows (of 256) per group of the pair kernel's tile order
+cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg);
 
 // copy op-independent stored matrix (rows x cols, ld) of 16-bit elements into an aligned layout (ld_out)
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,

@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
-               uint32_t idesc, uint32_t* status, const ConvTma conv, const TailSplit tail) {
+               uint32_t idesc, uint32_t* status, const ConvTma conv) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -81,29 +81,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // previous kernel in the stream; nothing below touches global memory before that kernel has completed.
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // Work items.  Without a tail split: tiles x k partitions (split-k).  With one (splits == 1): items below
-    // tail.first are whole tiles; the tiles of the last, partly filled round come after them, cut into tail.splits
-    // k ranges each (raw partial sums into tile-local slots, finished by a small reduction pass).
-    const int64_t tiles = (int64_t)tiles_m * tiles_n;
-    const int64_t items = tail.first < tiles ? tail.first + (tiles - tail.first) * tail.splits : tiles * splits;
-    // slot >= 0: the item is a k range of a tail tile and writes slot `slot` of tail.partials
-    auto decode = [&](int64_t item, int& tm, int& tn, int& sp, int64_t& slot) {
-        int tile;
-        if (item >= tail.first) {
-            slot = item - tail.first;
-            tile = tail.first + (int)(slot / tail.splits);
-            sp = (int)(slot % tail.splits);
-        } else {
-            slot = -1;
-            sp = (int)(item / tiles);
-            tile = (int)(item % tiles);
-        }
-        decode_tile(tile, tiles_m, tiles_n, &tm, &tn, SIMT_GROUP);
+    const int64_t items = (int64_t)tiles_m * tiles_n * splits;
+    constexpr int GROUP = 16;
+    auto decode = [&](int64_t item, int& tm, int& tn, int& sp) {
+        const int64_t tiles = (int64_t)tiles_m * tiles_n;
+        sp = (int)(item / tiles);
+        const int tile = (int)(item % tiles);
+        const int per_group = GROUP * tiles_n;
+        const int g = tile / per_group;
+        const int gsz = min(GROUP, tiles_m - g * GROUP);
+        tm = g * GROUP + (tile % per_group) % gsz;
+        tn = (tile % per_group) / gsz;
     };
-    auto kblocks_of = [&](int sp, int64_t slot, int64_t& kbeg) {
-        const int64_t chunk = slot >= 0 ? tail.chunk : kchunk;
-        kbeg = (int64_t)sp * chunk;
-        const int64_t kend = min(k, kbeg + chunk);
+    auto kblocks_of = [&](int sp, int64_t& kbeg) {
+        kbeg = (int64_t)sp * kchunk;
+        const int64_t kend = min(k, kbeg + kchunk);
         return (int)((kend - kbeg + TBK - 1) / TBK);
     };
 
@@ -114,9 +106,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
                 int tm, tn, sp;
-                int64_t slot, kbeg;
-                decode(item, tm, tn, sp, slot);
-                const int kb_n = kblocks_of(sp, slot, kbeg);
+                decode(item, tm, tn, sp);
+                int64_t kbeg;
+                const int kb_n = kblocks_of(sp, kbeg);
                 const int32_t m0 = tm * TBM, n0 = tn * BN;
                 int32_t cw = 0, ch = 0, cn = 0;
                 if (CONV) conv_tile_origin(conv, (int64_t)tn * BN, cw, ch, cn);
@@ -165,9 +157,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
                 int tm, tn, sp;
-                int64_t slot, kbeg;
-                decode(item, tm, tn, sp, slot);
-                const int kb_n = kblocks_of(sp, slot, kbeg);
+                decode(item, tm, tn, sp);
+                int64_t kbeg;
+                const int kb_n = kblocks_of(sp, kbeg);
                 const uint32_t acc = it % NACC, aph = (it / NACC) & 1;
                 if (!mbar_wait(tempty_bar(acc), aph ^ 1, abort_flag, status,
                                STATUS_MARK | (ROLE_MMA << 16) | (BAR_TMEM_EMPTY << 8) | acc)) { ok = false; break; }
@@ -210,24 +202,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
             int tm, tn, sp;
-            int64_t slot;
-            decode(item, tm, tn, sp, slot);
+            decode(item, tm, tn, sp);
             const uint32_t acc = it % NACC, aph = (it / NACC) & 1;
             if (!mbar_wait(tfull_bar(acc), aph, abort_flag, status,
                            STATUS_MARK | (ROLE_EPI << 16) | (BAR_TMEM_FULL << 8) | acc)) { ok = false; break; }
             tc_fence_after();
-            // a tail item stores its whole 128 x BN block, unscaled, into its tile-local slot [column][row];
-            // everything else goes to C (or to the split-k partial sums) at the tile's place
-            const bool tail_item = slot >= 0;
-            const bool raw = tail_item || splits > 1;
-            const int64_t row0 = (tail_item ? 0 : (int64_t)tm * TBM) + q * 32;
-            float* out = tail_item ? tail.partials + slot * (int64_t)(TBM * BN) : (raw ? partials + (int64_t)sp * m * n : C);
+            const int64_t row0 = (int64_t)tm * TBM + q * 32;
+            const bool raw = splits > 1;
+            float* out = raw ? partials + (int64_t)sp * m * n : C;
             // store_via_tma: 0 = direct stores, 1 = tmC maps C (2-D), 2 = tmC maps the split-k partials (3-D: m, n, split)
-            const bool via_tma = !tail_item && (raw ? (store_via_tma == 2) : (store_via_tma == 1));
+            const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
             epilogue_tile<BN, Cfg::STORE_BUFS>(
-                tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row0, tail_item ? 0 : (int64_t)tn * BN, half, lane,
-                tail_item ? (int64_t)TBM : m, tail_item ? (int64_t)BN : n, alpha, beta, out,
-                tail_item ? (int64_t)TBM : (raw ? m : ldc), raw, via_tma, &tmC, sp, stage, sbuf, [&]() {
+                tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta,
+                out, raw ? m : ldc, raw, via_tma, &tmC, sp, stage, sbuf, [&]() {
                     // the accumulator may be overwritten once this warp has read its last chunk
                     tc_fence_before();
                     __syncwarp();
@@ -398,8 +385,7 @@ uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n) {
 
 template <int BN, bool A_MN, bool B_MN, bool CONV>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
-                             const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma,
-                             const TailSplit& tail) {
+                             const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
     static bool attr_set[64] = {};
@@ -413,8 +399,7 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     }
     const int64_t tiles_m = (a.m + TBM - 1) / TBM, tiles_n = (a.n + BN - 1) / BN;
     if (tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF || tiles_m * tiles_n > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    int64_t items = tiles_m * tiles_n * ks.splits;
-    if (tail.first < tiles_m * tiles_n) items = tail.first + (tiles_m * tiles_n - tail.first) * tail.splits;
+    const int64_t items = tiles_m * tiles_n * ks.splits;
     const int grid = (int)(items < sm_count() ? items : sm_count());
     cfg->tile_m = TBM; cfg->tile_n = BN; cfg->tile_k = TBK; cfg->stages = Cfg::STAGES; cfg->grid = grid;
     cudaLaunchConfig_t lc = {};
@@ -430,13 +415,12 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN), a.status, conv_tma_params(a.conv), tail);
+                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN), a.status, conv_tma_params(a.conv));
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <bool A_MN, bool B_MN, bool CONV>
-static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg,
-                                const TailSplit& tail) {
+static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg) {
     CUtensorMap tmA, tmB;
     // stored A: (m x k) if transA = N [contiguous m], (k x m) otherwise [contiguous k]
     bool ok = A_MN ? make_map(&tmA, a.dtype, a.A, a.m, a.k, a.lda, 64, TBK)
@@ -459,24 +443,24 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
         a.m * a.n * 4 < (1LL << 40))
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
     switch (tile_n) {
-        case 256: return launch_tc<256, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, tail);
-        case 128: return launch_tc<128, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, tail);
-        default:  return launch_tc<64, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, tail);
+        case 256: return launch_tc<256, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 128: return launch_tc<128, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        default:  return launch_tc<64, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
     }
 }
 
-cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
+cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg) {
     cfg->kernel = GEMM_KERNEL_TENSOR;
     cfg->split_k = ks.splits;
     cfg->vector_a = cfg->vector_b = 1;
     const bool a_mn = !a.ta, b_mn = a.tb;
     if (a.conv != nullptr)
-        return a_mn ? launch_tc_bn<true, false, true>(a, tile_n, ks, partials, cfg, tail)
-                    : launch_tc_bn<false, false, true>(a, tile_n, ks, partials, cfg, tail);
-    if (a_mn && b_mn) return launch_tc_bn<true, true, false>(a, tile_n, ks, partials, cfg, tail);
-    if (a_mn && !b_mn) return launch_tc_bn<true, false, false>(a, tile_n, ks, partials, cfg, tail);
-    if (!a_mn && b_mn) return launch_tc_bn<false, true, false>(a, tile_n, ks, partials, cfg, tail);
-    return launch_tc_bn<false, false, false>(a, tile_n, ks, partials, cfg, tail);
+        return a_mn ? launch_tc_bn<true, false, true>(a, tile_n, ks, partials, cfg)
+                    : launch_tc_bn<false, false, true>(a, tile_n, ks, partials, cfg);
+    if (a_mn && b_mn) return launch_tc_bn<true, true, false>(a, tile_n, ks, partials, cfg);
+    if (a_mn && !b_mn) return launch_tc_bn<true, false, false>(a, tile_n, ks, partials, cfg);
+    if (!a_mn && b_mn) return launch_tc_bn<false, true, false>(a, tile_n, ks, partials, cfg);
+    return launch_tc_bn<false, false, false>(a, tile_n, ks, partials, cfg);
 }
 
 }  // namespace b200gemm

@@ -78,8 +78,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k,
                     float alpha, float beta, float* __restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int splits,
-                    int64_t kchunk, float* __restrict__ partials, uint32_t idesc, uint32_t* status, const ConvTma conv,
-                    const TailSplit tail) {
+                    int64_t kchunk, float* __restrict__ partials, uint32_t idesc, uint32_t* status, const ConvTma conv) {
     constexpr int STAGES = PAIR_STAGES, NACC = PAIR_NACC, BN = PAIR_BN;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -120,31 +119,22 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // Work items.  Without a tail split: tiles x k partitions (split-k).  With one (splits == 1): items below
-    // tail.first are whole tiles; the tiles of the last, partly filled round come after them, cut into tail.splits
-    // k ranges each, so that the round still gives every pair work and lasts 1 / tail.splits as long; their raw
-    // partial sums go to tile-local slots and a small reduction pass finishes them.
-    const int64_t tiles = (int64_t)tiles_m * tiles_n;
-    const int64_t items = tail.first < tiles ? tail.first + (tiles - tail.first) * tail.splits : tiles * splits;
+    const int64_t items = (int64_t)tiles_m * tiles_n * splits;
     const int64_t pair_id = blockIdx.x >> 1, pairs = gridDim.x >> 1;
-    // slot >= 0: the item is a k range of a tail tile and writes slot `slot` of tail.partials
-    auto decode = [&](int64_t item, int& tm, int& tn, int& sp, int64_t& slot) {
-        int tile;
-        if (item >= tail.first) {
-            slot = item - tail.first;
-            tile = tail.first + (int)(slot / tail.splits);
-            sp = (int)(slot % tail.splits);
-        } else {
-            slot = -1;
-            sp = (int)(item / tiles);
-            tile = (int)(item % tiles);
-        }
-        decode_tile(tile, tiles_m, tiles_n, &tm, &tn, PAIR_GROUP);
+    constexpr int GROUP = 8;     // 8 tile rows of 256 = the 2048 rows a group of the single-CTA kernel covers
+    auto decode = [&](int64_t item, int& tm, int& tn, int& sp) {
+        const int64_t tiles = (int64_t)tiles_m * tiles_n;
+        sp = (int)(item / tiles);
+        const int tile = (int)(item % tiles);
+        const int per_group = GROUP * tiles_n;
+        const int g = tile / per_group;
+        const int gsz = min(GROUP, tiles_m - g * GROUP);
+        tm = g * GROUP + (tile % per_group) % gsz;
+        tn = (tile % per_group) / gsz;
     };
-    auto kblocks_of = [&](int sp, int64_t slot, int64_t& kbeg) {
-        const int64_t chunk = slot >= 0 ? tail.chunk : kchunk;
-        kbeg = (int64_t)sp * chunk;
-        const int64_t kend = min(k, kbeg + chunk);
+    auto kblocks_of = [&](int sp, int64_t& kbeg) {
+        kbeg = (int64_t)sp * kchunk;
+        const int64_t kend = min(k, kbeg + kchunk);
         return (int)((kend - kbeg + TBK - 1) / TBK);
     };
 
@@ -155,9 +145,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             bool ok = true;
             for (int64_t item = pair_id; item < items && ok; item += pairs) {
                 int tm, tn, sp;
-                int64_t slot, kbeg;
-                decode(item, tm, tn, sp, slot);
-                const int kb_n = kblocks_of(sp, slot, kbeg);
+                decode(item, tm, tn, sp);
+                int64_t kbeg;
+                const int kb_n = kblocks_of(sp, kbeg);
                 const int32_t m0 = tm * (2 * TBM) + (int32_t)rank * TBM;            // this CTA's rows of op(A)
                 const int32_t n0 = tn * BN + (int32_t)rank * PAIR_HALF_N;           // this CTA's columns of op(B)
                 int32_t cw = 0, ch = 0, cn = 0;
@@ -211,9 +201,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             bool ok = true;
             for (int64_t item = pair_id; item < items && ok; item += pairs, ++it) {
                 int tm, tn, sp;
-                int64_t slot, kbeg;
-                decode(item, tm, tn, sp, slot);
-                const int kb_n = kblocks_of(sp, slot, kbeg);
+                decode(item, tm, tn, sp);
+                int64_t kbeg;
+                const int kb_n = kblocks_of(sp, kbeg);
                 const uint32_t acc = it % NACC, aph = (it / NACC) & 1;
                 if (!mbar_wait(tempty_bar(acc), aph ^ 1, abort_flag, status,
                                STATUS_MARK | (ROLE_MMA << 16) | (BAR_TMEM_EMPTY << 8) | acc)) { ok = false; break; }
@@ -253,28 +243,22 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         bool ok = true;
         for (int64_t item = pair_id; item < items && ok; item += pairs, ++it) {
             int tm, tn, sp;
-            int64_t slot;
-            decode(item, tm, tn, sp, slot);
+            decode(item, tm, tn, sp);
             const uint32_t acc = it % NACC, aph = (it / NACC) & 1;
             if (!mbar_wait(tfull_bar(acc), aph, abort_flag, status,
                            STATUS_MARK | (ROLE_EPI << 16) | (BAR_TMEM_FULL << 8) | acc)) { ok = false; break; }
             tc_fence_after();
-            // a tail item stores its whole 256 x 256 block, unscaled, into its tile-local slot [column][row];
-            // everything else goes to C (or to the split-k partial sums) at the tile's place
-            const bool tail_item = slot >= 0;
-            const bool raw = tail_item || splits > 1;
-            const int64_t row0 = (tail_item ? 0 : (int64_t)tm * (2 * TBM)) + (int64_t)rank * TBM + q * 32;
-            const int64_t n0 = tail_item ? 0 : (int64_t)tn * BN;
-            float* out = tail_item ? tail.partials + slot * (int64_t)(2 * TBM * BN) : (raw ? partials + (int64_t)sp * m * n : C);
-            const int64_t ldo = tail_item ? 2 * TBM : (raw ? m : ldc);
-            const bool via_tma = !tail_item && (raw ? (store_via_tma == 2) : (store_via_tma == 1));
-            epilogue_tile<BN, 1>(tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row0, n0, half, lane,
-                                 tail_item ? (int64_t)(2 * TBM) : m, tail_item ? (int64_t)BN : n, alpha, beta, out, ldo, raw,
-                                 via_tma, &tmC, sp, stage, sbuf, [&]() {
-                                     tc_fence_before();
-                                     __syncwarp();
-                                     if (lane == 0) mbar_arrive_cluster(tempty_leader0 + 8u * acc);
-                                 });
+            const int64_t row0 = (int64_t)tm * (2 * TBM) + (int64_t)rank * TBM + q * 32;
+            const bool raw = splits > 1;
+            float* out = raw ? partials + (int64_t)sp * m * n : C;
+            const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
+            epilogue_tile<BN, 1>(
+                tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta,
+                out, raw ? m : ldc, raw, via_tma, &tmC, sp, stage, sbuf, [&]() {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(tempty_leader0 + 8u * acc);
+                });
         }
         if (lane == 0) bulk_wait_all();
     }
@@ -291,7 +275,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 }
 
 template <bool A_MN, bool B_MN, bool CONV>
-static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg, const TailSplit& tail) {
+static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg) {
     CUtensorMap tmA, tmB;
     bool ok = A_MN ? make_map(&tmA, a.dtype, a.A, a.m, a.k, a.lda, 64, TBK)
                    : make_map(&tmA, a.dtype, a.A, a.k, a.m, a.lda, TBK, TBM);
@@ -320,8 +304,7 @@ static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     }
     const int64_t tiles_m = (a.m + 2 * TBM - 1) / (2 * TBM), tiles_n = (a.n + PAIR_BN - 1) / PAIR_BN;
     if (tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF || tiles_m * tiles_n > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    int64_t items = tiles_m * tiles_n * ks.splits;
-    if (tail.first < tiles_m * tiles_n) items = tail.first + (tiles_m * tiles_n - tail.first) * tail.splits;
+    const int64_t items = tiles_m * tiles_n * ks.splits;
     const int64_t max_pairs = sm_count() / 2;
     const int grid = 2 * (int)(items < max_pairs ? items : max_pairs);
     cfg->tile_m = 2 * TBM; cfg->tile_n = PAIR_BN; cfg->tile_k = TBK; cfg->stages = PAIR_STAGES; cfg->grid = grid;
@@ -342,21 +325,21 @@ static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status, conv_tma_params(a.conv), tail);
+                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status, conv_tma_params(a.conv));
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
-cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
+cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg) {
     cfg->kernel = GEMM_KERNEL_TENSOR;
     cfg->split_k = ks.splits;
     cfg->vector_a = cfg->vector_b = 1;
     const bool a_mn = !a.ta, b_mn = a.tb;
     if (a.conv != nullptr)
-        return a_mn ? launch_pair<true, false, true>(a, ks, partials, cfg, tail) : launch_pair<false, false, true>(a, ks, partials, cfg, tail);
-    if (a_mn && b_mn) return launch_pair<true, true, false>(a, ks, partials, cfg, tail);
-    if (a_mn && !b_mn) return launch_pair<true, false, false>(a, ks, partials, cfg, tail);
-    if (!a_mn && b_mn) return launch_pair<false, true, false>(a, ks, partials, cfg, tail);
-    return launch_pair<false, false, false>(a, ks, partials, cfg, tail);
+        return a_mn ? launch_pair<true, false, true>(a, ks, partials, cfg) : launch_pair<false, false, true>(a, ks, partials, cfg);
+    if (a_mn && b_mn) return launch_pair<true, true, false>(a, ks, partials, cfg);
+    if (a_mn && !b_mn) return launch_pair<true, false, false>(a, ks, partials, cfg);
+    if (!a_mn && b_mn) return launch_pair<false, true, false>(a, ks, partials, cfg);
+    return launch_pair<false, false, false>(a, ks, partials, cfg);
 }
 
 }  // namespace b200gemm

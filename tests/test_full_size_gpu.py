@@ -63,29 +63,6 @@ def test_config5_half_squares_4096_8192(dtype):
         assert (cfg["tile_m"], cfg["tile_n"]) == (256, 256)      # large squares run on CTA pairs
 
 
-def test_tensor_kernels_tail_split_of_the_last_round():
-    # 1021 x 10491: 164 tiles of 256 x 256 on 74 pairs (last round 16), 328 of 128 x 256 on 148 CTAs (last round 32),
-    # 656 of 128 x 128 (last round 64): the tiles of the last round are cut into k ranges, finished by the tile-local
-    # reduction; 4096^3 (256 tiles on pairs, last round 34) takes the same path by the selector's own choice
-    from workloads import Problem
-    try:
-        for tile in ((256, 256), (128, 256), (128, 128)):
-            g.gemm_force_tile(tile[0], tile[1], 0)
-            for dtype, kind in ((DTYPE_BF16, "normal"), (DTYPE_F16, "int")):
-                p = Problem("tail", dtype, 1024 - 3, 10496 - 5, 1024 + 64, 1.5, 0.5, kindA=kind, kindB=kind,
-                            kindC="int" if kind == "int" else "uniform", seed=21)
-                cfg, _ = run_and_check(p, seed=3)
-                assert (cfg["tile_m"], cfg["tile_n"], cfg["split_k"]) == (tile[0], tile[1], 1), cfg
-                assert cfg["tail_split"] >= 2 and cfg["launches"] >= 2, (cfg["tail_split"], cfg["launches"])     # + repacking passes
-    finally:
-        g.gemm_force_tile(0, 0, 0)
-    cfg, _ = run_and_check(config_problems(5, dtype=DTYPE_BF16)[0], seed=4)
-    assert cfg["tail_split"] == 2, cfg
-    # 256 tiles = 3 rounds of 74 pairs + 34; the 34 are cut in two along k, one fp32 256 x 256 slot each
-    assert g.gemm_workspace_bytes(DTYPE_BF16, "N", "N", 4096, 4096, 4096) == 34 * 2 * 256 * 256 * 4
-    assert g.gemm_workspace_bytes(DTYPE_BF16, "N", "N", 8192, 8192, 8192) == 0          # last round more than half full
-
-
 def test_config5_f16_square_16384():
     p = config_problems(5, dtype=DTYPE_F16)[2]
     cfg, _ = run_and_check(p)
