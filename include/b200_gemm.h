@@ -21,11 +21,17 @@
 extern "C" {
 #endif
 
-/* element types of A and B; C is always fp32 */
+/* element types of A and B, and of C: fp32 unless the name says otherwise */
 typedef enum {
     GEMM_F32  = 0,  /* A, B fp32; exact IEEE fp32 fused multiply-add arithmetic on the CUDA cores          */
     GEMM_F16  = 1,  /* A, B IEEE binary16; products accumulated in fp32 on the tensor cores (tcgen05/TMEM) */
-    GEMM_BF16 = 2   /* A, B bfloat16;      products accumulated in fp32 on the tensor cores                 */
+    GEMM_BF16 = 2,  /* A, B bfloat16;      products accumulated in fp32 on the tensor cores                 */
+    /* All-16-bit forms (Section III, "Data types": the generated f16 micro-kernel keeps A, B and C in 16-bit
+     * storage).  A, B and C are of the one 16-bit type; products are still accumulated in fp32, and
+     * alpha*acc + beta*C is rounded once, to nearest even, when it is stored.  Wherever this header says that C
+     * is fp32, read "of the 16-bit type" for these two; ldc counts elements of that type. */
+    GEMM_F16_C16  = 3,
+    GEMM_BF16_C16 = 4
 } gemm_dtype_t;
 
 /* return codes (0 = success; -1 .. -15 = the 1-based position of the first invalid argument of gemm()) */
@@ -74,7 +80,7 @@ typedef struct {
  *   A, lda         device pointer; stored m x k (lda >= max(1,m)) if transA = N, else k x m (lda >= max(1,k));
  *                  elements of `dtype`; never written
  *   B, ldb         device pointer; stored k x n (ldb >= max(1,k)) if transB = N, else n x k (ldb >= max(1,n))
- *   C, ldc         device pointer to fp32, m x n, ldc >= max(1,m); read only if beta != 0 (so NaN/Inf in C
+ *   C, ldc         device pointer to fp32 (16-bit for the *_C16 types), m x n, ldc >= max(1,m); read only if beta != 0 (so NaN/Inf in C
  *                  do not propagate when beta == 0); rows m..ldc-1 of every column are never touched
  *   alpha, beta    fp32 scalars by value
  *   stream         cudaStream_t (NULL = the default stream)
@@ -157,7 +163,7 @@ int gemm_f32_splitk_static(char transA, char transB, int64_t m, int64_t n, int64
  *     X       device pointer, NHWC activations of `dtype`: element (b, h, w, c) at ((b*H + h)*W + w)*C_in + c
  *     W, ldw  device pointer, the filters as a column-major C_out x k matrix of `dtype` (ldw >= C_out), i.e.
  *             element (co; r, s, c) at co + ((r*kw + s)*C_in + c)*ldw
- *     Y, ldy  device pointer to fp32, NHWC result: element (co; pixel j) at co + j*ldy, ldy >= C_out; read only if
+ *     Y, ldy  device pointer to fp32 (16-bit for the *_C16 types: a layer's result can then feed the next layer), NHWC result: element (co; pixel j) at co + j*ldy, ldy >= C_out; read only if
  *             beta != 0; rows C_out..ldy-1 are never touched
  *   Where it can, the lowering is fused into the operand staging of the GEMM kernels and L never exists in memory:
  *   fp32 reads X through the index map inside the SIMT kernel's loads; fp16/bf16 layers with C_in a multiple of

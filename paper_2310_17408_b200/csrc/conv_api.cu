@@ -94,7 +94,8 @@ static cudaError_t launch_im2row(int dtype, const ConvIndex& cv, int64_t pixels,
 
 // ---- validation shared by the entry points: fills the index map; returns 0 or the negative argument position
 static int conv_setup(int dtype, const conv_shape_t* sh, const void* X, ConvIndex* cv, int64_t* m, int64_t* n, int64_t* k) {
-    if (dtype != GEMM_F32 && dtype != GEMM_F16 && dtype != GEMM_BF16) return -1;
+    if (dtype != GEMM_F32 && dtype != GEMM_F16 && dtype != GEMM_BF16 && dtype != GEMM_F16_C16 && dtype != GEMM_BF16_C16)
+        return -1;
     if (sh == nullptr) return -2;
     if (sh->batch < 0 || sh->h < 1 || sh->w < 1 || sh->c_in < 1 || sh->c_out < 0 || sh->kh < 1 || sh->kw < 1 ||
         sh->stride_h < 1 || sh->stride_w < 1 || sh->pad_h < 0 || sh->pad_w < 0)
@@ -149,7 +150,7 @@ int im2row(int dtype, const conv_shape_t* shape, const void* X, void* out, int64
     if (X == nullptr || (reinterpret_cast<uintptr_t>(X) % es) != 0) return -3;
     if (out == nullptr || (reinterpret_cast<uintptr_t>(out) % es) != 0) return -4;
     if (ld < k) return -5;
-    const cudaError_t e = launch_im2row(dtype, cv, n, X, out, ld, static_cast<cudaStream_t>(stream));
+    const cudaError_t e = launch_im2row(input_dtype(dtype), cv, n, X, out, ld, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
     return GEMM_OK;
 }
@@ -162,7 +163,7 @@ size_t conv2d_workspace_bytes(int dtype, const conv_shape_t* shape) {
     size_t need = gemm_workspace_bytes(dtype, 'N', 'N', m, n, k);
     if (lowering_is_identity(cv)) return need;
     // judged for 16-byte aligned tensors and a filter matrix TMA can address
-    const bool fused = fused_possible(dtype, cv, shape->batch, reinterpret_cast<const void*>(16), 8);
+    const bool fused = fused_possible(input_dtype(dtype), cv, shape->batch, reinterpret_cast<const void*>(16), 8);
     const bool scalar_map = dtype == GEMM_F32 && cv.c_in % 4 != 0;       // served faster by writing L first
     if (!fused || scalar_map || g_force_lowering == CONV_LOWERING_EXPLICIT)
         need += (size_t)rup(rup(k, 8) * n * elem_size(dtype), 256);
@@ -183,7 +184,7 @@ int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void*
     if (W != nullptr && (reinterpret_cast<uintptr_t>(W) % es) != 0) return -5;
     if (ldw < (m > 1 ? m : 1)) return -6;
     if (m > 0 && n > 0 && Y == nullptr) return -8;
-    if (Y != nullptr && (reinterpret_cast<uintptr_t>(Y) % 4) != 0) return -8;
+    if (Y != nullptr && (reinterpret_cast<uintptr_t>(Y) % c_elem_size(dtype)) != 0) return -8;
     if (ldy < (m > 1 ? m : 1)) return -9;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
@@ -194,8 +195,9 @@ int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void*
         return rc;
     }
 
-    GemmArgs a{dtype, false, false, m, n, k, alpha, beta, W, nullptr, static_cast<float*>(Y), ldw, k, ldy, s, nullptr};
-    const bool can_fuse = fused_possible(dtype, cv, shape->batch, W, ldw);
+    GemmArgs a{input_dtype(dtype), false, false, m, n, k, alpha, beta, W, nullptr, static_cast<float*>(Y), ldw, k, ldy, s, nullptr};
+    a.out16 = output16(dtype);
+    const bool can_fuse = fused_possible(input_dtype(dtype), cv, shape->batch, W, ldw);
     void* ws = nullptr;
     size_t ws_bytes = 0;
     if (!registered_workspace(&ws, &ws_bytes)) return GEMM_ERR_LAUNCH;
@@ -223,7 +225,7 @@ int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void*
         if (rc == GEMM_OK) note_lowering(CONV_LOWERING_FUSED);
         return rc;
     }
-    const cudaError_t e = launch_im2row(dtype, cv, n, X, ws, ld, s);
+    const cudaError_t e = launch_im2row(input_dtype(dtype), cv, n, X, ws, ld, s);
     if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
     a.B = ws;
     a.ldb = ld;

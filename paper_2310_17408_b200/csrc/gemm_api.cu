@@ -281,7 +281,8 @@ static int validate(int dtype, char ta, char tb, int64_t m, int64_t n, int64_t k
             default: return false;
         }
     };
-    if (dtype != GEMM_F32 && dtype != GEMM_F16 && dtype != GEMM_BF16) return -1;
+    if (dtype != GEMM_F32 && dtype != GEMM_F16 && dtype != GEMM_BF16 && dtype != GEMM_F16_C16 && dtype != GEMM_BF16_C16)
+        return -1;
     if (!tr(ta, tA)) return -2;
     if (!tr(tb, tB)) return -3;
     if (m < 0) return -4;
@@ -297,7 +298,7 @@ static int validate(int dtype, char ta, char tb, int64_t m, int64_t n, int64_t k
     if (B != nullptr && (reinterpret_cast<uintptr_t>(B) % es) != 0) return -10;
     if (ldb < (b_rows > 1 ? b_rows : 1)) return -11;
     if (m > 0 && n > 0 && C == nullptr) return -13;
-    if (C != nullptr && (reinterpret_cast<uintptr_t>(C) % 4) != 0) return -13;
+    if (C != nullptr && (reinterpret_cast<uintptr_t>(C) % c_elem_size(dtype)) != 0) return -13;
     if (ldc < (m > 1 ? m : 1)) return -14;
     return 0;
 }
@@ -424,8 +425,9 @@ int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, f
     DeviceState* st = device_state();
     if (!st) return GEMM_ERR_LAUNCH;
     if (!st->arch_ok) return GEMM_ERR_ARCH;
-    GemmArgs a{dtype, ta, tb, m, n, k, alpha, beta, A, B, static_cast<float*>(C), lda, ldb, ldc,
+    GemmArgs a{input_dtype(dtype), ta, tb, m, n, k, alpha, beta, A, B, static_cast<float*>(C), lda, ldb, ldc,
                static_cast<cudaStream_t>(stream), st->status};
+    a.out16 = output16(dtype);
     return run_gemm(a, st);
 }
 
@@ -468,16 +470,17 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
             pipe->init = true;
         }
     }
-    const int es = elem_size(dtype);
+    const int es = elem_size(dtype);       // of A and B
     const bool needs_ab = (k > 0 && alpha != 0.0f);
     const int64_t a_rows = ta ? k : m, a_cols = ta ? m : k;
     const size_t a_bytes = needs_ab ? (size_t)lda * a_cols * es : 0;
     const size_t b_bytes = needs_ab ? (size_t)ldb * (tb ? k : n) * es : 0;
-    const size_t c_bytes = (size_t)ldc * n * sizeof(float);
+    const int es_c = c_elem_size(dtype);
+    const size_t c_bytes = (size_t)ldc * n * es_c;
 
     // Column panels of C (and of op(B)) flow through a three-stream pipeline: panel p+1 is copied in while panel p
     // is multiplied and panel p-1 is copied out.  Small problems use one panel.
-    const double traffic = (double)b_bytes + (double)m * n * 4.0 * (beta != 0.0f ? 2.0 : 1.0);
+    const double traffic = (double)b_bytes + (double)m * n * es_c * (beta != 0.0f ? 2.0 : 1.0);
     int64_t panel = n;
     if (traffic > 32e6 && n >= 1024) {
         int64_t panels = (int64_t)(traffic / 48e6) + 1;
@@ -532,10 +535,10 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
             if (tb) chk(copy_window(dBp + b_off, hB + b_off, cols, k, ldb, es, cudaMemcpyHostToDevice, pipe->in));
             else chk(copy_window(dBp + b_off, hB + b_off, k, cols, ldb, es, cudaMemcpyHostToDevice, pipe->in));
         }
-        const size_t c_off = (size_t)j0 * ldc * sizeof(float);
+        const size_t c_off = (size_t)j0 * ldc * es_c;
         // only the m x cols window of C travels: the host's padding rows are never touched
         if (beta != 0.0f)
-            chk(copy_window(static_cast<char*>(dC) + c_off, static_cast<const char*>(C_host) + c_off, m, cols, ldc, 4,
+            chk(copy_window(static_cast<char*>(dC) + c_off, static_cast<const char*>(C_host) + c_off, m, cols, ldc, es_c,
                             cudaMemcpyHostToDevice, pipe->in));
         chk(cudaEventRecord(ev_in, pipe->in));
         chk(cudaStreamWaitEvent(s, ev_in, 0));
@@ -554,7 +557,7 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
                 chk(cudaStreamWaitEvent(s, ev_row, 0));
                 if (e != cudaSuccess) break;
                 rc = gemm(dtype, transA, transB, rows, cols, k, alpha, dAp, lda, dBp + b_off, ldb, beta,
-                          static_cast<char*>(dC) + c_off + (size_t)i0 * sizeof(float), ldc, stream);
+                          static_cast<char*>(dC) + c_off + (size_t)i0 * es_c, ldc, stream);
             }
         } else {
             rc = gemm(dtype, transA, transB, m, cols, k, alpha, dA, lda, needs_ab ? dBp + b_off : nullptr, ldb, beta,
@@ -563,7 +566,7 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
         if (rc != GEMM_OK || e != cudaSuccess) break;
         chk(cudaEventRecord(ev_mul, s));
         chk(cudaStreamWaitEvent(pipe->out, ev_mul, 0));
-        chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols, ldc, 4,
+        chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols, ldc, es_c,
                         cudaMemcpyDeviceToHost, pipe->out));
     }
     if (made > 2) {
@@ -591,7 +594,7 @@ size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int6
     DeviceState* st = device_state();
     const int sms = st ? st->sms : 148;
     // judged for 16-byte aligned pointers and minimal leading dimensions (lda = rows of the stored A, ...)
-    GemmArgs a{dtype, ta, tb, m, n, k, 1.0f, 0.0f, (const void*)16, (const void*)16, nullptr,
+    GemmArgs a{input_dtype(dtype), ta, tb, m, n, k, 1.0f, 0.0f, (const void*)16, (const void*)16, nullptr,
                ta ? k : m, tb ? n : k, m, nullptr, nullptr};
     Plan p = make_plan(a, sms, ~(size_t)0);
     return p.kernel < 0 ? 0 : p.ws_total;

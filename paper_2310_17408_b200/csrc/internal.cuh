@@ -30,7 +30,32 @@ struct GemmArgs {
     cudaStream_t stream;
     uint32_t* status;      // device status word (bounded waits report here)
     const ConvIndex* conv = nullptr;   // non-null: op(B) is the lowered activation matrix of this layer (B, ldb, tb unused)
+    int out16 = 0;                     // element type of C: 0 = fp32, GEMM_F16 / GEMM_BF16 = that 16-bit type (C then points to it)
 };
+
+// The all-16-bit data types (GEMM_F16_C16, GEMM_BF16_C16) are a 16-bit input type plus a 16-bit result:
+// inside the library dtype is always the input type and out16 names the result's type.
+inline int input_dtype(int dtype) { return dtype == GEMM_F16_C16 ? GEMM_F16 : (dtype == GEMM_BF16_C16 ? GEMM_BF16 : dtype); }
+inline int output16(int dtype) { return dtype == GEMM_F16_C16 ? GEMM_F16 : (dtype == GEMM_BF16_C16 ? GEMM_BF16 : 0); }
+inline int c_elem_size(int dtype) { return output16(dtype) ? 2 : 4; }
+
+// fp32 <-> the 16-bit result types, round to nearest even (device)
+#ifdef __CUDACC__
+__device__ __forceinline__ uint16_t f32_to_bits16(float v, int out16) {
+    return out16 == GEMM_F16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+__device__ __forceinline__ float bits16_to_f32(uint16_t b, int out16) {
+    return out16 == GEMM_F16 ? __half2float(__ushort_as_half(b)) : __bfloat162float(__ushort_as_bfloat16(b));
+}
+// element i of C in either representation
+__device__ __forceinline__ float load_c(const float* C, int out16, int64_t i) {
+    return out16 ? bits16_to_f32(reinterpret_cast<const uint16_t*>(C)[i], out16) : C[i];
+}
+__device__ __forceinline__ void store_c(float* C, int out16, int64_t i, float v) {
+    if (out16) reinterpret_cast<uint16_t*>(C)[i] = f32_to_bits16(v, out16);
+    else C[i] = v;
+}
+#endif
 
 // k partition used by every split-k path: split s covers [s*chunk, min(k, (s+1)*chunk))
 struct KSplit {
@@ -62,7 +87,7 @@ __host__ __device__ inline void decode_tile(int tile, int tiles_m, int tiles_n, 
     *tn = (tile % per_group) / gsz;
 }
 
-inline int elem_size(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }
+inline int elem_size(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }      // of A and B
 
 // C <- beta*C  (beta == 0: store +0 without reading)
 cudaError_t launch_scale(const GemmArgs& a);

@@ -16,6 +16,12 @@ __device__ __forceinline__ float epilogue(float alpha, float acc, float beta, co
     if (beta != 0.0f) r = fmaf(beta, *c, r);
     return r;
 }
+// the same on element i of a C that may be 16-bit: one rounding to the result type at the store
+__device__ __forceinline__ void epilogue_store(float alpha, float acc, float beta, float* C, int out16, int64_t i) {
+    float r = alpha * acc;
+    if (beta != 0.0f) r = fmaf(beta, load_c(C, out16, i), r);
+    store_c(C, out16, i, r);
+}
 
 constexpr int GT = 64;   // CTA tile (GT x GT) of C
 constexpr int GK = 16;   // k extent of one shared-memory stage
@@ -25,7 +31,7 @@ template <typename T, bool TA, bool TB>
 __global__ void __launch_bounds__(256)
 simt_generic_kernel(int64_t m, int64_t n, int64_t k, float alpha, const T* __restrict__ A, int64_t lda,
                     const T* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
-                    int64_t tiles_m) {
+                    int64_t tiles_m, int out16) {
     __shared__ float As[GK][GT + 1];
     __shared__ float Bs[GK][GT + 1];
     const int t = threadIdx.x;
@@ -80,10 +86,7 @@ simt_generic_kernel(int64_t m, int64_t n, int64_t k, float alpha, const T* __res
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             int64_t gi = i0 + tx + 16 * i;
-            if (gi < m) {
-                float* c = C + gi + gj * ldc;
-                *c = epilogue(alpha, acc[i][j], beta, c);
-            }
+            if (gi < m) epilogue_store(alpha, acc[i][j], beta, C, out16, gi + gj * ldc);
         }
     }
 }
@@ -98,7 +101,7 @@ static cudaError_t launch_generic_t(const GemmArgs& a) {
     const T* B = (const T*)a.B;
 #define LAUNCH(TA_, TB_)                                                                              \
     simt_generic_kernel<T, TA_, TB_><<<grid, block, 0, a.stream>>>(a.m, a.n, a.k, a.alpha, A, a.lda, B, \
-                                                                   a.ldb, a.beta, a.C, a.ldc, tiles_m)
+                                                                   a.ldb, a.beta, a.C, a.ldc, tiles_m, a.out16)
     if (!a.ta && !a.tb) LAUNCH(false, false);
     else if (a.ta && !a.tb) LAUNCH(true, false);
     else if (!a.ta && a.tb) LAUNCH(false, true);
@@ -121,18 +124,18 @@ cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg) {
 // ---------------------------------------------------------------- C <- beta*C
 
 __global__ void __launch_bounds__(256)
-scale_kernel(int64_t m, int64_t n, float beta, float* __restrict__ C, int64_t ldc) {
+scale_kernel(int64_t m, int64_t n, float beta, float* __restrict__ C, int64_t ldc, int out16) {
     for (int64_t j = blockIdx.y; j < n; j += gridDim.y)
         for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (int64_t)gridDim.x * blockDim.x) {
-            float* c = C + i + j * ldc;
-            *c = (beta == 0.0f) ? 0.0f : beta * *c;
+            const int64_t e = i + j * ldc;
+            store_c(C, out16, e, (beta == 0.0f) ? 0.0f : beta * load_c(C, out16, e));
         }
 }
 
 cudaError_t launch_scale(const GemmArgs& a) {
     unsigned gx = (unsigned)((a.m + 255) / 256 > 1024 ? 1024 : (a.m + 255) / 256);
     unsigned gy = (unsigned)(a.n > 32768 ? 32768 : a.n);
-    scale_kernel<<<dim3(gx, gy), 256, 0, a.stream>>>(a.m, a.n, a.beta, a.C, a.ldc);
+    scale_kernel<<<dim3(gx, gy), 256, 0, a.stream>>>(a.m, a.n, a.beta, a.C, a.ldc, a.out16);
     return cudaGetLastError();
 }
 
@@ -143,7 +146,7 @@ cudaError_t launch_scale(const GemmArgs& a) {
 template <int V>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(int64_t m, int64_t n, int splits, const float* __restrict__ partials, float alpha, float beta,
-                     float* __restrict__ C, int64_t ldc) {
+                     float* __restrict__ C, int64_t ldc, int out16) {
     const int64_t plane = m * n;
     const int64_t mv = m / V;
     for (int64_t j = (int64_t)blockIdx.y * blockDim.y + threadIdx.y; j < n; j += (int64_t)gridDim.y * blockDim.y)
@@ -166,21 +169,21 @@ splitk_reduce_kernel(int64_t m, int64_t n, int splits, const float* __restrict__
             } else {
                 float s = *p;
                 for (int z = 1; z < splits; ++z) s += p[(int64_t)z * plane];
-                *c = epilogue(alpha, s, beta, c);
+                epilogue_store(alpha, s, beta, C, out16, iv + j * ldc);
             }
         }
 }
 
 cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* partials) {
-    const bool vec = a.m % 4 == 0 && a.ldc % 4 == 0 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 &&
-                     (reinterpret_cast<uintptr_t>(a.C) & 15) == 0;
+    const bool vec = a.out16 == 0 && a.m % 4 == 0 && a.ldc % 4 == 0 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 &&
+                     (reinterpret_cast<uintptr_t>(a.C) & 15) == 0;       // 128-bit path: fp32 results only
     const int64_t mv = vec ? a.m / 4 : a.m;
     int64_t gx = (mv + 31) / 32, gy = (a.n + 7) / 8;
     if (gx > 1024) gx = 1024;
     if (gy > 32768) gy = 32768;
     dim3 grid((unsigned)gx, (unsigned)gy), block(32, 8);
-    if (vec) splitk_reduce_kernel<4><<<grid, block, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc);
-    else splitk_reduce_kernel<1><<<grid, block, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc);
+    if (vec) splitk_reduce_kernel<4><<<grid, block, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc, a.out16);
+    else splitk_reduce_kernel<1><<<grid, block, 0, a.stream>>>(a.m, a.n, splits, partials, a.alpha, a.beta, a.C, a.ldc, a.out16);
     return cudaGetLastError();
 }
 

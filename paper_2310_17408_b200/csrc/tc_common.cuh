@@ -204,6 +204,71 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int64_t row0, i
     if (!released) release_acc();
 }
 
+// The same for a 16-bit result (out16 = GEMM_F16 or GEMM_BF16; never for split-k partial sums): `out` and tmC are
+// in that type and alpha*acc + beta*C0 is rounded once, to nearest even, at the store.  Two rows of one column are
+// packed into a 32-bit word before they go to the staging tile: neighbouring lanes swap one value per column pair, so
+// that the even lane holds rows (2i, 2i+1) of column j and the odd lane those of column j+1, and each converts and
+// stores one word (one packed conversion and one shared-memory store per two entries).
+template <int BN, int STORE_BUFS, typename Release>
+__device__ __forceinline__ void epilogue_tile16(uint32_t tmem_acc, int64_t row0, int64_t n0, int half, int lane,
+                                                int64_t m, int64_t n, float alpha, float beta, float* out, int64_t ldo,
+                                                bool via_tma, const CUtensorMap* tmC, float* stage, uint32_t& sbuf,
+                                                int out16, Release&& release_acc) {
+    const int64_t row = row0 + lane;
+    const bool odd = lane & 1;
+    bool released = false;
+    if (row0 < m) {
+#pragma unroll 1
+        for (int c = half; c < BN / 32; c += 2) {
+            const int64_t col0 = n0 + c * 32;
+            if (col0 >= n) break;
+            const bool last_chunk = (c + 2 >= BN / 32) || (col0 + 64 >= n);
+            uint32_t v[32];
+            tmem_ld32(tmem_acc + c * 32, v);
+            const int64_t e0 = row + col0 * ldo;
+            tmem_ld_wait();
+            if (last_chunk) { release_acc(); released = true; }
+            float* r = reinterpret_cast<float*>(v);       // scaled in place
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                r[j] *= alpha;
+                if (beta != 0.0f && row < m && col0 + j < n) r[j] = fmaf(beta, load_c(out, out16, e0 + j * ldo), r[j]);
+            }
+            if (via_tma) {
+                if (lane == 0) bulk_wait_read<STORE_BUFS - 1>();   // the store that last used this staging tile has read it
+                __syncwarp();
+                uint32_t* st32 = reinterpret_cast<uint32_t*>(stage + sbuf * (32 * 32));      // [column][16 row pairs]
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    const float got = __shfl_xor_sync(0xFFFFFFFFu, odd ? r[j] : r[j + 1], 1);
+                    const float lo = odd ? got : r[j], hi = odd ? r[j + 1] : got;       // rows 2i, 2i+1 of this lane's column
+                    uint32_t word;
+                    if (out16 == GEMM_F16) {
+                        const __half2 h = __floats2half2_rn(lo, hi);
+                        word = *reinterpret_cast<const uint32_t*>(&h);
+                    } else {
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+                        word = *reinterpret_cast<const uint32_t*>(&h);
+                    }
+                    st32[(j + (odd ? 1 : 0)) * 16 + (lane >> 1)] = word;
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(tmC, smem_u32(st32), (int32_t)row0, (int32_t)col0);
+                    bulk_commit();
+                }
+                sbuf = (sbuf + 1 == (uint32_t)STORE_BUFS) ? 0 : sbuf + 1;
+            } else if (row < m) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (col0 + j < n) store_c(out, out16, e0 + j * ldo, r[j]);
+            }
+        }
+    }
+    if (!released) release_acc();
+}
+
 // ---------------------------------------------------------------- host side (defined in tc_gemm.cu)
 
 // 2-D map over a stored column-major matrix of 16-bit elements: dim0 = contiguous dimension (rows), dim1 = columns
@@ -212,13 +277,19 @@ bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_
               uint32_t box_rows, uint32_t box_cols);
 // map over the split-k partial sums [split][n][m] (fp32, dense): 32 x 32 x 1 boxes
 bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits);
-// map over the fp32 result for the epilogue's tile stores: 32 x 32 boxes, no swizzle
-bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc);
+// map over the result (fp32, or the 16-bit type out16) for the epilogue's tile stores: 32 x 32 boxes, no swizzle
+bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc, int out16);
+// whether C (of either element size) can be written by TMA tile stores: 16-byte aligned base and column stride, and
+// columns whose m elements end on a 16-byte boundary.  The last condition keeps the rows m..ldc-1 untouched: a tile
+// store that is clipped at the matrix edge was seen to write the whole 16-byte unit the edge falls into (binary16
+// result, m = 5, ldc = 8: rows 5..7 came back as zeros).
+inline bool c_tma_addressable(const float* C, int64_t m, int64_t ldc, int out16) {
+    const int es = out16 ? 2 : 4;
+    return (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc * es) % 16 == 0 && ldc * es < (1LL << 40) && (m * es) % 16 == 0;
+}
 // im2col-mode map over NHWC activations of a 16-bit type: boxes of `pixels` output pixels x 64 channels, 128-byte
 // swizzle; square filter ksize, the same stride and padding in both directions
 bool make_im2col_map(CUtensorMap* tm, int dtype, const ConvIndex& cv, int64_t batch, uint32_t pixels);
-// whether the lowering of this layer can be done by TMA (channel count, alignment, symmetric geometry, field ranges)
-bool conv_tma_eligible(int dtype, const ConvIndex& cv, int64_t batch);
 inline ConvTma conv_tma_params(const ConvIndex* cv) {
     if (!cv) return ConvTma{1, 1, 1, 0, 1, 1};
     return ConvTma{cv->ho, cv->wo, cv->sh, cv->ph, cv->kw, (int32_t)(cv->c_in / 64)};

@@ -33,12 +33,12 @@ template <int BN> struct TcCfg {
 // A_MN: op(A) is contiguous along m in memory (transA = N); B_MN: op(B) contiguous along n (transB = T).
 // CONV: op(B) is the im2row-lowered activation matrix of a convolution layer, fetched by TMA in im2col mode
 // straight from the NHWC tensor (tmB is then an im2col map); the lowered matrix never exists in memory.
-template <int BN, bool A_MN, bool B_MN, bool CONV>
+template <int BN, bool A_MN, bool B_MN, bool CONV, bool OUT16>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
-               uint32_t idesc, uint32_t* status, const ConvTma conv) {
+               uint32_t idesc, uint32_t* status, const ConvTma conv, int out16) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -212,14 +212,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float* out = raw ? partials + (int64_t)sp * m * n : C;
             // store_via_tma: 0 = direct stores, 1 = tmC maps C (2-D), 2 = tmC maps the split-k partials (3-D: m, n, split)
             const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
-            epilogue_tile<BN, Cfg::STORE_BUFS>(
-                tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta,
-                out, raw ? m : ldc, raw, via_tma, &tmC, sp, stage, sbuf, [&]() {
-                    // the accumulator may be overwritten once this warp has read its last chunk
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar(acc));
-                });
+            auto release = [&]() {      // the accumulator may be overwritten once this warp has read its last chunk
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+            };
+            const uint32_t tacc = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+            bool done = false;
+            if constexpr (OUT16) {
+                if (!raw) {      // 16-bit result: one rounding at the store (split-k partial sums stay fp32)
+                    epilogue_tile16<BN, Cfg::STORE_BUFS>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, out, ldc,
+                                                store_via_tma == 1, &tmC, stage, sbuf, out16, release);
+                    done = true;
+                }
+            }
+            if (!done)
+                epilogue_tile<BN, Cfg::STORE_BUFS>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, out, raw ? m : ldc,
+                                          raw, via_tma, &tmC, sp, stage, sbuf, release);
         }
         if (lane == 0) bulk_wait_all();       // staging tiles must outlive the stores that read them
     }
@@ -303,14 +312,16 @@ bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n,
 }
 
 // map over the fp32 result for the epilogue's tile stores: 32 x 32 boxes, no swizzle
-bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc) {
+bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc, int out16) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)n};
-    cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+    cuuint64_t strides[1] = {(cuuint64_t)ldc * (out16 ? 2 : 4)};
+    const CUtensorMapDataType dt = out16 == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                   : out16 == GEMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
     cuuint32_t box[2] = {32, 32};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+    CUresult r = fn(tm, dt, 2, const_cast<float*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
@@ -383,13 +394,13 @@ uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n) {
     return d;
 }
 
-template <int BN, bool A_MN, bool B_MN, bool CONV>
+template <int BN, bool A_MN, bool B_MN, bool CONV, bool OUT16>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
                              const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
     static bool attr_set[64] = {};
-    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV>;
+    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV, OUT16>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
@@ -415,7 +426,7 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN), a.status, conv_tma_params(a.conv));
+                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN), a.status, conv_tma_params(a.conv), a.out16);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
@@ -436,16 +447,18 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
     // the result goes out through TMA tile stores when C is 16-byte addressable and this is not a split-k pass
     CUtensorMap tmC = tmA;
     int store_via_tma = 0;
-    if (ks.splits == 1 && (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 && a.ldc % 4 == 0 &&
-        a.ldc * 4 < (1LL << 40))
-        store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc) ? 1 : 0;
+    if (ks.splits == 1 && c_tma_addressable(a.C, a.m, a.ldc, a.out16))
+        store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc, a.out16) ? 1 : 0;
     if (ks.splits > 1 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && a.m % 4 == 0 &&
         a.m * a.n * 4 < (1LL << 40))
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
     switch (tile_n) {
-        case 256: return launch_tc<256, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        case 128: return launch_tc<128, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        default:  return launch_tc<64, A_MN, B_MN, CONV>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, CONV, true>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
+                                  : launch_tc<256, A_MN, B_MN, CONV, false>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, CONV, true>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
+                                  : launch_tc<128, A_MN, B_MN, CONV, false>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, CONV, true>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
+                                  : launch_tc<64, A_MN, B_MN, CONV, false>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
     }
 }
 

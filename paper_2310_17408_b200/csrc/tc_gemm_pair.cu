@@ -73,12 +73,13 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t mask) {
 }
 
 // CONV: op(B) is the lowered activation matrix of a convolution layer, fetched in im2col mode (see tc_gemm.cu)
-template <bool A_MN, bool B_MN, bool CONV>
+template <bool A_MN, bool B_MN, bool CONV, bool OUT16>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k,
                     float alpha, float beta, float* __restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int splits,
-                    int64_t kchunk, float* __restrict__ partials, uint32_t idesc, uint32_t* status, const ConvTma conv) {
+                    int64_t kchunk, float* __restrict__ partials, uint32_t idesc, uint32_t* status, const ConvTma conv,
+                    int out16) {
     constexpr int STAGES = PAIR_STAGES, NACC = PAIR_NACC, BN = PAIR_BN;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -252,13 +253,23 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const bool raw = splits > 1;
             float* out = raw ? partials + (int64_t)sp * m * n : C;
             const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
-            epilogue_tile<BN, 1>(
-                tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta,
-                out, raw ? m : ldc, raw, via_tma, &tmC, sp, stage, sbuf, [&]() {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(tempty_leader0 + 8u * acc);
-                });
+            auto release = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(tempty_leader0 + 8u * acc);
+            };
+            const uint32_t tacc = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+            bool done = false;
+            if constexpr (OUT16) {
+                if (!raw) {      // 16-bit result: one rounding at the store (split-k partial sums stay fp32)
+                    epilogue_tile16<BN, 1>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, out, ldc,
+                                                store_via_tma == 1, &tmC, stage, sbuf, out16, release);
+                    done = true;
+                }
+            }
+            if (!done)
+                epilogue_tile<BN, 1>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, out, raw ? m : ldc,
+                                          raw, via_tma, &tmC, sp, stage, sbuf, release);
         }
         if (lane == 0) bulk_wait_all();
     }
@@ -274,7 +285,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
 }
 
-template <bool A_MN, bool B_MN, bool CONV>
+template <bool A_MN, bool B_MN, bool CONV, bool OUT16>
 static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg) {
     CUtensorMap tmA, tmB;
     bool ok = A_MN ? make_map(&tmA, a.dtype, a.A, a.m, a.k, a.lda, 64, TBK)
@@ -288,13 +299,13 @@ static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     if (!ok) return cudaErrorInvalidValue;
     CUtensorMap tmC = tmA;
     int store_via_tma = 0;
-    if (ks.splits == 1 && (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 && a.ldc % 4 == 0 && a.ldc * 4 < (1LL << 40))
-        store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc) ? 1 : 0;
+    if (ks.splits == 1 && c_tma_addressable(a.C, a.m, a.ldc, a.out16))
+        store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc, a.out16) ? 1 : 0;
     if (ks.splits > 1 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && a.m % 4 == 0 && a.m * a.n * 4 < (1LL << 40))
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
 
     static bool attr_set[64] = {};
-    auto kern = tc_gemm_pair_kernel<A_MN, B_MN, CONV>;
+    auto kern = tc_gemm_pair_kernel<A_MN, B_MN, CONV, OUT16>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
@@ -325,7 +336,7 @@ static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status, conv_tma_params(a.conv));
+                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status, conv_tma_params(a.conv), a.out16);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
@@ -335,11 +346,14 @@ cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     cfg->vector_a = cfg->vector_b = 1;
     const bool a_mn = !a.ta, b_mn = a.tb;
     if (a.conv != nullptr)
-        return a_mn ? launch_pair<true, false, true>(a, ks, partials, cfg) : launch_pair<false, false, true>(a, ks, partials, cfg);
-    if (a_mn && b_mn) return launch_pair<true, true, false>(a, ks, partials, cfg);
-    if (a_mn && !b_mn) return launch_pair<true, false, false>(a, ks, partials, cfg);
-    if (!a_mn && b_mn) return launch_pair<false, true, false>(a, ks, partials, cfg);
-    return launch_pair<false, false, false>(a, ks, partials, cfg);
+        return a_mn ? (a.out16 ? launch_pair<true, false, true, true>(a, ks, partials, cfg)
+                               : launch_pair<true, false, true, false>(a, ks, partials, cfg))
+                    : (a.out16 ? launch_pair<false, false, true, true>(a, ks, partials, cfg)
+                               : launch_pair<false, false, true, false>(a, ks, partials, cfg));
+    if (a_mn && b_mn) return (a.out16 ? launch_pair<true, true, false, true>(a, ks, partials, cfg) : launch_pair<true, true, false, false>(a, ks, partials, cfg));
+    if (a_mn && !b_mn) return (a.out16 ? launch_pair<true, false, false, true>(a, ks, partials, cfg) : launch_pair<true, false, false, false>(a, ks, partials, cfg));
+    if (!a_mn && b_mn) return (a.out16 ? launch_pair<false, true, false, true>(a, ks, partials, cfg) : launch_pair<false, true, false, false>(a, ks, partials, cfg));
+    return (a.out16 ? launch_pair<false, false, false, true>(a, ks, partials, cfg) : launch_pair<false, false, false, false>(a, ks, partials, cfg));
 }
 
 }  // namespace b200gemm
