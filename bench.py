@@ -42,6 +42,8 @@ WORKLOADS = {
     "cfg5_bf16": lambda: config_problems(5, dtype=DTYPE_BF16),
     "cfg5_f16_squares": lambda: config_problems(5, dtype=DTYPE_F16)[:3],
     "cfg5_bf16_squares": lambda: config_problems(5, dtype=DTYPE_BF16)[:3],
+    # config 5 with the result in the operands' 16-bit type as well (the library's GEMM_BF16_C16)
+    "cfg5_bf16_c16": lambda: config_problems(5, dtype=DTYPE_BF16, c16=True),
     # second workload (VGG16, batch 32) and the paper's own orientation (m = batch*pixels, n = channels)
     "vgg16_fp32": lambda: im2row_problems("vgg16"),
     "vgg16_bf16": lambda: im2row_problems("vgg16", dtype=DTYPE_BF16),
@@ -295,10 +297,10 @@ def run_cuda(args, problems, workload_name):
     for p, (A, B, C0) in zip(problems, operands):
         view = (lambda x: x.view(np.int16)) if p.dtype != DTYPE_F32 else (lambda x: x)
         hA, hB, hC = (torch.from_numpy(view(A.buf)).pin_memory(), torch.from_numpy(view(B.buf)).pin_memory(),
-                      torch.from_numpy(C0.buf).pin_memory())
+                      torch.from_numpy(view(C0.buf) if C0.buf.dtype == np.uint16 else C0.buf).pin_memory())
         host.append((hA, hB, hC, A.ld, B.ld, C0.ld))
         dev.append((hA.cuda(), hB.cuda(), hC.cuda(), hC.cuda()))      # A, B, C0 (pristine), C (working)
-        ws_need = max(ws_need, g.gemm_workspace_bytes(p.dtype, p.transA, p.transB, p.m, p.n, p.k))
+        ws_need = max(ws_need, g.gemm_workspace_bytes(p.api_dtype, p.transA, p.transB, p.m, p.n, p.k))
     ws = torch.empty(max(ws_need, 1 << 20), dtype=torch.uint8, device="cuda")
     assert g.gemm_set_workspace(ws.data_ptr(), ws.numel(), 0) == 0
 
@@ -318,7 +320,7 @@ def run_cuda(args, problems, workload_name):
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-            rc = g.gemm(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), lda, dB.data_ptr(), ldb,
+            rc = g.gemm(p.api_dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), lda, dB.data_ptr(), ldb,
                         p.beta, dC.data_ptr(), ldc, stream)
             if rc != 0:
                 raise RuntimeError(f"gemm failed: {g.gemm_status_string(rc)} (cuda error {g.gemm_last_cuda_error()})")
@@ -362,7 +364,7 @@ def run_cuda(args, problems, workload_name):
     for p in problems:   # what the selector chose (one untimed call each)
         i = problems.index(p)
         dA, dB, dC0, dC = dev[i]
-        g.gemm(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), host[i][3], dB.data_ptr(), host[i][4],
+        g.gemm(p.api_dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), host[i][3], dB.data_ptr(), host[i][4],
                p.beta, dC.data_ptr(), host[i][5], stream)
         configs.append(g.gemm_last_config())
     torch.cuda.synchronize()
@@ -378,7 +380,7 @@ def run_cuda(args, problems, workload_name):
 
         def call(r):
             a, b, c = sets[r % nsets]
-            rc = g.gemm(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, a.data_ptr(), lda, b.data_ptr(), ldb,
+            rc = g.gemm(p.api_dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, a.data_ptr(), lda, b.data_ptr(), ldb,
                         p.beta, c.data_ptr(), ldc, stream)
             if rc != 0:
                 raise RuntimeError(g.gemm_status_string(rc))
@@ -406,7 +408,7 @@ def run_cuda(args, problems, workload_name):
                     with torch.cuda.graph(graph, stream=side):
                         for r in range(reps):
                             a, b, c = sets[r % nsets]
-                            rc = g.gemm(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, a.data_ptr(), lda,
+                            rc = g.gemm(p.api_dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, a.data_ptr(), lda,
                                         b.data_ptr(), ldb, p.beta, c.data_ptr(), ldc, cap)
                             if rc != 0:
                                 raise RuntimeError(g.gemm_status_string(rc))
@@ -435,7 +437,7 @@ def run_cuda(args, problems, workload_name):
         def host_step():
             for i, p in enumerate(problems):
                 hA, hB, hC, lda, ldb, ldc = host[i]
-                rc = g.gemm_host(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, hA.data_ptr(), lda, hB.data_ptr(),
+                rc = g.gemm_host(p.api_dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, hA.data_ptr(), lda, hB.data_ptr(),
                                  ldb, p.beta, hC.data_ptr(), ldc, stream)
                 if rc != 0:
                     raise RuntimeError(f"gemm_host failed: {g.gemm_status_string(rc)}")
@@ -452,8 +454,8 @@ def run_cuda(args, problems, workload_name):
         barrier()
         e2e_s = time.perf_counter() - t0
         h2d = sum(h[0].numel() * h[0].element_size() + h[1].numel() * h[1].element_size() +
-                  (h[2].numel() * 4 if p.beta != 0.0 else 0) for h, p in zip(host, problems))   # C goes in only when beta != 0
-        d2h = sum(h[2].numel() * 4 for h in host)
+                  (h[2].numel() * h[2].element_size() if p.beta != 0.0 else 0) for h, p in zip(host, problems))   # C goes in only when beta != 0
+        d2h = sum(h[2].numel() * h[2].element_size() for h in host)
         e2e = (e2e_s / e2e_steps, h2d, d2h, e2e_steps)
 
     # ---- reduce over ranks (max time), report on rank 0

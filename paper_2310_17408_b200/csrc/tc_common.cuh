@@ -173,7 +173,7 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int64_t row0, i
             tmem_ld_wait();
             if (last_chunk) { release_acc(); released = true; }
             float* r = reinterpret_cast<float*>(v);       // scaled in place
-            if (!raw) {
+            if (!raw && (alpha != 1.0f || need_c0)) {      // alpha == 1, beta == 0: nothing to do (x * 1 is x exactly)
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     r[j] *= alpha;
@@ -206,9 +206,10 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int64_t row0, i
 
 // The same for a 16-bit result (out16 = GEMM_F16 or GEMM_BF16; never for split-k partial sums): `out` and tmC are
 // in that type and alpha*acc + beta*C0 is rounded once, to nearest even, at the store.  Two rows of one column are
-// packed into a 32-bit word before they go to the staging tile: neighbouring lanes swap one value per column pair, so
-// that the even lane holds rows (2i, 2i+1) of column j and the odd lane those of column j+1, and each converts and
-// stores one word (one packed conversion and one shared-memory store per two entries).
+// packed into a 32-bit word before they go to the staging tile: every lane converts its values of a column pair
+// (j, j+1) into one packed word, neighbouring lanes exchange these words, and a byte permute leaves the even lane with
+// rows (2i, 2i+1) of column j and the odd lane with those of column j+1 (per two entries: one packed conversion,
+// one shuffle, one permute, one shared-memory store).
 template <int BN, int STORE_BUFS, typename Release>
 __device__ __forceinline__ void epilogue_tile16(uint32_t tmem_acc, int64_t row0, int64_t n0, int half, int lane,
                                                 int64_t m, int64_t n, float alpha, float beta, float* out, int64_t ldo,
@@ -229,28 +230,33 @@ __device__ __forceinline__ void epilogue_tile16(uint32_t tmem_acc, int64_t row0,
             tmem_ld_wait();
             if (last_chunk) { release_acc(); released = true; }
             float* r = reinterpret_cast<float*>(v);       // scaled in place
+            if (alpha != 1.0f || beta != 0.0f) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                r[j] *= alpha;
-                if (beta != 0.0f && row < m && col0 + j < n) r[j] = fmaf(beta, load_c(out, out16, e0 + j * ldo), r[j]);
+                for (int j = 0; j < 32; ++j) {
+                    r[j] *= alpha;
+                    if (beta != 0.0f && row < m && col0 + j < n) r[j] = fmaf(beta, load_c(out, out16, e0 + j * ldo), r[j]);
+                }
             }
             if (via_tma) {
                 if (lane == 0) bulk_wait_read<STORE_BUFS - 1>();   // the store that last used this staging tile has read it
                 __syncwarp();
                 uint32_t* st32 = reinterpret_cast<uint32_t*>(stage + sbuf * (32 * 32));      // [column][16 row pairs]
+                // own = (column j, column j+1) of this lane's row as one packed word; the partner lane's word holds the
+                // same columns of the neighbouring row; a byte permute picks (row 2i, row 2i+1) of this lane's column
+                const uint32_t pick = odd ? 0x3276u : 0x5410u;
+                uint32_t* dst = st32 + (odd ? 16 : 0) + (lane >> 1);
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    const float got = __shfl_xor_sync(0xFFFFFFFFu, odd ? r[j] : r[j + 1], 1);
-                    const float lo = odd ? got : r[j], hi = odd ? r[j + 1] : got;       // rows 2i, 2i+1 of this lane's column
-                    uint32_t word;
+                    uint32_t own;
                     if (out16 == GEMM_F16) {
-                        const __half2 h = __floats2half2_rn(lo, hi);
-                        word = *reinterpret_cast<const uint32_t*>(&h);
+                        const __half2 h = __floats2half2_rn(r[j], r[j + 1]);
+                        own = *reinterpret_cast<const uint32_t*>(&h);
                     } else {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-                        word = *reinterpret_cast<const uint32_t*>(&h);
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(r[j], r[j + 1]);
+                        own = *reinterpret_cast<const uint32_t*>(&h);
                     }
-                    st32[(j + (odd ? 1 : 0)) * 16 + (lane >> 1)] = word;
+                    const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, own, 1);
+                    dst[j * 16] = __byte_perm(own, got, pick);
                 }
                 fence_async_smem();
                 __syncwarp();

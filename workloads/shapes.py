@@ -109,15 +109,21 @@ class Problem:
     scaleB: float = 1.0
     seed: int = 0
     pad: tuple = field(default=(0, 0, 0))   # extra leading-dimension rows for A, B, C
+    c16: bool = False                       # C in the 16-bit type of A and B (the library's *_C16 data types)
 
     @property
     def flops(self) -> float:
         return 2.0 * self.m * self.n * self.k
 
+    @property
+    def api_dtype(self) -> int:
+        """Data-type code of the library call: dtype, or its all-16-bit form (3 = f16, 4 = bf16) when C is 16-bit."""
+        return self.dtype + 2 if self.c16 else self.dtype
+
     def algorithmic_bytes(self) -> float:
         es = 4 if self.dtype == DTYPE_F32 else 2
         c_passes = 1 + (1 if self.beta != 0.0 else 0)
-        return es * (self.m * self.k + self.k * self.n) + 4.0 * self.m * self.n * c_passes
+        return es * (self.m * self.k + self.k * self.n) + (2.0 if self.c16 else 4.0) * self.m * self.n * c_passes
 
     def stored_dims(self):
         a = (self.m, self.k) if self.transA in "Nn" else (self.k, self.m)
@@ -131,12 +137,12 @@ class Problem:
                         ld=max(1, ar) + self.pad[0], scale=self.scaleA)
         B = make_matrix(br, bc, kind=self.kindB, seed=self.seed, matrix_id=1, dtype=self.dtype,
                         ld=max(1, br) + self.pad[1], scale=self.scaleB)
-        C = make_matrix(self.m, self.n, kind=self.kindC, seed=self.seed, matrix_id=2, dtype=DTYPE_F32,
-                        ld=max(1, self.m) + self.pad[2])
+        C = make_matrix(self.m, self.n, kind=self.kindC, seed=self.seed, matrix_id=2,
+                        dtype=self.dtype if self.c16 else DTYPE_F32, ld=max(1, self.m) + self.pad[2])
         return A, B, C
 
 
-def config_problems(config: int, *, integer: bool = False, dtype: int | None = None) -> list[Problem]:
+def config_problems(config: int, *, integer: bool = False, dtype: int | None = None, c16: bool = False) -> list[Problem]:
     """The problems of workload `config` (1..5).
 
     1: single fp32 512^3, seed 0, alpha=1, beta=0 (integer=True: entries in [-4,4])
@@ -186,6 +192,11 @@ def config_problems(config: int, *, integer: bool = False, dtype: int | None = N
             i += 1
     else:
         raise ValueError("config must be 1..5")
+    if c16:      # the same problems with C in the 16-bit type of the operands (config 5 only)
+        if config != 5:
+            raise ValueError("c16 needs 16-bit operands")
+        import dataclasses
+        probs = [dataclasses.replace(p, name=p.name + "_c16", c16=True) for p in probs]
     return probs
 
 
