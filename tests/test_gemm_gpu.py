@@ -359,3 +359,29 @@ def test_fp32_tail_split_of_the_last_wave():
     C, cfg = run_problem(p, A, B, C0, workspace=False)
     assert cfg["tail_split"] == 0
     check_against_oracle(p, A, B, C0, C)
+
+
+@pytest.mark.parametrize("api_dtype", [DTYPE_F16, DTYPE_BF16, g.GEMM_F16_C16, g.GEMM_BF16_C16, DTYPE_F32])
+def test_nothing_is_written_outside_the_m_by_n_window(api_dtype):
+    """C sits in the middle of a larger buffer filled with a sentinel: the elements before it, the rows m..ldc-1 of
+    every column and everything after column n-1 must keep it.  The shapes end inside a tile in both directions and
+    take the TMA tile stores (columns ending on 16-byte boundaries) as well as the direct stores."""
+    s = torch.cuda.current_stream().cuda_stream
+    in_t = {DTYPE_F32: torch.float32, DTYPE_F16: torch.float16, DTYPE_BF16: torch.bfloat16,
+            g.GEMM_F16_C16: torch.float16, g.GEMM_BF16_C16: torch.bfloat16}[api_dtype]
+    out_t = in_t if api_dtype in (g.GEMM_F16_C16, g.GEMM_BF16_C16) else torch.float32
+    ensure_workspace(64 << 20)
+    for (m, n, k, ldc) in [(136, 257, 64, 136), (136, 257, 64, 144), (130, 300, 64, 136), (264, 70, 48, 272), (8, 1000, 40, 16)]:      # |sums| <= 256: exact in bf16 too
+        A = torch.randint(-2, 3, (k * m,), device="cuda").to(in_t)
+        B = torch.randint(-2, 3, (n * k,), device="cuda").to(in_t)
+        guard = 4096
+        buf = torch.full((guard + ldc * n + guard,), 7.0, device="cuda", dtype=out_t)
+        C = buf[guard:]
+        rc = g.gemm(api_dtype, "N", "N", m, n, k, 1.0, A.data_ptr(), m, B.data_ptr(), k, 0.0, C.data_ptr(), ldc, s)
+        assert rc == 0 and g.gemm_poll_status() == 0
+        host = buf.float().cpu().numpy()
+        body = host[guard:guard + ldc * n].reshape(n, ldc)
+        want = (B.float().reshape(n, k) @ A.float().reshape(k, m)).cpu().numpy()          # small integers: exact
+        assert np.array_equal(body[:, :m], want), (m, n, k, ldc)
+        assert np.all(body[:, m:] == 7.0), "rows m..ldc-1 were written"
+        assert np.all(host[:guard] == 7.0) and np.all(host[guard + ldc * n:] == 7.0), "written outside the buffer of C"
