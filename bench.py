@@ -58,6 +58,9 @@ CONV_WORKLOADS = {
     "resnet50_conv_bf16": lambda: conv_layer_problems("resnet50", dtype=DTYPE_BF16),
     "vgg16_conv_fp32": lambda: conv_layer_problems("vgg16"),
     "vgg16_conv_bf16": lambda: conv_layer_problems("vgg16", dtype=DTYPE_BF16),
+    # the same layers with the result in bf16 as well: a layer's output is the next layer's input type
+    "resnet50_conv_bf16_c16": lambda: conv_layer_problems("resnet50", dtype=DTYPE_BF16, c16=True),
+    "vgg16_conv_bf16_c16": lambda: conv_layer_problems("vgg16", dtype=DTYPE_BF16, c16=True),
 }
 
 
@@ -533,7 +536,7 @@ def run_conv_layers(args, layers, workload_name):
     stream = torch.cuda.current_stream().cuda_stream
     shapes = [g.conv_shape(p.batch, p.h, p.w, p.c_in, p.c_out, p.kh, p.kw, p.stride, p.stride, p.pad, p.pad) for p in layers]
     g.conv2d_force_lowering(g.CONV_LOWERING_EXPLICIT)
-    ws_need = max(g.conv2d_workspace_bytes(p.dtype, s) for p, s in zip(layers, shapes))
+    ws_need = max(g.conv2d_workspace_bytes(p.api_dtype, s) for p, s in zip(layers, shapes))
     g.conv2d_force_lowering(0)
     ws = torch.empty(ws_need + (64 << 20), dtype=torch.uint8, device="cuda")
     assert g.gemm_set_workspace(ws.data_ptr(), ws.numel(), 0) == 0
@@ -549,7 +552,7 @@ def run_conv_layers(args, layers, workload_name):
         nsets = int(min(16, max(1, -(-2 * 126e6 // p.algorithmic_bytes()))))
         dX = [torch.from_numpy(view(X.buf)).cuda() for _ in range(nsets)]
         dW = [torch.from_numpy(view(W.buf)).cuda() for _ in range(nsets)]
-        dY = [torch.from_numpy(Y0.buf).cuda() for _ in range(nsets)]
+        dY = [torch.from_numpy(view(Y0.buf) if Y0.buf.dtype == np.uint16 else Y0.buf).cuda() for _ in range(nsets)]
 
         def timed(call, reps):
             for r in range(3):
@@ -565,7 +568,7 @@ def run_conv_layers(args, layers, workload_name):
 
         def conv_call(r):
             i = r % nsets
-            rc = g.conv2d_im2row(p.dtype, shp, p.alpha, dX[i].data_ptr(), dW[i].data_ptr(), W.ld, p.beta, dY[i].data_ptr(), Y0.ld, stream)
+            rc = g.conv2d_im2row(p.api_dtype, shp, p.alpha, dX[i].data_ptr(), dW[i].data_ptr(), W.ld, p.beta, dY[i].data_ptr(), Y0.ld, stream)
             if rc != 0:
                 raise RuntimeError(f"conv2d_im2row failed on {p.name}: {g.gemm_status_string(rc)}")
 
@@ -583,7 +586,7 @@ def run_conv_layers(args, layers, workload_name):
 
         def gemm_call(r):
             i = r % nsets
-            rc = g.gemm(p.dtype, "N", "N", m, n, k, p.alpha, dW[i].data_ptr(), W.ld, low.data_ptr(), ld, p.beta, dY[i].data_ptr(), Y0.ld, stream)
+            rc = g.gemm(p.api_dtype, "N", "N", m, n, k, p.alpha, dW[i].data_ptr(), W.ld, low.data_ptr(), ld, p.beta, dY[i].data_ptr(), Y0.ld, stream)
             if rc != 0:
                 raise RuntimeError(g.gemm_status_string(rc))
         ms_gemm = timed(gemm_call, reps)

@@ -248,6 +248,11 @@ class ConvProblem:
     kindY: str = "uniform"
     seed: int = 0
     ld_pad: tuple = field(default=(0, 0))     # extra leading-dimension rows for the filter matrix and for Y
+    c16: bool = False                         # result in the 16-bit type of the activations (the library's *_C16 types)
+
+    @property
+    def api_dtype(self) -> int:
+        return self.dtype + 2 if self.c16 else self.dtype
 
     @property
     def out_hw(self):
@@ -269,7 +274,7 @@ class ConvProblem:
         lowering has to move.  The lowered matrix itself (k x pixels) is never counted."""
         es = 4 if self.dtype == DTYPE_F32 else 2
         m, n, k = self.gemm_mnk
-        return es * (self.batch * self.h * self.w * self.c_in + m * k) + 4.0 * m * n * (2 if self.beta != 0.0 else 1)
+        return es * (self.batch * self.h * self.w * self.c_in + m * k) + (2.0 if self.c16 else 4.0) * m * n * (2 if self.beta != 0.0 else 1)
 
     def operands(self) -> tuple[Matrix, Matrix, Matrix]:
         """(X, W, Y0): X as the C_in x (batch*H*W) column-major matrix that an NHWC tensor is, W as C_out x k,
@@ -278,11 +283,13 @@ class ConvProblem:
         scale_w = 1.0 if self.kindW == "int" else (2.0 / k) ** 0.5
         X = make_matrix(self.c_in, self.batch * self.h * self.w, kind=self.kindX, seed=self.seed, matrix_id=1, dtype=self.dtype)
         W = make_matrix(m, k, kind=self.kindW, seed=self.seed, matrix_id=0, dtype=self.dtype, ld=m + self.ld_pad[0], scale=scale_w)
-        Y0 = make_matrix(m, n, kind=self.kindY, seed=self.seed, matrix_id=2, dtype=DTYPE_F32, ld=m + self.ld_pad[1])
+        Y0 = make_matrix(m, n, kind=self.kindY, seed=self.seed, matrix_id=2, dtype=self.dtype if self.c16 else DTYPE_F32,
+                         ld=m + self.ld_pad[1])
         return X, W, Y0
 
 
-def conv_layer_problems(network: str = "resnet50", *, batch: int = 32, dtype: int = DTYPE_F32, integer: bool = False) -> list[ConvProblem]:
+def conv_layer_problems(network: str = "resnet50", *, batch: int = 32, dtype: int = DTYPE_F32, integer: bool = False,
+                        c16: bool = False) -> list[ConvProblem]:
     """The convolution layers behind the rows of Tables "resnet50" / "vgg16", with the usual geometry of those
     networks: 7 x 7 stride 2 pad 3 on a 224 x 224 image for the ResNet stem, 3 x 3 stride 1 pad 1 and 1 x 1 layers on
     an input of the output's size.  Their lowered GEMM dimensions equal im2row_shapes(..., weights_as_A=True).
@@ -297,6 +304,6 @@ def conv_layer_problems(network: str = "resnet50", *, batch: int = 32, dtype: in
             geo = dict(h=2 * L.out_hw, w=2 * L.out_hw, stride=2, pad=3)
         else:
             geo = dict(h=L.out_hw, w=L.out_hw, stride=1, pad=L.ksize // 2)
-        out.append(ConvProblem(f"{tag}_{i + 1:02d}", dtype, batch, c_in=L.cin, c_out=L.cout, kh=L.ksize, kw=L.ksize,
-                               seed=base + i, **geo, **kinds))
+        out.append(ConvProblem(f"{tag}_{i + 1:02d}" + ("_c16" if c16 else ""), dtype, batch, c_in=L.cin, c_out=L.cout,
+                               kh=L.ksize, kw=L.ksize, seed=base + i, c16=c16, **geo, **kinds))
     return out
