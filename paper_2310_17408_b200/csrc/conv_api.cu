@@ -17,18 +17,20 @@ static inline int64_t rup(int64_t a, int64_t b) { return cdiv(a, b) * b; }
 //   MODE 1  one thread per 16-byte chunk of L, gathered element by element and stored whole (any C_in; L aligned);
 //           rows k..ld-1 that fall into a chunk are written as zeros
 //   MODE 2  one thread per element (no alignment at all)
-template <typename T, int MODE>
+// Idx: type of the flat work index (32-bit whenever the element count allows: the index is taken apart by divisions,
+// and 64-bit divisions would cost more than the copy itself)
+template <typename T, int MODE, typename Idx>
 __global__ void __launch_bounds__(256)
 im2row_kernel(const ConvIndex cv, int64_t pixels, int k, const T* __restrict__ X, T* __restrict__ out, int64_t ld) {
     constexpr int PER = MODE == 2 ? 1 : (int)(16 / sizeof(T));      // elements of L written by one thread
     const uint32_t cin = (uint32_t)cv.c_in, kw = (uint32_t)cv.kw;
     const uint32_t per_col = MODE == 1 ? (uint32_t)(ld / PER) : (uint32_t)(k / PER);     // threads per column of L
-    const int64_t total = pixels * per_col;
+    const Idx total = (Idx)pixels * (Idx)per_col;
     const uint32_t hw = (uint32_t)(cv.ho * cv.wo);
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t j = idx / per_col;
-        const uint32_t p0 = (uint32_t)(idx - j * per_col) * PER;     // first row of L this thread writes
-        const uint32_t b = (uint32_t)(j / hw), rem = (uint32_t)(j - (int64_t)b * hw);
+    for (Idx idx = (Idx)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (Idx)gridDim.x * blockDim.x) {
+        const Idx j = idx / (Idx)per_col;
+        const uint32_t p0 = (uint32_t)(idx - j * (Idx)per_col) * PER;     // first row of L this thread writes
+        const uint32_t b = (uint32_t)(j / (Idx)hw), rem = (uint32_t)(j - (Idx)b * (Idx)hw);
         const int oh = (int)(rem / (uint32_t)cv.wo), ow = (int)(rem - (uint32_t)oh * (uint32_t)cv.wo);
         const int h0 = oh * cv.sh - cv.ph, w0 = ow * cv.sw - cv.pw;
         const int64_t base = (((int64_t)b * cv.h + h0) * cv.w + w0) * cv.c_in;
@@ -38,24 +40,27 @@ im2row_kernel(const ConvIndex cv, int64_t pixels, int k, const T* __restrict__ X
             inside = p < (uint32_t)k && (unsigned)(h0 + fr) < (unsigned)cv.h && (unsigned)(w0 + fs) < (unsigned)cv.w;
             return base + ((int64_t)fr * cv.w + fs) * cv.c_in + c;
         };
-        T* dst = out + j * ld + p0;
+        T* dst = out + (int64_t)j * ld + p0;
         if (MODE == 0) {
             bool inside;
             const int64_t src = source(p0, inside);
             *reinterpret_cast<uint4*>(dst) = inside ? __ldg(reinterpret_cast<const uint4*>(X + src)) : make_uint4(0, 0, 0, 0);
         } else if (MODE == 1) {
-            // one division for the chunk's first row, then the (tap, channel) position walks forward element by element
+            // Inside one filter row r the k index runs over (s, c), which is also how the NHWC image row lies in
+            // memory: the source of row p is rowbase(r) + q with q = p - r*kw*C_in, and the horizontal bounds become
+            // a range of q.  One division for the chunk's first row; after that q and r walk forward.
             union { uint4 q; T e[PER]; } v;
-            uint32_t tap = p0 / cin, c = p0 - tap * cin;
-            int fr = (int)(tap / kw), fs = (int)(tap - (uint32_t)fr * kw);
+            const uint32_t seg = kw * cin;                                       // elements per filter row
+            uint32_t fr = p0 / seg, q = p0 - fr * seg;
+            const uint32_t qlo = (uint32_t)max(0, -w0) * cin;
+            const uint32_t qhi = (uint32_t)max(0, min((int)kw, (int)cv.w - w0)) * cin;
+            const int64_t rowstep = cv.w * cv.c_in;
+            int64_t rowbase = base + (int64_t)fr * rowstep;
 #pragma unroll
             for (int i = 0; i < PER; ++i) {
-                const bool inside = p0 + i < (uint32_t)k && (unsigned)(h0 + fr) < (unsigned)cv.h && (unsigned)(w0 + fs) < (unsigned)cv.w;
-                v.e[i] = inside ? __ldg(X + base + ((int64_t)fr * cv.w + fs) * cv.c_in + c) : T(0);
-                if (++c == cin) {
-                    c = 0;
-                    if (++fs == (int)kw) { fs = 0; ++fr; }
-                }
+                const bool inside = p0 + i < (uint32_t)k && (unsigned)(h0 + (int)fr) < (unsigned)cv.h && q >= qlo && q < qhi;
+                v.e[i] = inside ? __ldg(X + rowbase + q) : T(0);
+                if (++q == seg) { q = 0; ++fr; rowbase += rowstep; }
             }
             *reinterpret_cast<uint4*>(dst) = v.q;
         } else {
@@ -79,9 +84,19 @@ static cudaError_t launch_im2row_t(const ConvIndex& cv, int64_t pixels, const vo
     int64_t blocks = cdiv(total, 256);
     const int64_t cap = (int64_t)sm_count() * 32;
     if (blocks > cap) blocks = cap;
-    if (mode == 0) im2row_kernel<T, 0><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (int)k, (const T*)X, (T*)out, ld);
-    else if (mode == 1) im2row_kernel<T, 1><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (int)k, (const T*)X, (T*)out, ld);
-    else im2row_kernel<T, 2><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (int)k, (const T*)X, (T*)out, ld);
+    const bool small = total + blocks * 256 < 0x7FFFFFFFLL && pixels < 0x7FFFFFFFLL;      // flat index and its stride fit 32 bits
+#define IM2ROW_LAUNCH(MODE_, IDX_) \
+    im2row_kernel<T, MODE_, IDX_><<<(unsigned)blocks, 256, 0, s>>>(cv, pixels, (int)k, (const T*)X, (T*)out, ld)
+    if (small) {
+        if (mode == 0) IM2ROW_LAUNCH(0, uint32_t);
+        else if (mode == 1) IM2ROW_LAUNCH(1, uint32_t);
+        else IM2ROW_LAUNCH(2, uint32_t);
+    } else {
+        if (mode == 0) IM2ROW_LAUNCH(0, int64_t);
+        else if (mode == 1) IM2ROW_LAUNCH(1, int64_t);
+        else IM2ROW_LAUNCH(2, int64_t);
+    }
+#undef IM2ROW_LAUNCH
     return cudaGetLastError();
 }
 
