@@ -59,3 +59,18 @@ def test_second_workload_and_paper_orientation():
     assert len(px) == 20 and (px[0].m, px[0].n, px[0].k) == (32 * 112 * 112, 64, 147)
     assert px[0].kindA == "absnormal" and px[0].kindB == "normal" and abs(px[0].scaleB ** 2 - 2 / 147) < 1e-15
     assert len({p.seed for p in v + px}) == 29
+
+
+def test_sixteen_bit_result_variants_of_the_workloads():
+    from workloads import DTYPE_BF16, config_problems, conv_layer_problems
+    plain, c16 = config_problems(5, dtype=DTYPE_BF16), config_problems(5, dtype=DTYPE_BF16, c16=True)
+    assert [p.name + "_c16" for p in plain] == [p.name for p in c16]
+    p, q = plain[5], c16[5]
+    assert (q.api_dtype, p.api_dtype) == (4, 2)                               # the library's GEMM_BF16_C16 / GEMM_BF16
+    assert p.algorithmic_bytes() - q.algorithmic_bytes() == 2 * p.m * p.n     # the result is half as large
+    small = config_problems(5, dtype=DTYPE_BF16, c16=True)[3]
+    A, B, C = type(small)("t", DTYPE_BF16, 8, 6, 4, c16=True).operands()
+    assert C.buf.dtype.itemsize == 2 and A.buf.dtype.itemsize == 2
+    layer = conv_layer_problems("vgg16", dtype=DTYPE_BF16, c16=True)[8]
+    assert layer.api_dtype == 4 and layer.name.endswith("_c16")
+    assert layer.algorithmic_bytes() < conv_layer_problems("vgg16", dtype=DTYPE_BF16)[8].algorithmic_bytes()
