@@ -205,7 +205,8 @@ int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void*
 
     if (m == 0 || n == 0 || alpha == 0.0f || lowering_is_identity(cv)) {
         // nothing to lower: scaling-only cases and 1 x 1 layers, whose lowered matrix is the NHWC tensor itself
-        const int rc = gemm(dtype, 'N', 'N', m, n, k, alpha, W, ldw, X, cv.c_in, beta, Y, ldy, stream);
+        // (in the scaling-only cases the operands are not read; the leading dimension only has to be a legal one)
+        const int rc = gemm(dtype, 'N', 'N', m, n, k, alpha, W, ldw, X, lowering_is_identity(cv) ? cv.c_in : k, beta, Y, ldy, stream);
         if (rc == GEMM_OK) note_lowering(CONV_LOWERING_IDENTITY);
         return rc;
     }

@@ -191,6 +191,18 @@ def test_sixteen_bit_layer_without_workspace_reports_it():
     assert np.array_equal(dY.cpu().numpy().view(np.uint32), Y0.buf.view(np.uint32))       # nothing written
 
 
+def test_scaling_only_layer_call():
+    # alpha == 0: Y <- beta*Y, activations and filters are not read (and may be null)
+    p = make(SMALL[4], DTYPE_F32, alpha=0.0, beta=0.5, ld_pad=(0, 4))
+    X, W, Y0 = p.operands()
+    dY = to_device(Y0)
+    rc = g.conv2d_im2row(p.dtype, shape_of(p), 0.0, 0, 0, W.ld, 0.5, dY.data_ptr(), Y0.ld, 0)
+    assert rc == 0 and g.gemm_poll_status() == 0
+    from workloads import Matrix
+    Y = Matrix(dY.cpu().numpy(), Y0.rows, Y0.cols, Y0.ld, DTYPE_F32)
+    assert Y.padding_intact() and np.array_equal(Y.window(), 0.5 * Y0.window())
+
+
 def test_invalid_arguments():
     s = g.conv_shape(1, 4, 4, 4, 4, 5, 5, 1, 1, 0, 0)              # filter larger than the padded image
     assert g.conv2d_im2row(DTYPE_F32, s, 1.0, 16, 16, 4, 0.0, 16, 4, 0) == -2

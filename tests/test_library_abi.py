@@ -47,6 +47,10 @@ def test_convolution_argument_checks_run_without_a_device():
     assert g.conv2d_im2row(0, s, 1.0, 16, 16, 5, 0.0, 16, 6) == -6
     assert g.im2row(0, s, 16, 16, 35) == -5                         # ld < k = 36
     assert g.conv2d_force_lowering(7) == -1 and g.conv2d_force_lowering(0) == 0
+    # nothing to compute: an empty batch or no output channels succeed without touching anything
+    assert g.conv2d_im2row(0, g.conv_shape(0, 8, 8, 4, 6, 3, 3, 1, 1, 1, 1), 1.0, 0, 16, 6, 0.0, 0, 6) == 0
+    assert g.conv2d_im2row(2, g.conv_shape(2, 8, 8, 4, 0, 3, 3, 1, 1, 1, 1), 1.0, 16, 0, 1, 0.0, 0, 1) == 0
+    assert g.im2row(0, g.conv_shape(0, 8, 8, 4, 6, 3, 3, 1, 1, 1, 1), 0, 0, 36) == 0
     # a layer whose lowered matrix must be written asks for room for it: k = 27 padded to 32 rows, 2 bytes each
     s = g.conv_shape(4, 32, 32, 3, 64, 3, 3, 1, 1, 1, 1)
     assert g.conv2d_workspace_bytes(2, s) >= 32 * 4 * 32 * 32 * 2
