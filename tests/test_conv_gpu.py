@@ -191,6 +191,33 @@ def test_sixteen_bit_layer_without_workspace_reports_it():
     assert np.array_equal(dY.cpu().numpy().view(np.uint32), Y0.buf.view(np.uint32))       # nothing written
 
 
+@pytest.mark.parametrize("dtype", [DTYPE_F32, DTYPE_BF16])
+def test_activations_off_a_sixteen_byte_boundary(dtype):
+    # X one element past an aligned address: no 128-bit loads, no TMA; with and without room for the lowered matrix
+    gm = (2, 11, 9, 64, 48, 3, 3, 1, 1)
+    p = make(gm, dtype, kind="int", alpha=1.0, beta=1.0)
+    X, W, Y0 = p.operands()
+    dX = to_device(X)
+    shifted = torch.empty(dX.numel() + 1, dtype=dX.dtype, device="cuda")
+    shifted[1:] = dX
+    es = 4 if dtype == DTYPE_F32 else 2
+    from workloads import Matrix
+    for room in (True, False):
+        if room:
+            ensure_workspace(64 << 20)
+        else:
+            drop_workspace()
+        dW, dY = to_device(W), to_device(Y0)
+        rc = g.conv2d_im2row(dtype, shape_of(p), 1.0, shifted.data_ptr() + es, dW.data_ptr(), W.ld, 1.0, dY.data_ptr(), Y0.ld, 0)
+        if dtype == DTYPE_BF16 and not room:
+            assert rc == g.GEMM_ERR_WORKSPACE          # a 16-bit layer that TMA cannot lower needs the workspace
+            continue
+        assert rc == 0 and g.gemm_poll_status() == 0
+        want = g.CONV_LOWERING_EXPLICIT if room else g.CONV_LOWERING_FUSED
+        assert g.gemm_last_config()["lowering"] == want
+        check(p, X, W, Y0, Matrix(dY.cpu().numpy(), Y0.rows, Y0.cols, Y0.ld, DTYPE_F32), integer=True)
+
+
 def test_scaling_only_layer_call():
     # alpha == 0: Y <- beta*Y, activations and filters are not read (and may be null)
     p = make(SMALL[4], DTYPE_F32, alpha=0.0, beta=0.5, ld_pad=(0, 4))
