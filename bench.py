@@ -276,6 +276,43 @@ def cpu_baseline(problems, operands, budget_s=30.0):
 
 # ------------------------------------------------------------------------------------------ CUDA arm
 
+def run_probes(g, torch, stream, peaks):
+    """The library's own peak-confirmation probes on this device: HBM copy, register-only fp32 FMA loops and
+    tcgen05.mma on shared-memory-resident operands.  Each is run a few times; best and median are reported."""
+    out = {}
+
+    def series(call, reps=5):
+        vals = []
+        for _ in range(reps):
+            rc, rate, ms = call()
+            if rc != 0:
+                raise RuntimeError(f"probe failed: {g.gemm_status_string(rc)}")
+            vals.append(rate)
+        return {"best": max(vals), "median": statistics.median(vals)}
+
+    nbytes = 1 << 30
+    src = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    dst = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    src.zero_()
+    out["hbm_copy_gbs"] = series(lambda: g.gemm_probe_copy(dst.data_ptr(), src.data_ptr(), nbytes, stream))
+    del src, dst
+    out["fp32_ffma_tflops"] = {
+        "independent_chains": series(lambda: g.gemm_probe_ffma(0, 4096, stream)),
+        "block_8x8": series(lambda: g.gemm_probe_ffma(1, 4096, stream)),
+        "block_8x8_packed_f32x2": series(lambda: g.gemm_probe_ffma(2, 4096, stream)),
+    }
+    out["tensor_umma_tflops"] = {
+        "bf16_128x256x16": series(lambda: g.gemm_probe_umma(DTYPE_BF16, 0, 60000, stream)),
+        "bf16_pair_256x256x16": series(lambda: g.gemm_probe_umma(DTYPE_BF16, 1, 60000, stream)),
+        "f16_pair_256x256x16": series(lambda: g.gemm_probe_umma(DTYPE_F16, 1, 60000, stream)),
+    }
+    if g.gemm_poll_status() != 0:
+        raise RuntimeError(f"device status {hex(g.gemm_status_detail())} after the probes")
+    out["note"] = ("measured by this library's probe kernels in this run (5 runs each); the roofline fractions divide by "
+                   f"the {peaks['source']} peaks, 'frac_of_probe' by these")
+    return out
+
+
 def run_cuda(args, problems, workload_name):
     import torch
     import paper_2310_17408_b200 as g
@@ -288,11 +325,58 @@ def run_cuda(args, problems, workload_name):
     peaks = load_peaks()
     stream = torch.cuda.current_stream().cuda_stream
 
-    # operands: generated on the host (seeded); the CPU baseline runs first (rank 0, N = 1 only), before the GPU is busy
-    operands = [p.operands() for p in problems]
+    # the CPU baseline runs first (rank 0, N = 1 only), before the GPU is busy
     base = None
+    operands = [p.operands(need_c0=p.beta != 0.0) for p in problems]
     if world == 1 and not args.no_cpu_baseline:
         base = cpu_baseline(problems, operands, args.cpu_budget)
+    probes = None
+    if not args.no_probes:
+        probes = run_probes(g, torch, stream, peaks)
+        peaks["probes"] = probes
+    ctx = dict(torch=torch, g=g, rank=rank, world=world, local_rank=local_rank, peaks=peaks, stream=stream, args=args)
+    main = measure_workload(ctx, problems, operands, workload_name)
+    del operands
+    tensor = None
+    if args.tensor_leg and workload_name == "cfg2_fp32_squares":
+        # the tensor-core half of the metric in the same run: config 5's squares in both 16-bit input types
+        tprobs = WORKLOADS["cfg5_bf16_squares"]() + WORKLOADS["cfg5_f16_squares"]()
+        if args.only_tensor:
+            names = set(args.only_tensor.split(","))
+            tprobs = [p for p in tprobs if p.name in names]
+        tops = [p.operands(need_c0=False) for p in tprobs]
+        tensor = measure_workload(ctx, tprobs, tops, "cfg5_bf16_squares+cfg5_f16_squares", e2e_steps=2,
+                                  steps=max(3, args.steps // 2))
+        del tops
+    if rank == 0:
+        line = main
+        if tensor is not None:
+            tensor["dtype"] = "bf16+f16"
+            line["tensor"] = tensor
+            line["gpu_launches_tensor"] = tensor["gpu_launches"]
+        if probes is not None:
+            line["peaks_confirmed"] = probes
+        if base:
+            line["cpu_baseline"] = base
+        print(json.dumps(line))
+        if args.table:
+            with open(args.table, "w") as f:
+                json.dump(line, f, indent=1)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+def measure_workload(ctx, problems, operands, workload_name, e2e_steps=None, steps=None):
+    """Times one workload (a list of problems with their host operands): `value` with operands resident, per-shape
+    cold-cache numbers, the end-to-end leg through gemm_host, clocks, roofline.  Returns the report dict (on every
+    rank; times are the maximum over ranks)."""
+    torch, g, args = ctx["torch"], ctx["g"], ctx["args"]
+    rank, world, local_rank, peaks, stream = ctx["rank"], ctx["world"], ctx["local_rank"], ctx["peaks"], ctx["stream"]
+    n_steps = steps or args.steps
+    if world > 1:
+        import torch.distributed as dist
 
     # pinned host copies for the end-to-end leg, resident device copies for `value`
     host, dev = [], []
@@ -344,7 +428,7 @@ def run_cuda(args, problems, workload_name):
     barrier()
     wall_begin = time.time()
     t_begin.record()
-    for _ in range(args.steps):
+    for _ in range(n_steps):
         one_step(events)
     t_end.record()
     barrier()
@@ -451,7 +535,7 @@ def run_cuda(args, problems, workload_name):
             h[2].copy_(c0)
         barrier()
         t0 = time.perf_counter()
-        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        e2e_steps = max(1, min(n_steps, e2e_steps or args.e2e_steps))
         for _ in range(e2e_steps):
             host_step()
         barrier()
@@ -462,7 +546,7 @@ def run_cuda(args, problems, workload_name):
         e2e = (e2e_s / e2e_steps, h2d, d2h, e2e_steps)
 
     # ---- reduce over ranks (max time), report on rank 0
-    step_ms = total_ms / args.steps
+    step_ms = total_ms / n_steps
     e2e_ms = e2e[0] * 1e3 if e2e else 0.0
     step_ms, e2e_ms = max_over_ranks([step_ms, e2e_ms], device="cuda")
     flops_step = sum(p.flops for p in problems)
@@ -484,42 +568,48 @@ def run_cuda(args, problems, workload_name):
                        "launches": configs[i]["launches"]})
         if avg > dom_ms:
             dom_ms, dominant = avg, (p, bound, peak, unit, achieved, configs[i])
-    if rank == 0:
-        p, bound, peak, unit, achieved, cfg = dominant
-        kernel_names = {1: "simt_generic_kernel", 2: "simt_fast_kernel", 3: "tc_gemm_kernel", 6: "scale_kernel"}
-        kname = kernel_names.get(cfg["kernel"], "?")
-        if cfg["kernel"] == 3 and cfg["tile_m"] == 256:
-            kname = "tc_gemm_pair_kernel"          # 256 x 256 tiles on CTA pairs
-        roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": recorded_traffic(kname, p),
-                "kernel": kname, "problem": p.name,
-                "peak_source": (f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz (max SM clock)"
-                                if bound == "alu" else f"{peaks['source']} ({'MEASURED_PEAKS.json' if peaks['source'] == 'measured' else 'recipe fallback'})")}
-        if bound == "alu" and clocks.get("sm_mhz"):
-            roof["frac_at_sampled_clock"] = achieved / fp32_alu_peak_tflops(clocks["sm_mhz"])
-        line = {"metric": "gemm_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": DTYPE_NAMES[problems[0].dtype], "data": "synthetic",
-                "config": {"workload": workload_name, "problems": [f"{q.m}x{q.n}x{q.k}" for q in problems],
-                           "alpha": problems[0].alpha, "beta": problems[0].beta, "layout": "column-major N,N",
-                           "l2": "inputs larger than L2: one step touches more than 126 MB of operands"
-                                 if sum(q.algorithmic_bytes() for q in problems) > 126e6 else
-                                 "working set smaller than L2 (warm-cache number)",
-                           "parallelism": "replicas only" if world > 1 else "single GPU"},
-                "roofline": roof, "clocks": clocks, "gpu_launches": timed_launches, "shapes": shapes}
-        if e2e:
-            line["e2e"] = {"value": aggregate_throughput(flops_step, e2e_ms, world), "unit": "TFLOP/s",
-                           "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3],
-                           "api": "gemm_host (pinned host buffers, copies inside the timed region)"}
-        if base:
-            line["cpu_baseline"] = base
-        print(json.dumps(line))
-        if args.table:
-            with open(args.table, "w") as f:
-                json.dump(line, f, indent=1)
-    if world > 1:
-        dist.destroy_process_group()
-    return 0
+    p, bound, peak, unit, achieved, cfg = dominant
+    kernel_names = {1: "simt_generic_kernel", 2: "simt_fast_kernel", 3: "tc_gemm_kernel", 6: "scale_kernel"}
+    kname = kernel_names.get(cfg["kernel"], "?")
+    if cfg["kernel"] == 3 and cfg["tile_m"] == 256:
+        kname = "tc_gemm_pair_kernel"          # 256 x 256 tiles on CTA pairs
+    roof = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+            "traffic": recorded_traffic(kname, p),
+            "kernel": kname, "problem": p.name,
+            "peak_source": (f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz (max SM clock)"
+                            if bound == "alu" else f"{peaks['source']} ({'MEASURED_PEAKS.json' if peaks['source'] == 'measured' else 'recipe fallback'})")}
+    if bound == "alu" and clocks.get("sm_mhz"):
+        roof["frac_at_sampled_clock"] = achieved / fp32_alu_peak_tflops(clocks["sm_mhz"])
+    if bound == "tensor":
+        # a kernel timed inside a step that runs for a long time sits at the power-capped clock: the sustained figure
+        roof["peak_sustained"] = peaks["tensor_tflops_sustained"]
+        roof["frac_of_sustained"] = achieved / peaks["tensor_tflops_sustained"]
+        roof["frac_of_nominal_2250"] = achieved / 2250.0
+    probes = peaks.get("probes")
+    if probes:      # the same achieved rate against what this library's own probe kernels reached in this run
+        own = {"alu": probes["fp32_ffma_tflops"]["independent_chains"]["best"],
+               "tensor": probes["tensor_umma_tflops"]["bf16_pair_256x256x16"]["best"],
+               "hbm": probes["hbm_copy_gbs"]["best"]}[bound]
+        roof["peak_probe"] = own
+        roof["frac_of_probe"] = achieved / own if own else None
+    line = {"metric": "gemm_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": n_steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": DTYPE_NAMES[problems[0].dtype], "data": "synthetic",
+            "config": {"workload": workload_name, "problems": [f"{q.m}x{q.n}x{q.k}" for q in problems],
+                       "alpha": problems[0].alpha, "beta": problems[0].beta, "layout": "column-major N,N",
+                       "l2": "inputs larger than L2: one step touches more than 126 MB of operands"
+                             if sum(q.algorithmic_bytes() for q in problems) > 126e6 else
+                             "working set smaller than L2 (warm-cache number)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "roofline": roof, "clocks": clocks, "gpu_launches": timed_launches, "shapes": shapes}
+    if e2e:
+        line["e2e"] = {"value": aggregate_throughput(flops_step, e2e_ms, world), "unit": "TFLOP/s",
+                       "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3],
+                       "api": "gemm_host (pinned host buffers, copies inside the timed region)"}
+    g.gemm_set_workspace(0, 0, 0)
+    del dev, host, ws
+    torch.cuda.empty_cache()
+    return line
 
 
 # ------------------------------------------------------------------------------------------ convolution layers
@@ -639,6 +729,10 @@ def main():
     ap.add_argument("--table", default=None, help="also write the JSON (indented, with per-shape rows) to this file")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-probes", action="store_true", help="skip the peak-confirmation probes")
+    ap.add_argument("--no-tensor-leg", dest="tensor_leg", action="store_false",
+                    help="default workload only: skip config 5's 16-bit squares (the `tensor` key)")
+    ap.add_argument("--only-tensor", default=None, help="comma-separated problem names: members of the tensor leg to keep")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-budget", type=float, default=30.0)
     args = ap.parse_args()

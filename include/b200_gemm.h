@@ -115,9 +115,14 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
  * (the counterpart of the paper's packing buffers Ac / Bc).  Without a workspace, or with one that is
  * too small, gemm() silently picks a configuration that needs none.
  *   gemm_workspace_bytes  bytes the selector would like for this problem (0 = none)
- *   gemm_set_workspace    registers `dev` (>= 256-byte aligned) of `bytes` bytes for the current device;
- *                         dev == NULL unregisters.  One workspace per device: calls that use it must be
- *                         ordered on one stream.  `stream` is unused (reserved) and may be NULL.
+ *   gemm_set_workspace    registers `dev` (>= 256-byte aligned) of `bytes` bytes on the current device for calls
+ *                         made on `stream`; dev == NULL unregisters that entry.  A workspace registered with
+ *                         stream == NULL serves every stream that has no workspace of its own.  The library never
+ *                         frees or reallocates a workspace; it must stay valid while calls that may use it are
+ *                         in flight.
+ * Thread safety: gemm() may be called from several host threads at once.  Calls that share a workspace must be
+ * ordered on one stream (the library does not order them); calls on distinct streams with distinct workspaces,
+ * or that need none, are independent.
  */
 size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k);
 int gemm_set_workspace(void* dev, size_t bytes, void* stream);
@@ -137,13 +142,16 @@ int gemm_set_workspace(void* dev, size_t bytes, void* stream);
  * exits.  The caller passes only inputs and outputs (device pointers, fp32, layout and leading dimensions as
  * for gemm()); split_k in 2..64 is the number of k partitions asked for (fewer are used when k is short).
  *   - split_k * m * n * 4 bytes must fit the array; otherwise GEMM_ERR_TOO_LARGE is returned and nothing runs.
- *   - k >= 1; alpha and beta as for gemm(); C is not read when beta == 0.
+ *   - k >= 1; alpha and beta as for gemm(): C is not read when beta == 0, and alpha == 0 computes C <- beta*C
+ *     without reading A or B (which may then be NULL).
  *   - The first call on each device looks up the array's device address (a symbol query, not an allocation).
  *     Make that first call outside any stream capture.
  *   - All calls share the one array, and it keeps what the previous call left in it.  Nothing has to be cleared:
  *     each call overwrites every partial sum that it later reads.  Two calls that may be on the GPU at the same
  *     time (different streams or host threads) race on the array: order them on one stream.
- * Returns GEMM_OK, -(position of the first invalid argument), GEMM_ERR_TOO_LARGE or GEMM_ERR_LAUNCH.
+ * Returns GEMM_OK, -(position of the first invalid argument of THIS function: 1 = transA ... 14 = split_k;
+ * gemm_status_string() names the positions of gemm() and does not apply), GEMM_ERR_TOO_LARGE, GEMM_ERR_ARCH or
+ * GEMM_ERR_LAUNCH (then gemm_last_cuda_error() has the CUDA error).  gemm_last_config() reports the call.
  */
 #define GEMM_STATIC_SCRATCH_BYTES (8u << 20)
 int gemm_f32_splitk_static(char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha,
@@ -205,7 +213,8 @@ int conv2d_force_lowering(int how);
 int gemm_last_config(gemm_config_t* out);
 
 /* tests / benchmarks: force a kernel family (GEMM_KERNEL_AUTO restores the selector).  A forced family
- * that cannot run the problem (wrong dtype, alignment) falls back to the selector's choice.
+ * that cannot run the problem (wrong dtype, alignment) falls back to the selector's choice.  The forcing
+ * functions (these two and conv2d_force_lowering) act on the calling host thread only.
  * gemm_force_tile: force the tile (0 = auto) and split_k (0 = auto; 1 = no split of any kind) of the chosen family. */
 int gemm_force_kernel(int kernel);
 int gemm_force_tile(int tile_m, int tile_n, int split_k);
@@ -224,6 +233,33 @@ uint32_t gemm_status_detail(void);
 int gemm_selftest_wait_expiry(void* stream);
 const char* gemm_status_string(int code);
 int gemm_last_cuda_error(void);   /* cudaError_t of the last failed launch, 0 if none */
+
+/*
+ * Peak-confirmation probes.  The paper measures its micro-kernels in "solo mode" (Section IV-B: the micro-kernel
+ * called repeatedly on operands that stay in the fastest memory, apart from the GEMM around it).  These are the
+ * counterparts for the three units that bound the kernels of this library; a benchmark calls them on the device
+ * it reports on and quotes the results beside the peaks it divides by.  Each call runs its kernel twice on
+ * `stream` (once to warm up, once between two CUDA events), synchronises, and returns the rate of the timed run.
+ * Run times are bounded by the caps on the iteration counts (at most a few hundred milliseconds).
+ *
+ *   gemm_probe_copy   streams `bytes` (a multiple of 16, at most 64 GiB) from src to dst (device pointers, 16-byte
+ *                     aligned, not overlapping; dst is overwritten).  *gbs = (bytes read + bytes written) / time, GB/s.
+ *   gemm_probe_ffma   register-only fp32 fused multiply-adds on all SMs, no memory traffic.  pattern 0: 16 independent
+ *                     chains per thread, 2048 threads per SM (the issue-rate ceiling); pattern 1: an 8 x 8 block of
+ *                     accumulators updated by outer products, 2 x 256 threads per SM (what a thread of the SIMT
+ *                     GEMM kernel does between shared-memory reads); pattern 2: the same block on packed
+ *                     fma.rn.f32x2.  iters in 1..65536 loop trips of 8 steps each.  *tflops = 2 * FMAs / time.
+ *   gemm_probe_umma   tcgen05.mma (kind::f16, fp32 accumulators in TMEM) on operand tiles that stay in shared memory:
+ *                     one CTA per SM issuing 128 x 256 x 16 MMAs (pair = 0), or one CTA pair per two SMs issuing
+ *                     256 x 256 x 16 MMAs with cta_group::2 (pair = 1); dtype GEMM_F16 or GEMM_BF16; kblocks in
+ *                     1..262144 blocks of four MMAs (k = 64).  *tflops = 2*M*N*K per MMA / time.  Its waits are
+ *                     bounded like all others; an expiry shows in gemm_poll_status().
+ *   ms (may be NULL) receives the duration of the timed run in milliseconds.
+ * Return GEMM_OK, -(position of the first invalid argument), GEMM_ERR_ARCH or GEMM_ERR_LAUNCH.
+ */
+int gemm_probe_copy(void* dst, const void* src, size_t bytes, double* gbs, double* ms, void* stream);
+int gemm_probe_ffma(int pattern, int iters, double* tflops, double* ms, void* stream);
+int gemm_probe_umma(int dtype, int pair, int kblocks, double* tflops, double* ms, void* stream);
 
 #ifdef __cplusplus
 }

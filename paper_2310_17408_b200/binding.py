@@ -21,7 +21,7 @@ EXPORTS = ("gemm", "gemm_host", "gemm_workspace_bytes", "gemm_set_workspace", "g
            "gemm_force_kernel", "gemm_force_tile", "gemm_poll_status", "gemm_status_detail",
            "gemm_status_string", "gemm_last_cuda_error", "gemm_f32_splitk_static",
            "gemm_selftest_wait_expiry", "conv2d_im2row", "im2row", "conv2d_workspace_bytes",
-           "conv2d_force_lowering")
+           "conv2d_force_lowering", "gemm_probe_copy", "gemm_probe_ffma", "gemm_probe_umma")
 CONV_LOWERING_NONE, CONV_LOWERING_FUSED, CONV_LOWERING_EXPLICIT, CONV_LOWERING_IDENTITY = 0, 1, 2, 3
 GEMM_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -85,6 +85,13 @@ def _load() -> ctypes.CDLL:
     lib.conv2d_force_lowering.argtypes = [ci]
     lib.gemm_f32_splitk_static.restype = ci
     lib.gemm_f32_splitk_static.argtypes = [cc, cc, i64, i64, i64, cf, vp, i64, vp, i64, cf, vp, i64, ci, vp]
+    dp = ctypes.POINTER(ctypes.c_double)
+    lib.gemm_probe_copy.restype = ci
+    lib.gemm_probe_copy.argtypes = [vp, vp, ctypes.c_size_t, dp, dp, vp]
+    lib.gemm_probe_ffma.restype = ci
+    lib.gemm_probe_ffma.argtypes = [ci, ci, dp, dp, vp]
+    lib.gemm_probe_umma.restype = ci
+    lib.gemm_probe_umma.argtypes = [ci, ci, ci, dp, dp, vp]
     return lib
 
 
@@ -178,3 +185,24 @@ def conv2d_workspace_bytes(dtype, shape: ConvShape) -> int:
 
 def conv2d_force_lowering(how) -> int:
     return _lib.conv2d_force_lowering(how)
+
+
+def _probe(fn, *args):
+    rate, ms = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = fn(*args[:-1], ctypes.byref(rate), ctypes.byref(ms), args[-1])
+    return rc, rate.value, ms.value
+
+
+def gemm_probe_copy(dst, src, nbytes, stream=0):
+    """(rc, GB/s, ms) of the library's streaming copy between two device buffers."""
+    return _probe(_lib.gemm_probe_copy, dst, src, nbytes, stream)
+
+
+def gemm_probe_ffma(pattern, iters, stream=0):
+    """(rc, TFLOP/s, ms) of the register-only fp32 FMA loops (pattern 0 chains, 1 8x8 block, 2 packed 8x8 block)."""
+    return _probe(_lib.gemm_probe_ffma, pattern, iters, stream)
+
+
+def gemm_probe_umma(dtype, pair, kblocks, stream=0):
+    """(rc, TFLOP/s, ms) of tcgen05.mma on shared-memory-resident operands (pair = 1: CTA pairs, 256-row MMAs)."""
+    return _probe(_lib.gemm_probe_umma, dtype, pair, kblocks, stream)

@@ -6,7 +6,7 @@
 
 namespace b200gemm {
 
-static int g_force_lowering = 0;
+static thread_local int g_force_lowering = 0;     // per host thread, like the other forcing knobs
 
 static inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline int64_t rup(int64_t a, int64_t b) { return cdiv(a, b) * b; }
@@ -216,7 +216,7 @@ int conv2d_im2row(int dtype, const conv_shape_t* shape, float alpha, const void*
     const bool can_fuse = fused_possible(input_dtype(dtype), cv, shape->batch, W, ldw);
     void* ws = nullptr;
     size_t ws_bytes = 0;
-    if (!registered_workspace(&ws, &ws_bytes)) return GEMM_ERR_LAUNCH;
+    if (!registered_workspace(s, &ws, &ws_bytes)) return GEMM_ERR_LAUNCH;
     const int64_t ld = rup(k, 8);
     const size_t l_bytes = (size_t)rup(ld * n * es, 256);
     const bool room = ws != nullptr && ws_bytes >= l_bytes;

@@ -2,8 +2,10 @@
 // fast-path eligibility — the role the paper gives to choosing the (mr, nr) micro-kernel and the cache
 // parameters per problem, Sections I and IV) and dispatch to the kernels.
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include "internal.cuh"
 
@@ -13,23 +15,42 @@ __device__ uint32_t g_device_status;   // written by bounded waits that expire
 
 constexpr int MAX_DEVICES = 64;
 
+// one registered workspace: stream == nullptr is the entry that serves every stream without one of its own
+struct Workspace {
+    cudaStream_t stream;
+    void* ptr;
+    size_t bytes;
+};
+
 struct DeviceState {
     bool init = false;
     bool arch_ok = false;
     int sms = 0;
     uint32_t* status = nullptr;
-    void* ws = nullptr;
-    size_t ws_bytes = 0;
+    std::vector<Workspace> ws;       // guarded by g_mutex
 };
 
 static DeviceState g_dev[MAX_DEVICES];
 static std::mutex g_mutex;
 static thread_local gemm_config_t t_last_cfg = {};
 static thread_local int t_last_cuda_error = 0;
-static int g_force_kernel = GEMM_KERNEL_AUTO;
-static int g_force_tile_m = 0, g_force_tile_n = 0, g_force_split = 0;
-static bool g_no_tail_split = false;   // gemm_force_tile(.., split_k = 1) also switches the tail split off
-static uint32_t g_last_detail = 0;
+// forcing knobs (tests, benchmarks): per host thread, so that a thread that forces a configuration does not change
+// what concurrent callers on other threads get
+static thread_local int g_force_kernel = GEMM_KERNEL_AUTO;
+static thread_local int g_force_tile_m = 0, g_force_tile_n = 0, g_force_split = 0;
+static thread_local bool g_no_tail_split = false;   // gemm_force_tile(.., split_k = 1) also switches the tail split off
+static std::atomic<uint32_t> g_last_detail{0};
+
+// the workspace a call on `stream` may use: the one registered for that stream, else the stream-less one
+static void workspace_for(DeviceState* st, cudaStream_t stream, void** ws, size_t* bytes) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    *ws = nullptr;
+    *bytes = 0;
+    for (const Workspace& w : st->ws)
+        if (w.stream == stream) { *ws = w.ptr; *bytes = w.bytes; return; }
+    for (const Workspace& w : st->ws)
+        if (w.stream == nullptr) { *ws = w.ptr; *bytes = w.bytes; return; }
+}
 
 static DeviceState* device_state() {
     int dev = 0;
@@ -52,6 +73,14 @@ static DeviceState* device_state() {
 int sm_count() {
     DeviceState* s = device_state();
     return (s && s->sms > 0) ? s->sms : 148;
+}
+
+bool device_info(uint32_t** status, bool* arch_ok) {
+    DeviceState* s = device_state();
+    if (!s) return false;
+    *status = s->status;
+    *arch_ok = s->arch_ok;
+    return true;
 }
 
 static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -325,11 +354,7 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
 
     void* ws;
     size_t ws_bytes;
-    {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        ws = st->ws;
-        ws_bytes = st->ws_bytes;
-    }
+    workspace_for(st, a.stream, &ws, &ws_bytes);
     if (ws_skip > 0) {      // the head of the workspace is in use by the caller (a lowered activation matrix)
         if (ws == nullptr || ws_bytes < ws_skip) return GEMM_ERR_WORKSPACE;
         ws = static_cast<uint8_t*>(ws) + ws_skip;
@@ -393,17 +418,16 @@ int dispatch_gemm(const GemmArgs& a, size_t ws_skip) {
     return run_gemm(b, st, ws_skip);
 }
 
-bool registered_workspace(void** ws, size_t* bytes) {
+bool registered_workspace(cudaStream_t stream, void** ws, size_t* bytes) {
     DeviceState* st = device_state();
     if (!st) return false;
-    std::lock_guard<std::mutex> lock(g_mutex);
-    *ws = st->ws;
-    *bytes = st->ws_bytes;
+    workspace_for(st, stream, ws, bytes);
     return true;
 }
 
 void note_lowering(int how) { t_last_cfg.lowering = how; }
 void note_launch_error(cudaError_t e) { t_last_cuda_error = (int)e; }
+void note_config(const gemm_config_t& cfg) { t_last_cfg = cfg; }
 
 }  // namespace b200gemm
 
@@ -600,13 +624,21 @@ size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int6
     return p.kernel < 0 ? 0 : p.ws_total;
 }
 
-int gemm_set_workspace(void* dev, size_t bytes, void* /*stream*/) {
+int gemm_set_workspace(void* dev, size_t bytes, void* stream) {
     DeviceState* st = device_state();
     if (!st) return GEMM_ERR_LAUNCH;
     if (dev != nullptr && (reinterpret_cast<uintptr_t>(dev) & 255) != 0) return -1;
+    cudaStream_t key = static_cast<cudaStream_t>(stream);
     std::lock_guard<std::mutex> lock(g_mutex);
-    st->ws = dev;
-    st->ws_bytes = dev ? bytes : 0;
+    for (size_t i = 0; i < st->ws.size(); ++i)
+        if (st->ws[i].stream == key) {
+            if (dev) { st->ws[i].ptr = dev; st->ws[i].bytes = bytes; }
+            else st->ws.erase(st->ws.begin() + (std::ptrdiff_t)i);
+            return GEMM_OK;
+        }
+    if (dev) {
+        try { st->ws.push_back(Workspace{key, dev, bytes}); } catch (...) { return GEMM_ERR_LAUNCH; }
+    }
     return GEMM_OK;
 }
 
@@ -641,7 +673,7 @@ int gemm_poll_status(void) {
     uint32_t word = 0;
     e = cudaMemcpy(&word, st->status, sizeof(word), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail_launch(e);
-    g_last_detail = word;
+    g_last_detail.store(word);
     if (word != 0) {
         uint32_t zero = 0;
         cudaMemcpy(st->status, &zero, sizeof(zero), cudaMemcpyHostToDevice);
@@ -650,7 +682,7 @@ int gemm_poll_status(void) {
     return GEMM_OK;
 }
 
-uint32_t gemm_status_detail(void) { return g_last_detail; }
+uint32_t gemm_status_detail(void) { return g_last_detail.load(); }
 
 int gemm_selftest_wait_expiry(void* stream) {
     DeviceState* st = device_state();

@@ -54,14 +54,32 @@ extern "C" int gemm_f32_splitk_static(char transA, char transB, int64_t m, int64
     if (n < 0) return -4;
     if (k < 1) return -5;
     const int64_t a_rows = ta ? k : m, b_rows = tb ? n : k;
-    if (A == nullptr || (reinterpret_cast<uintptr_t>(A) & 3)) return -7;
+    const bool needs_ab = m > 0 && n > 0 && alpha != 0.0f;      // alpha == 0: A and B are not read and may be NULL
+    if ((needs_ab && A == nullptr) || (reinterpret_cast<uintptr_t>(A) & 3)) return -7;
     if (lda < (a_rows > 1 ? a_rows : 1)) return -8;
-    if (B == nullptr || (reinterpret_cast<uintptr_t>(B) & 3)) return -9;
+    if ((needs_ab && B == nullptr) || (reinterpret_cast<uintptr_t>(B) & 3)) return -9;
     if (ldb < (b_rows > 1 ? b_rows : 1)) return -10;
     if (m > 0 && n > 0 && (C == nullptr || (reinterpret_cast<uintptr_t>(C) & 3))) return -12;
     if (ldc < (m > 1 ? m : 1)) return -13;
     if (split_k < 2 || split_k > 64) return -14;
     if (m == 0 || n == 0) return GEMM_OK;
+
+    uint32_t* status = nullptr;
+    bool arch_ok = false;
+    if (!device_info(&status, &arch_ok)) return GEMM_ERR_LAUNCH;
+    if (!arch_ok) return GEMM_ERR_ARCH;
+
+    gemm_config_t cfg{};
+    cfg.split_k = 1;
+    if (alpha == 0.0f) {      // as gemm(): C <- beta*C exactly, whatever A and B hold (NaN, Inf) or point to
+        GemmArgs sc{GEMM_F32, ta, tb, m, n, k, alpha, beta, A, B, C, lda, ldb, ldc, static_cast<cudaStream_t>(stream), status};
+        cfg.kernel = GEMM_KERNEL_SCALE_ONLY;
+        cfg.launches = beta == 1.0f ? 0 : 1;
+        const cudaError_t se = beta == 1.0f ? cudaSuccess : launch_scale(sc);
+        note_config(cfg);
+        if (se != cudaSuccess) { note_launch_error(se); return GEMM_ERR_LAUNCH; }
+        return GEMM_OK;
+    }
 
     // k partition in multiples of the kernel's k slice (16); fewer splits than asked for when k is short
     const int64_t quantum = 16;
@@ -73,21 +91,23 @@ extern "C" int gemm_f32_splitk_static(char transA, char transB, int64_t m, int64
     if (need > (unsigned __int128)GEMM_STATIC_SCRATCH_BYTES) return GEMM_ERR_TOO_LARGE;
 
     float* scratch = nullptr;
-    if (scratch_address(&scratch) != cudaSuccess) return GEMM_ERR_LAUNCH;
+    cudaError_t e = scratch_address(&scratch);
+    if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
 
-    GemmArgs a{GEMM_F32, ta, tb, m, n, k, alpha, beta, A, B, C, lda, ldb, ldc, static_cast<cudaStream_t>(stream), nullptr};
-    gemm_config_t cfg{};
-    cudaError_t e;
+    GemmArgs a{GEMM_F32, ta, tb, m, n, k, alpha, beta, A, B, C, lda, ldb, ldc, static_cast<cudaStream_t>(stream), status};
     if (splits > 1) {
         // 64 x 64 CTA tiles: the problems that fit the array have few tiles, and the smallest tile spreads them
         // over the most SMs.  Every entry (split, i < m, j < n) of the scratch is written by this kernel before
         // the reduction reads it, so nothing has to be cleared between calls.
         e = launch_simt_fast(a, /*tile id of 64 x 64*/ 3, KSplit{splits, chunk}, scratch, &cfg);
-        if (e != cudaSuccess) return GEMM_ERR_LAUNCH;
-        e = launch_splitk_reduce(a, splits, scratch);
+        if (e == cudaSuccess) e = launch_splitk_reduce(a, splits, scratch);
+        cfg.launches = 2;
     } else {
         // k no longer than one slice: a single pass with the epilogue fused, no scratch involved
         e = launch_simt_fast(a, 3, KSplit{1, chunk}, nullptr, &cfg);
+        cfg.launches = 1;
     }
-    return e == cudaSuccess ? GEMM_OK : GEMM_ERR_LAUNCH;
+    note_config(cfg);
+    if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
+    return GEMM_OK;
 }

@@ -121,13 +121,16 @@ cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t
 cudaError_t launch_wait_expiry_probe(uint32_t* status, cudaStream_t stream);
 
 int sm_count();
+// status word of the current device and whether it is compute capability 10.x; false if the device cannot be queried
+bool device_info(uint32_t** status, bool* arch_ok);
 
 // runs one GEMM (possibly with an im2row index map in a.conv) through the selector on the current device;
 // the first ws_skip bytes of the registered workspace are left alone
 int dispatch_gemm(const GemmArgs& a, size_t ws_skip);
-bool registered_workspace(void** ws, size_t* bytes);
+bool registered_workspace(cudaStream_t stream, void** ws, size_t* bytes);   // the one a call on `stream` may use
 void note_lowering(int how);             // recorded in the calling thread's last configuration
 void note_launch_error(cudaError_t e);
+void note_config(const gemm_config_t& cfg);   // becomes the calling thread's gemm_last_config()
 // whether TMA's im2col mode can do the lowering of this layer (defined with the tensor kernels)
 bool conv_tma_eligible(int dtype, const ConvIndex& cv, int64_t batch);
 

@@ -1,0 +1,337 @@
+// Peak-confirmation probes: the three rates the GEMM kernels are judged against, measured by this library's own
+// code on the device it runs on.  They are the counterpart of the paper's "solo mode" (Section IV-B: the micro-kernel
+// called on its own, operands resident in the fastest memory), one per unit that bounds a kernel here:
+//   gemm_probe_copy   HBM: a streaming copy (bytes read + bytes written per second)
+//   gemm_probe_ffma   CUDA cores: register-only fp32 FMA loops, as independent chains and in the 8 x 8 outer-product
+//                     register pattern of the SIMT kernel's micro-tile (scalar and packed fma.rn.f32x2 forms)
+//   gemm_probe_umma   tensor cores: tcgen05.mma on operands that stay in shared memory, accumulators in TMEM
+// Every probe has a bounded run time (iteration counts are capped), touches no caller memory except the two
+// buffers handed to the copy probe, and times itself with CUDA events on the caller's stream.
+#include "tc_common.cuh"
+
+namespace b200gemm {
+
+__device__ float g_probe_sink[32];      // results land here only under a condition that never holds
+
+// ---------------------------------------------------------------- HBM copy
+
+__global__ void __launch_bounds__(512)
+probe_copy_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n; i += 4 * stride) {       // four independent 16-byte loads in flight per thread
+        const uint4 a = __ldcs(src + i), b = __ldcs(src + i + stride), c = __ldcs(src + i + 2 * stride),
+                    d = __ldcs(src + i + 3 * stride);
+        __stcs(dst + i, a); __stcs(dst + i + stride, b); __stcs(dst + i + 2 * stride, c); __stcs(dst + i + 3 * stride, d);
+    }
+    for (; i < n; i += stride) __stcs(dst + i, __ldcs(src + i));
+}
+
+// ---------------------------------------------------------------- fp32 FMA, registers only
+
+// 16 independent dependency chains per thread: the issue-rate ceiling of the FMA pipes
+__global__ void __launch_bounds__(256)
+probe_ffma_chains_kernel(int iters, float x, float y) {
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = (float)(threadIdx.x + i);
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = fmaf(acc[i], x, y);
+    }
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s += acc[i];
+    if (s == 1.2345678e-30f) g_probe_sink[threadIdx.x & 31] = s;
+}
+
+// the register pattern of a GEMM thread: an 8 x 8 block of accumulators receives one outer product a (8) x b (8) per
+// step; a and b change every step (here: rotated among registers that the loop keeps alive), as they do when they
+// come from shared memory.  PACKED: two FMAs per fma.rn.f32x2, accumulators held as the diagonal / anti-diagonal
+// pairs of 2 x 2 sub-blocks, the arrangement of the SIMT kernel.
+template <bool PACKED>
+__global__ void __launch_bounds__(256, 2)
+probe_ffma_block_kernel(int iters, float x) {
+    float a[2][8], b[2][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        a[0][i] = x * (float)(threadIdx.x + i); a[1][i] = x * (float)(threadIdx.x + 2 * i + 1);
+        b[0][i] = x * (float)(blockIdx.x + i);  b[1][i] = x * (float)(blockIdx.x + 3 * i + 2);
+    }
+    float s = 0.0f;
+    if (!PACKED) {
+        float acc[8][8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[j][i] = 0.0f;
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(a[u & 1][(i + u) & 7], b[u & 1][(j + u) & 7], acc[j][i]);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) s += acc[j][i];
+    } else {
+        uint64_t P[4][4], Q[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) P[j][i] = Q[j][i] = 0ull;
+        auto pack = [](float lo, float hi) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; };
+        uint64_t ap[2][4], bp[2][4], bs[2][4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                ap[h][i] = pack(a[h][2 * i], a[h][2 * i + 1]);
+                bp[h][i] = pack(b[h][2 * i], b[h][2 * i + 1]);
+                bs[h][i] = pack(b[h][2 * i + 1], b[h][2 * i]);
+            }
+        for (int it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(P[j][i]) : "l"(ap[u & 1][(i + u) & 3]), "l"(bp[u & 1][(j + u) & 3]));
+                        asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(Q[j][i]) : "l"(ap[u & 1][(i + u) & 3]), "l"(bs[u & 1][(j + u) & 3]));
+                    }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float lo, hi;
+                asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(P[j][i]));
+                s += lo + hi;
+                asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(Q[j][i]));
+                s += lo + hi;
+            }
+    }
+    if (s == 1.2345678e-30f) g_probe_sink[threadIdx.x & 31] = s;
+}
+
+// ---------------------------------------------------------------- tcgen05.mma on shared-memory-resident operands
+
+constexpr int PROBE_RING = 6;           // k blocks in flight between issue and completion, as in the GEMM pipelines
+constexpr int PROBE_N = 256;
+constexpr int PROBE_A_BYTES = TBM * TBK * 2;
+
+// One CTA per SM (PAIR: one cluster of two CTAs per SM pair).  The operand tiles (A 128 x 64, B 256 x 64 — PAIR: each
+// CTA half of B's rows — 16-bit, K-major, 128-byte swizzle atoms) are written once by plain stores and then read by
+// every MMA; no TMA, no global memory traffic.  One thread issues k blocks of four 128(256) x 256 x 16 MMAs, commits
+// each block to a ring of mbarriers and waits (bounded) for the block issued PROBE_RING earlier.
+template <bool PAIR>
+__global__ void __launch_bounds__(128, 1)
+probe_umma_kernel(int kblocks, uint32_t idesc, uint32_t* status, int f16) {
+    constexpr int B_BYTES = (PAIR ? PROBE_N / 2 : PROBE_N) * TBK * 2;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + PROBE_A_BYTES + B_BYTES);
+    const uint32_t bar0 = smem_base + PROBE_A_BYTES + B_BYTES;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + PROBE_RING);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool leader = !PAIR || cluster_ctarank() == 0;
+
+    if (threadIdx.x == 0) {
+        for (int r = 0; r < PROBE_RING; ++r) mbar_init(bar0 + 8u * r, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {      // a whole, converged warp allocates tensor memory (warp 0 is busy with the barriers)
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)PROBE_N) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)PROBE_N) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+    }
+    // operand values: a fixed pattern of small finite numbers (any bits that are not NaN / Inf would do; real
+    // values keep the multipliers' switching activity, and with it power and clocks, like a GEMM's)
+    {
+        uint16_t* ops = reinterpret_cast<uint16_t*>(smem_al);
+        for (int i = threadIdx.x; i < (PROBE_A_BYTES + B_BYTES) / 2; i += blockDim.x) {
+            uint32_t h = (uint32_t)i * 2654435761u + blockIdx.x * 40503u;
+            h ^= h >> 15;
+            const float v = (float)((int)(h & 0xFF) - 128) * (1.0f / 256.0f);
+            ops[i] = f16 ? __half_as_ushort(__float2half_rn(v)) : __bfloat16_as_ushort(__float2bfloat16_rn(v));
+        }
+        fence_async_smem();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (PAIR) { __syncwarp(); cluster_sync_all(); }
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0 && lane == 0 && leader) {
+        const uint32_t sa = smem_base, sb = smem_base + PROBE_A_BYTES;
+        bool ok = true;
+        for (int kb = 0; kb < kblocks && ok; ++kb) {
+            const int r = kb % PROBE_RING;
+            if (kb >= PROBE_RING) {
+                ok = mbar_wait(bar0 + 8u * r, (uint32_t)(kb / PROBE_RING - 1) & 1u, abort_flag, status,
+                               STATUS_MARK | (ROLE_SELFTEST << 16) | (BAR_EMPTY << 8) | r);
+                if (!ok) break;
+                tc_fence_after();
+            }
+#pragma unroll
+            for (int kk = 0; kk < TBK / UMMA_K; ++kk) {
+                const uint64_t ad = smem_desc(sa + kk * (UMMA_K * 2), 0, 1024);
+                const uint64_t bd = smem_desc(sb + kk * (UMMA_K * 2), 0, 1024);
+                if (PAIR) umma_f16_pair(tmem_base, ad, bd, idesc, (kb | kk) != 0);
+                else umma_f16(tmem_base, ad, bd, idesc, (kb | kk) != 0);
+            }
+            if (PAIR) umma_commit_pair(bar0 + 8u * r, 1);      // arrives in the leader only
+            else umma_commit(bar0 + 8u * r);
+        }
+        // completion of everything still in flight (each barrier's last use)
+        const int tail = kblocks < PROBE_RING ? kblocks : PROBE_RING;
+        for (int i = 0; i < tail && ok; ++i) {
+            const int kb = kblocks - 1 - i;
+            ok = mbar_wait(bar0 + 8u * (kb % PROBE_RING), (uint32_t)(kb / PROBE_RING) & 1u, abort_flag, status,
+                           STATUS_MARK | (ROLE_SELFTEST << 16) | (BAR_FULL << 8) | (kb % PROBE_RING));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (PAIR) { __syncwarp(); cluster_sync_all(); }     // the peer's shared memory is read by the pair's MMAs until here
+    if (warp == 1) {
+        tc_fence_after();
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)PROBE_N) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)PROBE_N) : "memory");
+    }
+}
+
+// runs `launch` once untimed and once between two events on `s`; returns the timed duration
+template <typename F>
+static cudaError_t timed(cudaStream_t s, F&& launch, double* ms_out) {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    if (e == cudaSuccess) e = launch();
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = cudaEventRecord(e0, s);
+    if (e == cudaSuccess) e = launch();
+    if (e == cudaSuccess) e = cudaEventRecord(e1, s);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    float ms = 0.0f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    *ms_out = (double)ms;
+    return e;
+}
+
+}  // namespace b200gemm
+
+using namespace b200gemm;
+
+extern "C" {
+
+int gemm_probe_copy(void* dst, const void* src, size_t bytes, double* gbs, double* ms, void* stream) {
+    if (dst == nullptr || (reinterpret_cast<uintptr_t>(dst) & 15)) return -1;
+    if (src == nullptr || (reinterpret_cast<uintptr_t>(src) & 15)) return -2;
+    if (bytes < 16 || bytes % 16 != 0 || bytes > ((size_t)64 << 30)) return -3;
+    if (gbs == nullptr) return -4;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n = bytes / 16;
+    const int blocks = sm_count() * 4;
+    double t = 0.0;
+    const cudaError_t e = timed(s, [&]() {
+        probe_copy_kernel<<<blocks, 512, 0, s>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst), n);
+        return cudaGetLastError();
+    }, &t);
+    if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
+    *gbs = t > 0.0 ? 2.0 * (double)bytes / (t * 1e-3) / 1e9 : 0.0;
+    if (ms) *ms = t;
+    return GEMM_OK;
+}
+
+int gemm_probe_ffma(int pattern, int iters, double* tflops, double* ms, void* stream) {
+    if (pattern < 0 || pattern > 2) return -1;
+    if (iters < 1 || iters > (1 << 16)) return -2;
+    if (tflops == nullptr) return -3;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int sms = sm_count();
+    double t = 0.0, flops = 0.0;
+    cudaError_t e;
+    if (pattern == 0) {
+        const int blocks = sms * 8;       // 2048 threads per SM
+        flops = (double)blocks * 256.0 * iters * 8.0 * 16.0 * 2.0;
+        e = timed(s, [&]() { probe_ffma_chains_kernel<<<blocks, 256, 0, s>>>(iters, 0.999f, 0.001f); return cudaGetLastError(); }, &t);
+    } else {
+        const int blocks = sms * 2;       // the SIMT kernel's residency: two 256-thread CTAs per SM
+        flops = (double)blocks * 256.0 * iters * 8.0 * 64.0 * 2.0;
+        e = timed(s, [&]() {
+            if (pattern == 1) probe_ffma_block_kernel<false><<<blocks, 256, 0, s>>>(iters, 1e-3f);
+            else probe_ffma_block_kernel<true><<<blocks, 256, 0, s>>>(iters, 1e-3f);
+            return cudaGetLastError();
+        }, &t);
+    }
+    if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
+    *tflops = t > 0.0 ? flops / (t * 1e-3) / 1e12 : 0.0;
+    if (ms) *ms = t;
+    return GEMM_OK;
+}
+
+int gemm_probe_umma(int dtype, int pair, int kblocks, double* tflops, double* ms, void* stream) {
+    if (dtype != GEMM_F16 && dtype != GEMM_BF16) return -1;
+    if (pair != 0 && pair != 1) return -2;
+    if (kblocks < 1 || kblocks > (1 << 18)) return -3;
+    if (tflops == nullptr) return -4;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t* status = nullptr;
+    bool arch_ok = false;
+    if (!device_info(&status, &arch_ok)) return GEMM_ERR_LAUNCH;
+    if (!arch_ok) return GEMM_ERR_ARCH;
+    const int sms = sm_count();
+    const int smem = PROBE_A_BYTES + (pair ? PROBE_N / 2 : PROBE_N) * TBK * 2 + 1024 + 256;
+    cudaError_t e = pair ? cudaFuncSetAttribute(probe_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                         : cudaFuncSetAttribute(probe_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
+    const int grid = pair ? (sms / 2) * 2 : sms;
+    const int mma_m = pair ? 2 * TBM : TBM;
+    const uint32_t idesc = instr_desc(dtype, false, false, mma_m, PROBE_N);
+    const double flops = (double)(pair ? grid / 2 : grid) * kblocks * 2.0 * mma_m * PROBE_N * TBK;
+    double t = 0.0;
+    e = timed(s, [&]() {
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((unsigned)grid);
+        lc.blockDim = dim3(128);
+        lc.dynamicSmemBytes = smem;
+        lc.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = pair ? 2 : 1;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        cudaError_t le = pair ? cudaLaunchKernelEx(&lc, probe_umma_kernel<true>, kblocks, idesc, status, dtype == GEMM_F16 ? 1 : 0)
+                              : cudaLaunchKernelEx(&lc, probe_umma_kernel<false>, kblocks, idesc, status, dtype == GEMM_F16 ? 1 : 0);
+        return le != cudaSuccess ? le : cudaGetLastError();
+    }, &t);
+    if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }
+    *tflops = t > 0.0 ? flops / (t * 1e-3) / 1e12 : 0.0;
+    if (ms) *ms = t;
+    return GEMM_OK;
+}
+
+}  // extern "C"

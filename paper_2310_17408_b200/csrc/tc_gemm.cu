@@ -13,6 +13,9 @@
 // quarter, alternating 32-column chunks).  Two to four accumulators in TMEM let the epilogue of one tile overlap the
 // main loops of the next ones.
 // Every mbarrier wait is bounded: on expiry the role records a code in the status word and all roles drain.
+#include <atomic>
+#include <mutex>
+
 #include "tc_common.cuh"
 
 namespace b200gemm {
@@ -270,15 +273,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 static EncodeTiledFn encode_fn() {
     static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    static std::once_flag once;           // several host threads may make their first 16-bit call at the same time
+    std::call_once(once, [] {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
             fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+    });
     return fn;
 }
 
@@ -334,15 +336,14 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
 
 static EncodeIm2colFn encode_im2col_fn() {
     static EncodeIm2colFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    static std::once_flag once;
+    std::call_once(once, [] {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
             fn = reinterpret_cast<EncodeIm2colFn>(p);
-    }
+    });
     return fn;
 }
 
@@ -399,14 +400,14 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
                              const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[64];      // zero-initialised; set once per device
     auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV, OUT16>;
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load()) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        if (dev >= 0 && dev < 64) attr_set[dev].store(true);
     }
     const int64_t tiles_m = (a.m + TBM - 1) / TBM, tiles_n = (a.n + BN - 1) / BN;
     if (tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF || tiles_m * tiles_n > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;

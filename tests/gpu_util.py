@@ -107,15 +107,18 @@ def check_large(p: Problem, A: Matrix, B: Matrix, C0: Matrix, C: Matrix, cfg, se
         bound = 4.0 * np.sqrt(n) * tol_entry
         worst = float(np.max(np.abs(resid)))
         assert worst <= bound, f"Freivalds residual {worst:.3e} > {bound:.3e}"
-    # (2) sampled entries, 16 full rows and 16 full columns against exact fp64 dot products
+    # (2) sampled entries, 64 full rows and 64 full columns against exact fp64 dot products (rows and columns longer
+    # than `line_cap` entries are sampled at that many random positions; the cap shrinks with k so that the CPU
+    # work stays near 2^35 multiply-adds)
     rows, cols = sample_positions(m, n, cfg["tile_m"], cfg["tile_n"], rng)
-    fr = rng.integers(0, m, 16)
-    fc = rng.integers(0, n, 16)
-    nrow_samples = min(n, 8192)
+    fr = rng.integers(0, m, 64)
+    fc = rng.integers(0, n, 64)
+    line_cap = int(max(512, min(8192, (1 << 35) // (128 * max(k, 1)))))
+    nrow_samples = min(n, line_cap)
     for i in fr:
         js = rng.choice(n, nrow_samples, replace=False) if n > nrow_samples else np.arange(n)
         rows = np.concatenate([rows, np.full(js.size, i)]); cols = np.concatenate([cols, js])
-    ncol_samples = min(m, 8192)
+    ncol_samples = min(m, line_cap)
     for j in fc:
         is_ = rng.choice(m, ncol_samples, replace=False) if m > ncol_samples else np.arange(m)
         rows = np.concatenate([rows, is_]); cols = np.concatenate([cols, np.full(is_.size, j)])

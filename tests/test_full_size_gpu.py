@@ -63,8 +63,9 @@ def test_config5_half_squares_4096_8192(dtype):
         assert (cfg["tile_m"], cfg["tile_n"]) == (256, 256)      # large squares run on CTA pairs
 
 
-def test_config5_f16_square_16384():
-    p = config_problems(5, dtype=DTYPE_F16)[2]
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+def test_config5_half_square_16384(dtype):
+    p = config_problems(5, dtype=dtype)[2]
     cfg, _ = run_and_check(p)
     assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
     assert (cfg["tile_m"], cfg["tile_n"]) == (256, 256)
@@ -75,6 +76,17 @@ def test_config5_half_im2row_all_layers(dtype):
     for i, p in enumerate(config_problems(5, dtype=dtype)[3:]):
         cfg, _ = run_and_check(p, seed=i)
         assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR, (p.name, cfg)
+
+
+def test_full_size_members_with_alpha_and_beta():
+    # the workloads are timed at alpha = 1, beta = 0; one member of each of configs 3, 4 and 5 is also checked at
+    # full size with alpha = 1.5, beta = 0.5 and a pre-filled C (the epilogue then reads C)
+    import dataclasses
+    cases = [config_problems(3)[2], config_problems(4)[0], config_problems(4)[3],
+             config_problems(5, dtype=DTYPE_BF16)[1], config_problems(5, dtype=DTYPE_F16)[9]]
+    for i, p in enumerate(cases):
+        q = dataclasses.replace(p, name=p.name + "_ab", alpha=1.5, beta=0.5)
+        cfg, _ = run_and_check(q, seed=100 + i)
 
 
 def test_integer_valued_large_shapes_bit_exact_on_samples():

@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2310_17408_b200 as g
 from workloads import DTYPE_BF16, DTYPE_F16, DTYPE_F32, Problem, make_matrix
 
@@ -381,7 +382,12 @@ def test_nothing_is_written_outside_the_m_by_n_window(api_dtype):
         assert rc == 0 and g.gemm_poll_status() == 0
         host = buf.float().cpu().numpy()
         body = host[guard:guard + ldc * n].reshape(n, ldc)
-        want = (B.float().reshape(n, k) @ A.float().reshape(k, m)).cpu().numpy()          # small integers: exact
-        assert np.array_equal(body[:, :m], want), (m, n, k, ldc)
+        # expected values from the CPU oracle's definition layer (small integers: exact in every type involved)
+        in_code = {DTYPE_F32: DTYPE_F32, DTYPE_F16: DTYPE_F16, DTYPE_BF16: DTYPE_BF16,
+                   g.GEMM_F16_C16: DTYPE_F16, g.GEMM_BF16_C16: DTYPE_BF16}[api_dtype]
+        bits = (lambda t: t.cpu().numpy()) if in_code == DTYPE_F32 else (lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16))
+        want = oracle.gemm_l0(in_code, "N", "N", m, n, k, 1.0, bits(A), m, bits(B), k, 0.0,
+                              np.zeros(m * n, dtype=np.float32), m, acc=oracle.ACC_F32)
+        assert np.array_equal(body[:, :m], want.T), (m, n, k, ldc)
         assert np.all(body[:, m:] == 7.0), "rows m..ldc-1 were written"
         assert np.all(host[:guard] == 7.0) and np.all(host[guard + ldc * n:] == 7.0), "written outside the buffer of C"

@@ -10,6 +10,8 @@ No GEMM arithmetic lives here.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass
 
 import numpy as np
@@ -28,6 +30,13 @@ _CHUNK = 1 << 22
 # multiplies them poisons its result, one that writes them is caught by the tests
 CANARY_F32 = np.uint32(0x7FC0DEAD)   # quiet NaN with a payload
 CANARY_16 = np.uint16(0x7FFF)        # NaN in both fp16 and bf16
+
+
+def _gen_threads() -> int:
+    try:
+        return max(1, min(32, len(os.sched_getaffinity(0))))
+    except AttributeError:
+        return max(1, min(32, os.cpu_count() or 1))
 
 
 def _mix(z: np.ndarray) -> np.ndarray:
@@ -179,7 +188,8 @@ def make_matrix(rows: int, cols: int, *, kind: str, seed: int, matrix_id: int,
     if n == 0:
         return Matrix(buf, rows, cols, ld, dtype)
     dense = np.empty(n, dtype=np_dt)
-    for s in range(0, n, _CHUNK):
+
+    def fill(s):      # chunks are independent (counter-based generator): any order, any number of threads
         c = min(_CHUNK, n - s)
         v = _values(kind, seed, matrix_id, s, c, rows, scale)
         if dtype == DTYPE_F32:
@@ -188,5 +198,14 @@ def make_matrix(rows: int, cols: int, *, kind: str, seed: int, matrix_id: int,
             dense[s:s + c] = encode_f16(v)
         else:
             dense[s:s + c] = encode_bf16(v)
+
+    starts = range(0, n, _CHUNK)
+    workers = min(len(starts), _gen_threads())
+    if workers <= 1:
+        for s in starts:
+            fill(s)
+    else:             # numpy releases the interpreter lock inside its array loops
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            list(ex.map(fill, starts))
     view[:, :rows] = dense.reshape(cols, rows)
     return Matrix(buf, rows, cols, ld, dtype)

@@ -130,14 +130,15 @@ class Problem:
         b = (self.k, self.n) if self.transB in "Nn" else (self.n, self.k)
         return a, b
 
-    def operands(self) -> tuple[Matrix, Matrix, Matrix]:
-        """(A, B, C0) as stored matrices; C0 is always fp32."""
+    def operands(self, need_c0: bool = True) -> tuple[Matrix, Matrix, Matrix]:
+        """(A, B, C0) as stored matrices; C0 is fp32 unless c16.  need_c0=False (callers that never read C0, beta = 0)
+        fills C0 with zeros instead of generating it."""
         (ar, ac), (br, bc) = self.stored_dims()
         A = make_matrix(ar, ac, kind=self.kindA, seed=self.seed, matrix_id=0, dtype=self.dtype,
                         ld=max(1, ar) + self.pad[0], scale=self.scaleA)
         B = make_matrix(br, bc, kind=self.kindB, seed=self.seed, matrix_id=1, dtype=self.dtype,
                         ld=max(1, br) + self.pad[1], scale=self.scaleB)
-        C = make_matrix(self.m, self.n, kind=self.kindC, seed=self.seed, matrix_id=2,
+        C = make_matrix(self.m, self.n, kind=self.kindC if need_c0 else "zeros", seed=self.seed, matrix_id=2,
                         dtype=self.dtype if self.c16 else DTYPE_F32, ld=max(1, self.m) + self.pad[2])
         return A, B, C
 
