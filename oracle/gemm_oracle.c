@@ -190,8 +190,9 @@ int oracle_freivalds(int dtype, int ta, int tb, int64_t m, int64_t n, int64_t k,
 /*
  * acc == ACC_F32: C is float* (in: C0, out: result), arithmetic in float (mul then add, no contraction).
  * acc == ACC_F64: C is double* (in: C0 widened by the caller, out: result), arithmetic in double.
- * paper_scaling != 0 applies alpha and beta where Fig. 3 does (Cb = C*beta; Ba = Bc*alpha; Cb += Ac*Ba);
- * otherwise the block contribution is accumulated from zero and folded in as alpha*acc + beta*C.
+ * paper_scaling != 0 places the scalars where Fig. 3 has them (alpha on the packed B panel, beta on the tile of C
+ * the sums start from); otherwise the block contribution is accumulated from zero and folded in as
+ * alpha*acc + beta*C.
  */
 int oracle_gemm_l1(int dtype, int acc, int ta, int tb, int64_t m, int64_t n, int64_t k,
                    double alpha, const void* A, int64_t lda, const void* B, int64_t ldb,
@@ -216,15 +217,25 @@ int oracle_pack_A_f32(int dtype, int ta, const void* A, int64_t lda, int64_t ic,
 }
 int oracle_pack_B_f32(int dtype, int tb, const void* B, int64_t ldb, int64_t pc, int64_t jc,
                       int64_t kcb, int64_t ncb, int nr, float* Bc) {
-    pack_B_f32(dtype, tb, B, ldb, pc, jc, kcb, ncb, nr, Bc);
+    pack_B_f32(dtype, tb, B, ldb, pc, jc, kcb, ncb, nr, Bc, 0, 1.0f);
     return 0;
 }
 
-/* the micro-kernel on its own (Fig. 3 signature; C is the contiguous [NR][MR] block), float */
+/* one full tile through the micro-kernel, with the argument list of Fig. 3 (C is the contiguous [NR][MR]
+ * block), float.  In the paper's placement of the scalars the B panel is scaled the way Pack-B scales it. */
 int oracle_ukernel_f32(int mr, int nr, int64_t kc, float alpha, const float* Ac, const float* Bc,
                        float beta, float* C, int paper_scaling) {
     if (mr > 64 || nr > 64) return -1;
-    ukernel_f32(mr, nr, kc, alpha, Ac, Bc, beta, C, paper_scaling);
+    const float* Bp = Bc;
+    float* scaled = NULL;
+    if (paper_scaling) {
+        scaled = (float*)malloc(sizeof(float) * (size_t)(kc > 0 ? kc : 1) * (size_t)nr);
+        if (!scaled) return -2;
+        for (int64_t e = 0; e < kc * nr; ++e) scaled[e] = Bc[e] * alpha;
+        Bp = scaled;
+    }
+    tile_update_f32(mr, nr, mr, nr, kc, alpha, beta, Ac, Bp, C, mr, paper_scaling);
+    free(scaled);
     return 0;
 }
 
