@@ -714,15 +714,104 @@ def run_conv_layers(args, layers, workload_name):
     return 0
 
 
+# ------------------------------------------------------------------------------------------ strided batches of small problems
+
+BATCHED_WORKLOADS = {
+    # (m, n, k, batch): many small fp32 problems in one call of gemm_strided_batched
+    "batched_fp32_small": [(64, 64, 64, 4096), (32, 32, 32, 16384), (16, 16, 16, 65535), (128, 128, 128, 1024),
+                           (96, 96, 200, 2048), (256, 256, 256, 128)],
+}
+
+
+def run_batched(args, cases, workload_name):
+    """One step = every case once through gemm_strided_batched.  Operands are seeded uniform[-1, 1) values generated on
+    the host for one problem and tiled over the batch with a per-problem sign flip (cheap and still distinct); calls
+    cycle through enough operand sets to exceed L2.  Roofline per case: the slower of 2*m*n*k*batch flops at the fp32
+    ALU peak and 4*(m*k + k*n + m*n)*batch bytes at the HBM peak."""
+    import torch
+    import paper_2310_17408_b200 as g
+    from workloads import make_matrix
+
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream().cuda_stream
+    rows, step_ms, step_flops, launches = [], 0.0, 0.0, 0
+    sampler = ClockSampler(0)
+    sampler.start()
+    wall_begin = time.time()
+    for idx, (m, n, k, batch) in enumerate(cases):
+        A1 = torch.from_numpy(make_matrix(m, k, kind="uniform", seed=7000 + idx, matrix_id=0).buf).cuda()
+        B1 = torch.from_numpy(make_matrix(k, n, kind="uniform", seed=7000 + idx, matrix_id=1).buf).cuda()
+        sign = (1.0 - 2.0 * (torch.arange(batch, device="cuda") % 2)).float()[:, None]
+        bytes_call = 4.0 * (m * k + k * n + m * n) * batch
+        flops = 2.0 * m * n * k * batch
+        nsets = int(min(16, max(1, -(-2 * 126e6 // bytes_call))))
+        sets = [((A1[None, :] * sign).contiguous(), (B1[None, :] * sign).contiguous(), torch.empty(batch * m * n, device="cuda"))
+                for _ in range(nsets)]
+
+        def call(r):
+            a, b, c = sets[r % nsets]
+            rc = g.gemm_strided_batched(DTYPE_F32, "N", "N", m, n, k, 1.0, a.data_ptr(), m, m * k, b.data_ptr(), k, k * n, 0.0,
+                                        c.data_ptr(), m, m * n, batch, stream)
+            if rc != 0:
+                raise RuntimeError(f"gemm_strided_batched failed: {rc}")
+        reps = max(args.steps, 10)
+        for r in range(3):
+            call(r)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for r in range(reps):
+            call(r)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        cfg = g.gemm_last_config()
+        launches += reps * cfg["launches"]
+        t_cmp = flops / (fp32_alu_peak_tflops(peaks["sm_max_mhz"]) * 1e12)
+        t_hbm = bytes_call / (peaks["hbm_gbs"] * 1e9)
+        bound = "alu" if t_cmp >= t_hbm else "hbm"
+        rows.append({"name": f"{m}x{n}x{k}x{batch}", "m": m, "n": n, "k": k, "batch": batch, "ms": ms,
+                     "tflops": flops / (ms * 1e-3) / 1e12, "gbs": bytes_call / (ms * 1e-3) / 1e9, "bound": bound,
+                     "frac": max(t_cmp, t_hbm) / (ms * 1e-3), "kernel": cfg["kernel"], "tile": [cfg["tile_m"], cfg["tile_n"]],
+                     "launches": cfg["launches"], "operand_sets": nsets})
+        step_ms += ms
+        step_flops += flops
+        del sets
+        torch.cuda.empty_cache()
+    clocks = sampler.stop(wall_begin, time.time())
+    if g.gemm_poll_status() != 0:
+        raise RuntimeError(f"device status {hex(g.gemm_status_detail())}")
+    dom = max(rows, key=lambda r: r["ms"])
+    line = {"metric": "gemm_tflops", "value": step_flops / (step_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": 1,
+            "steps": max(args.steps, 10), "warmup": 3, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_name, "api": "gemm_strided_batched", "layout": "column-major N,N, dense strides",
+                       "l2": "calls cycle through operand sets larger than L2", "parallelism": "single GPU"},
+            "roofline": {"bound": dom["bound"], "achieved": dom["tflops"] if dom["bound"] == "alu" else dom["gbs"],
+                         "peak": fp32_alu_peak_tflops(peaks["sm_max_mhz"]) if dom["bound"] == "alu" else peaks["hbm_gbs"],
+                         "unit": "TFLOP/s" if dom["bound"] == "alu" else "GB/s", "frac": dom["frac"], "traffic": None,
+                         "kernel": {2: "simt_batched_kernel", 4: "simt_direct_kernel", 1: "simt_generic_kernel"}.get(dom["kernel"], "?"),
+                         "problem": dom["name"]},
+            "clocks": clocks, "gpu_launches": launches, "shapes": rows}
+    print(json.dumps(line))
+    if args.table:
+        with open(args.table, "w") as f:
+            json.dump(line, f, indent=1)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS) + sorted(CONV_WORKLOADS))
+    ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS) + sorted(CONV_WORKLOADS) + sorted(BATCHED_WORKLOADS))
     ap.add_argument("--shape", default=None, help="M,N,K: time this single problem instead of a workload (alpha=1, beta=0)")
     ap.add_argument("--dtype", default="f32", choices=["f32", "f16", "bf16"], help="operand type for --shape")
+    ap.add_argument("--kind", default=None, choices=["uniform", "normal", "int"],
+                    help="value distribution for --shape (default: uniform for f32, normal for 16-bit inputs; int = integers in [-4, 4])")
     ap.add_argument("--alpha", type=float, default=1.0, help="alpha for --shape")
     ap.add_argument("--beta", type=float, default=0.0, help="beta for --shape")
     ap.add_argument("--only", default=None, help="comma-separated problem names: keep only these members of the workload")
@@ -744,6 +833,8 @@ def main():
         if not kept:
             raise SystemExit(f"--only {args.only}: no such problem in {args.workload} ({', '.join(p.name for p in items)})")
         return kept
+    if args.workload in BATCHED_WORKLOADS:
+        return run_batched(args, BATCHED_WORKLOADS[args.workload], args.workload)
     if args.workload in CONV_WORKLOADS:
         return run_conv_layers(args, keep(CONV_WORKLOADS[args.workload]()), args.workload)
     problems = keep(WORKLOADS[args.workload]())
@@ -751,7 +842,7 @@ def main():
         from workloads import Problem
         m, n, k = (int(t) for t in args.shape.split(","))
         dt = {"f32": DTYPE_F32, "f16": DTYPE_F16, "bf16": DTYPE_BF16}[args.dtype]
-        kind = "uniform" if dt == DTYPE_F32 else "normal"
+        kind = args.kind or ("uniform" if dt == DTYPE_F32 else "normal")
         problems = [Problem(f"{args.dtype}_{m}x{n}x{k}", dt, m, n, k, args.alpha, args.beta, kindA=kind, kindB=kind, seed=0)]
         args.workload = f"single:{args.dtype}:{m}x{n}x{k}"
     if args.impl == "reference":

@@ -50,6 +50,7 @@ enum {
     GEMM_KERNEL_SIMT_GENERIC = 1,  /* any dtype, any alignment: bounds-checked scalar loads, fp32 FMA          */
     GEMM_KERNEL_SIMT_FAST    = 2,  /* fp32: register-blocked 8x8 FFMA micro-tiles, shared-memory double buffer */
     GEMM_KERNEL_TENSOR       = 3,  /* fp16/bf16: TMA -> swizzled shared memory -> tcgen05.mma -> TMEM          */
+    GEMM_KERNEL_SIMT_DIRECT  = 4,  /* fp32, tiny problems: operands straight from global memory to registers   */
     GEMM_KERNEL_SCALE_ONLY   = 6   /* C <- beta*C (alpha == 0 or k == 0)                                        */
 };
 
@@ -96,6 +97,25 @@ typedef struct {
 int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k,
          float alpha, const void* A, int64_t lda, const void* B, int64_t ldb,
          float beta, void* C, int64_t ldc, void* stream);
+
+/*
+ * gemm_strided_batched — `batch` independent problems of one shape in a single call:
+ *        C_b  <-  alpha * op(A_b) * op(B_b) + beta * C_b,     b = 0 .. batch-1,
+ * with X_b = X + b*strideX (strides in elements of the matrix's type; strideA and strideB may be 0 to share an
+ * operand; strideC >= ldc*n so that results do not overlap).  Everything else as for gemm().
+ * This is the small-problem end of the path.  The paper keeps a family of micro-kernels for problems its 8 x 12
+ * kernel fits badly, among them a variant that skips packing altogether (Section III-B "Edge Cases": the
+ * non-packed variant reads A where it lies, because for small problems the packing is not paid back); here
+ * small fp32 problems (and every fp32 gemm() call below the same size) run in a kernel that reads its operands
+ * from global memory straight into registers, without shared-memory staging, workspace or reduction pass, larger
+ * ones share one launch of the register-blocked kernel, small 16-bit problems one launch of the bounds-checked
+ * kernel, and problems large enough to fill the GPU on their own go through gemm() one by one.
+ * Returns GEMM_OK, -(position of the first invalid argument of THIS function; 10, 13, 17 = the strides, 18 = batch)
+ * or a GEMM_ERR_* code.  Asynchronous on `stream`.
+ */
+int gemm_strided_batched(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha,
+                         const void* A, int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB,
+                         float beta, void* C, int64_t ldc, int64_t strideC, int64_t batch, void* stream);
 
 /*
  * gemm_host — the same operation on HOST buffers (pinned memory for full speed; pageable works but serialises).
@@ -218,6 +238,10 @@ int gemm_last_config(gemm_config_t* out);
  * gemm_force_tile: force the tile (0 = auto) and split_k (0 = auto; 1 = no split of any kind) of the chosen family. */
 int gemm_force_kernel(int kernel);
 int gemm_force_tile(int tile_m, int tile_n, int split_k);
+/* how a split of k is finished (fp32): 0 = choose; 1 = partial sums in the workspace and a separate reduction pass;
+ * 2 = inside the main kernel: the CTAs that hold the k ranges of a tile run as one thread-block cluster and sum the
+ * tile through distributed shared memory (at most 8 ranges, no workspace; a wish for more ranges is cut to 8) */
+int gemm_force_reduction(int how);
 
 /*
  * Device status.  Every wait inside the kernels (on an mbarrier) is bounded; a wait that expires
@@ -235,7 +259,7 @@ const char* gemm_status_string(int code);
 int gemm_last_cuda_error(void);   /* cudaError_t of the last failed launch, 0 if none */
 
 /*
- * Peak-confirmation probes.  The paper measures its micro-kernels in "solo mode" (Section IV-B: the micro-kernel
+ * Peak-confirmation probes.  The paper measures its micro-kernels in "solo mode" (Section IV-A: the micro-kernel
  * called repeatedly on operands that stay in the fastest memory, apart from the GEMM around it).  These are the
  * counterparts for the three units that bound the kernels of this library; a benchmark calls them on the device
  * it reports on and quotes the results beside the peaks it divides by.  Each call runs its kernel twice on

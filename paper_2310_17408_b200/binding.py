@@ -15,13 +15,14 @@ GEMM_F32, GEMM_F16, GEMM_BF16, GEMM_F16_C16, GEMM_BF16_C16 = 0, 1, 2, 3, 4
 GEMM_OK = 0
 GEMM_ERR_WORKSPACE, GEMM_ERR_LAUNCH, GEMM_ERR_ARCH, GEMM_ERR_DEVICE, GEMM_ERR_TOO_LARGE = -100, -101, -102, -103, -104
 GEMM_KERNEL_AUTO, GEMM_KERNEL_SIMT_GENERIC, GEMM_KERNEL_SIMT_FAST, GEMM_KERNEL_TENSOR = 0, 1, 2, 3
+GEMM_KERNEL_SIMT_DIRECT = 4
 GEMM_KERNEL_SCALE_ONLY = 6
 
 EXPORTS = ("gemm", "gemm_host", "gemm_workspace_bytes", "gemm_set_workspace", "gemm_last_config",
            "gemm_force_kernel", "gemm_force_tile", "gemm_poll_status", "gemm_status_detail",
            "gemm_status_string", "gemm_last_cuda_error", "gemm_f32_splitk_static",
            "gemm_selftest_wait_expiry", "conv2d_im2row", "im2row", "conv2d_workspace_bytes",
-           "conv2d_force_lowering", "gemm_probe_copy", "gemm_probe_ffma", "gemm_probe_umma")
+           "conv2d_force_lowering", "gemm_strided_batched", "gemm_force_reduction", "gemm_probe_copy", "gemm_probe_ffma", "gemm_probe_umma")
 CONV_LOWERING_NONE, CONV_LOWERING_FUSED, CONV_LOWERING_EXPLICIT, CONV_LOWERING_IDENTITY = 0, 1, 2, 3
 GEMM_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -85,6 +86,10 @@ def _load() -> ctypes.CDLL:
     lib.conv2d_force_lowering.argtypes = [ci]
     lib.gemm_f32_splitk_static.restype = ci
     lib.gemm_f32_splitk_static.argtypes = [cc, cc, i64, i64, i64, cf, vp, i64, vp, i64, cf, vp, i64, ci, vp]
+    lib.gemm_strided_batched.restype = ci
+    lib.gemm_strided_batched.argtypes = [ci, cc, cc, i64, i64, i64, cf, vp, i64, i64, vp, i64, i64, cf, vp, i64, i64, i64, vp]
+    lib.gemm_force_reduction.restype = ci
+    lib.gemm_force_reduction.argtypes = [ci]
     dp = ctypes.POINTER(ctypes.c_double)
     lib.gemm_probe_copy.restype = ci
     lib.gemm_probe_copy.argtypes = [vp, vp, ctypes.c_size_t, dp, dp, vp]
@@ -115,6 +120,16 @@ def gemm(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, st
 
 def gemm_host(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, stream=0) -> int:
     return _lib.gemm_host(dtype, _c(transA), _c(transB), m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, stream)
+
+
+def gemm_strided_batched(dtype, transA, transB, m, n, k, alpha, A, lda, strideA, B, ldb, strideB, beta, C, ldc, strideC,
+                         batch, stream=0) -> int:
+    return _lib.gemm_strided_batched(dtype, _c(transA), _c(transB), m, n, k, alpha, A, lda, strideA, B, ldb, strideB,
+                                     beta, C, ldc, strideC, batch, stream)
+
+
+def gemm_force_reduction(how) -> int:
+    return _lib.gemm_force_reduction(how)
 
 
 def gemm_workspace_bytes(dtype, transA, transB, m, n, k) -> int:

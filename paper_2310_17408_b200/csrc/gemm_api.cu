@@ -14,6 +14,7 @@ namespace b200gemm {
 __device__ uint32_t g_device_status;   // written by bounded waits that expire
 
 constexpr int MAX_DEVICES = 64;
+constexpr int64_t DIRECT_MAX_MN = 256 * 256, DIRECT_MAX_K = 384;
 
 // one registered workspace: stream == nullptr is the entry that serves every stream without one of its own
 struct Workspace {
@@ -39,6 +40,7 @@ static thread_local int t_last_cuda_error = 0;
 static thread_local int g_force_kernel = GEMM_KERNEL_AUTO;
 static thread_local int g_force_tile_m = 0, g_force_tile_n = 0, g_force_split = 0;
 static thread_local bool g_no_tail_split = false;   // gemm_force_tile(.., split_k = 1) also switches the tail split off
+static thread_local int g_force_reduction = 0;      // 0 = choose, 1 = separate reduction pass, 2 = inside the kernel (cluster)
 static std::atomic<uint32_t> g_last_detail{0};
 
 // the workspace a call on `stream` may use: the one registered for that stream, else the stream-less one
@@ -46,10 +48,13 @@ static void workspace_for(DeviceState* st, cudaStream_t stream, void** ws, size_
     std::lock_guard<std::mutex> lock(g_mutex);
     *ws = nullptr;
     *bytes = 0;
-    for (const Workspace& w : st->ws)
-        if (w.stream == stream) { *ws = w.ptr; *bytes = w.bytes; return; }
-    for (const Workspace& w : st->ws)
-        if (w.stream == nullptr) { *ws = w.ptr; *bytes = w.bytes; return; }
+    for (int pass = 0; pass < 2; ++pass)
+        for (const Workspace& w : st->ws)
+            if (w.stream == (pass == 0 ? stream : nullptr)) {
+                *ws = w.ptr;
+                *bytes = w.bytes;
+                return;
+            }
 }
 
 static DeviceState* device_state() {
@@ -97,6 +102,7 @@ struct Plan {
     int64_t lda_p, ldb_p;     // leading dimensions of the repacked operands
     size_t ws_partials;       // bytes
     size_t ws_total;
+    bool cluster_reduce;           // fp32 split-k finished inside the kernel by a thread-block cluster (no workspace)
     int tail_first, tail_splits;   // fp32 tail split (tail_splits <= 1: off)
     int64_t tail_chunk;
 };
@@ -119,6 +125,9 @@ static const int kSimtTileN[4] = {128, 64, 128, 64};
 // fp32: pick the CTA tile that fills the SMs best, then split k when the tile count is far below one wave
 static void plan_simt(const GemmArgs& a, int sms, size_t ws_avail, Plan* p) {
     p->kernel = GEMM_KERNEL_SIMT_FAST;
+    // k worth splitting over CTAs: a cluster sums the ranges inside the kernel, which makes two ranges of 128 pay;
+    // the index-map kernel of the convolution layers has no cluster form and needs the reduction pass
+    const int64_t k_min_split = a.conv ? 512 : 256;
     const double ctas_per_sm[4] = {2, 3, 3, 6};
     const double eff[4] = {1.0, 0.92, 0.92, 0.80};     // relative math efficiency of the smaller tiles
     int best = 0;
@@ -140,7 +149,7 @@ static void plan_simt(const GemmArgs& a, int sms, size_t ws_avail, Plan* p) {
                 full = full - 1.0 + 1.0 / (double)sp;
         }
         double util = waves / full;                                                 // tail effect
-        if (tiles * 2 <= slots && a.k >= 512 && g_force_split <= 1) {
+        if (tiles * 2 <= slots && a.k >= k_min_split && g_force_split <= 1) {
             // fewer tiles than half the slots: k will be split (below), so what counts is how full the machine is then
             const double smax = std::min(64.0, (double)(a.k / 128));
             util = std::min(1.0, tiles * std::max(1.0, std::floor(std::min(smax, slots / tiles))) / slots);
@@ -158,17 +167,25 @@ static void plan_simt(const GemmArgs& a, int sms, size_t ws_avail, Plan* p) {
     const int64_t slots = (int64_t)(sms * ctas_per_sm[best]);
     int want = 1;
     if (g_force_split > 0) want = g_force_split;
-    else if (tiles * 2 <= slots && a.k >= 512) {
+    else if (tiles * 2 <= slots && a.k >= k_min_split) {
         want = (int)(slots / tiles);
         const int64_t max_by_k = a.k / 128;             // keep at least 128 of k per split (measured on 512^3: 2 splits 20.6 us, 4 splits 14.4 us)
         if (want > max_by_k) want = (int)max_by_k;
         if (want > 64) want = 64;
     }
+    if (g_force_reduction == 2 && want > CLUSTER_REDUCE_MAX_SPLITS) want = CLUSTER_REDUCE_MAX_SPLITS;
     p->ks = make_split(a.k, want, 16);
-    p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
+    // Up to 8 k ranges per tile are summed inside the kernel by a thread-block cluster (no workspace).  More ranges,
+    // or the 128 x 128 tile, keep their partial sums in the workspace and a reduction pass follows; without room
+    // for them a wish for more than 8 ranges is cut to 8, which the cluster can do.
+    auto clusterable = [&]() { return p->ks.splits > 1 && p->ks.splits <= CLUSTER_REDUCE_MAX_SPLITS && simt_fast_can_cluster_reduce(best) && !a.conv; };
+    p->cluster_reduce = g_force_reduction != 1 && clusterable();
+    p->ws_partials = (p->ks.splits > 1 && !p->cluster_reduce) ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
     if (p->ws_partials > ws_avail) {
-        if (g_force_split > 0) { p->kernel = -1; return; }
-        p->ks = make_split(a.k, 1, 16);
+        if (g_force_split > 0 && g_force_reduction == 1) { p->kernel = -1; return; }
+        p->ks = make_split(a.k, g_force_reduction == 1 ? 1 : std::min(want, CLUSTER_REDUCE_MAX_SPLITS), 16);
+        p->cluster_reduce = g_force_reduction != 1 && clusterable();
+        if (!p->cluster_reduce) p->ks = make_split(a.k, 1, 16);
         p->ws_partials = 0;
     }
     p->ws_total = p->ws_partials;
@@ -277,12 +294,26 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
     p->ws_total = ws_repack + p->ws_partials;
 }
 
+// Problems this small are a few microseconds of work however they are run; what counts is the length of the
+// longest dependency chain, and the kernel without staging (no shared memory, no barriers, 16 entries of C per
+// thread) has the shortest one.  Thresholds measured on B200 against the staged kernel.
+static bool direct_preferred(int64_t m, int64_t n, int64_t k) {
+    // measured (graph replay, one problem): ahead of the staged kernel up to 256^3 (14 us against 16) and by 1.3-2x
+    // below 128^3; behind once k is long enough for the staged kernel to split it (128 x 128 x 512: 26 us against 10)
+    return (m * n <= 128 * 128 && k <= DIRECT_MAX_K) || (m * n <= DIRECT_MAX_MN && k <= 256);
+}
+
 static Plan make_plan(const GemmArgs& a, int sms, size_t ws_avail) {
     Plan p{};
     p.ks = KSplit{1, a.k > 0 ? a.k : 1};
     int forced = g_force_kernel;
     if (forced == GEMM_KERNEL_SIMT_GENERIC && !a.conv) { p.kernel = GEMM_KERNEL_SIMT_GENERIC; return p; }
     if (a.dtype == GEMM_F32) {
+        if (!a.conv && (forced == GEMM_KERNEL_SIMT_DIRECT || (forced == GEMM_KERNEL_AUTO && direct_preferred(a.m, a.n, a.k) &&
+                                                               g_force_tile_m == 0 && g_force_split == 0))) {
+            p.kernel = GEMM_KERNEL_SIMT_DIRECT;
+            return p;
+        }
         plan_simt(a, sms, ws_avail, &p);
         return p;
     }
@@ -368,6 +399,11 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
         t_last_cfg = cfg;
         return e == cudaSuccess ? GEMM_OK : fail_launch(e);
     }
+    if (p.kernel == GEMM_KERNEL_SIMT_DIRECT) {
+        e = launch_simt_direct(a, 0, 0, 0, 1, &cfg);
+        t_last_cfg = cfg;
+        return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+    }
 
     uint8_t* wsp = static_cast<uint8_t*>(ws);
     if (p.kernel == GEMM_KERNEL_TENSOR) {
@@ -398,9 +434,9 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
         cfg.launches++;
         cfg.tail_split = p.tail_splits;
     } else {
-        e = launch_simt_fast(a, p.tile, p.ks, partials, &cfg);
+        e = launch_simt_fast(a, p.tile, p.ks, partials, &cfg, TailSplit{0x7FFFFFFF, 1, 0, nullptr}, p.cluster_reduce);
     }
-    if (e == cudaSuccess && p.ks.splits > 1) {
+    if (e == cudaSuccess && p.ks.splits > 1 && !p.cluster_reduce) {
         e = launch_splitk_reduce(a, p.ks.splits, partials);
         cfg.launches++;
     }
@@ -453,6 +489,92 @@ int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, f
                static_cast<cudaStream_t>(stream), st->status};
     a.out16 = output16(dtype);
     return run_gemm(a, st);
+}
+
+int gemm_strided_batched(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha, const void* A,
+                         int64_t lda, int64_t strideA, const void* B, int64_t ldb, int64_t strideB, float beta, void* C,
+                         int64_t ldc, int64_t strideC, int64_t batch, void* stream) {
+    bool ta = false, tb = false;
+    // gemm()'s checks, with the positions of this argument list
+    static const int pos[16] = {0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 11, 12, 0, 15, 16, 0};
+    const int bad = validate(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, C, ldc, &ta, &tb);
+    if (bad) return -pos[-bad];
+    if (strideA < 0) return -10;
+    if (strideB < 0) return -13;
+    if (strideC < 0) return -17;
+    if (batch < 0) return -18;
+    if (batch > 1 && m > 0 && n > 0 && strideC < ldc * n) return -17;      // results of different problems would overlap
+    gemm_config_t cfg{};
+    cfg.kernel = GEMM_KERNEL_SCALE_ONLY;
+    cfg.split_k = 1;
+    if (m == 0 || n == 0 || batch == 0) { t_last_cfg = cfg; return GEMM_OK; }
+    DeviceState* st = device_state();
+    if (!st) return GEMM_ERR_LAUNCH;
+    if (!st->arch_ok) return GEMM_ERR_ARCH;
+    GemmArgs a{input_dtype(dtype), ta, tb, m, n, k, alpha, beta, A, B, static_cast<float*>(C), lda, ldb, ldc,
+               static_cast<cudaStream_t>(stream), st->status};
+    a.out16 = output16(dtype);
+    const int es = elem_size(dtype), es_c = c_elem_size(dtype);
+    auto at = [&](int64_t b0) {      // the call's arguments moved to problem b0
+        GemmArgs x = a;
+        if (A) x.A = static_cast<const uint8_t*>(A) + b0 * strideA * es;
+        if (B) x.B = static_cast<const uint8_t*>(B) + b0 * strideB * es;
+        x.C = reinterpret_cast<float*>(static_cast<uint8_t*>(C) + b0 * strideC * es_c);
+        return x;
+    };
+    constexpr int64_t CHUNK = 65535;      // problems per launch (grid limit of the batch dimension)
+    cudaError_t e = cudaSuccess;
+    int launches = 0;
+    if (alpha == 0.0f || k == 0) {
+        if (beta != 1.0f)
+            for (int64_t b0 = 0; b0 < batch && e == cudaSuccess; b0 += CHUNK, ++launches)
+                e = launch_scale(at(b0), strideC, std::min(CHUNK, batch - b0));
+        cfg.launches = launches;
+        t_last_cfg = cfg;
+        return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+    }
+    // one launch covers the whole batch when the problems are small: fp32 through the kernel without staging
+    // (tiny) or the register-blocked kernel with 64 x 64 or 128 x 128 CTA tiles; 16-bit inputs through the
+    // bounds-checked kernel.  Large problems gain nothing from sharing a launch: each goes through gemm().
+    const double work = (double)m * (double)n * (double)k;
+    const int forced = g_force_kernel;
+    if (a.dtype == GEMM_F32 && (work <= 512.0 * 512.0 * 512.0 || forced == GEMM_KERNEL_SIMT_FAST || forced == GEMM_KERNEL_SIMT_DIRECT) &&
+        forced != GEMM_KERNEL_SIMT_GENERIC) {
+        // A few problems: what counts is the length of one problem's dependency chain, as for a single call.  Many
+        // problems: throughput; the kernel without staging tops out near 22 TFLOP/s (every operand element comes
+        // through L1 once per thread that uses it), the staged kernel reaches 40-49, but its smallest tile is 64 x 64,
+        // so problems up to about 48 x 48 are still better off without staging (measured: 32^3 x 16384 71 us against
+        // 149, 64^3 x 4096 107 us against 55).
+        const bool direct = forced == GEMM_KERNEL_SIMT_DIRECT ||
+                            (forced == GEMM_KERNEL_AUTO && (batch <= 4 ? direct_preferred(m, n, k) : m * n <= 48 * 48));
+        auto padded = [&](int64_t t) { return (double)(ceil_div(m, t) * t) * (double)(ceil_div(n, t) * t); };
+        const int64_t tiles128 = ceil_div(m, 128) * ceil_div(n, 128);
+        // 64 x 64 tiles when they waste less of the padded area (their inner loop is ~20 % behind the 128 x 128 one) or when
+        // 128 x 128 tiles would not fill the GPU
+        const int tile = (padded(64) * 1.25 < padded(128) || tiles128 * batch < 2 * (int64_t)st->sms) ? 3 : 0;
+        for (int64_t b0 = 0; b0 < batch && e == cudaSuccess; b0 += CHUNK, ++launches) {
+            const int64_t nb = std::min(CHUNK, batch - b0);
+            e = direct ? launch_simt_direct(at(b0), strideA, strideB, strideC, nb, &cfg)
+                       : launch_simt_fast_batched(at(b0), tile, strideA, strideB, strideC, nb, &cfg);
+        }
+        cfg.launches = launches;
+        t_last_cfg = cfg;
+        return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+    }
+    if (forced == GEMM_KERNEL_SIMT_GENERIC || (a.dtype != GEMM_F32 && work <= 128.0 * 128.0 * 128.0)) {
+        for (int64_t b0 = 0; b0 < batch && e == cudaSuccess; b0 += CHUNK, ++launches)
+            e = launch_simt_generic(at(b0), &cfg, strideA, strideB, strideC, std::min(CHUNK, batch - b0));
+        cfg.launches = launches;
+        t_last_cfg = cfg;
+        return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+    }
+    int rc = GEMM_OK;
+    for (int64_t b0 = 0; b0 < batch && rc == GEMM_OK; ++b0) {
+        rc = run_gemm(at(b0), st);
+        launches += t_last_cfg.launches;
+    }
+    t_last_cfg.launches = launches;
+    return rc;
 }
 
 // copy a rows x cols window of a column-major matrix (element size es, leading dimension ld on both sides)
@@ -629,15 +751,16 @@ int gemm_set_workspace(void* dev, size_t bytes, void* stream) {
     if (!st) return GEMM_ERR_LAUNCH;
     if (dev != nullptr && (reinterpret_cast<uintptr_t>(dev) & 255) != 0) return -1;
     cudaStream_t key = static_cast<cudaStream_t>(stream);
+    Workspace w{key, dev, bytes};
     std::lock_guard<std::mutex> lock(g_mutex);
     for (size_t i = 0; i < st->ws.size(); ++i)
         if (st->ws[i].stream == key) {
-            if (dev) { st->ws[i].ptr = dev; st->ws[i].bytes = bytes; }
+            if (dev) st->ws[i] = w;
             else st->ws.erase(st->ws.begin() + (std::ptrdiff_t)i);
             return GEMM_OK;
         }
     if (dev) {
-        try { st->ws.push_back(Workspace{key, dev, bytes}); } catch (...) { return GEMM_ERR_LAUNCH; }
+        try { st->ws.push_back(w); } catch (...) { return GEMM_ERR_LAUNCH; }
     }
     return GEMM_OK;
 }
@@ -650,7 +773,7 @@ int gemm_last_config(gemm_config_t* out) {
 
 int gemm_force_kernel(int kernel) {
     if (kernel != GEMM_KERNEL_AUTO && kernel != GEMM_KERNEL_SIMT_GENERIC && kernel != GEMM_KERNEL_SIMT_FAST &&
-        kernel != GEMM_KERNEL_TENSOR)
+        kernel != GEMM_KERNEL_TENSOR && kernel != GEMM_KERNEL_SIMT_DIRECT)
         return -1;
     g_force_kernel = kernel;
     return GEMM_OK;
@@ -662,6 +785,12 @@ int gemm_force_tile(int tile_m, int tile_n, int split_k) {
     g_force_tile_n = tile_n;
     g_force_split = split_k;
     g_no_tail_split = (split_k == 1);
+    return GEMM_OK;
+}
+
+int gemm_force_reduction(int how) {
+    if (how < 0 || how > 2) return -1;
+    g_force_reduction = how;
     return GEMM_OK;
 }
 

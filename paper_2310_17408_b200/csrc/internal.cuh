@@ -75,6 +75,20 @@ struct TailSplit {
     float* partials;
 };
 
+// Extras of the fp32 SIMT kernel beyond one plain GEMM.
+//   cluster_reduce  split-k finished inside the kernel: the CTAs that hold the k ranges of one tile are launched as one
+//                   thread-block cluster (gridDim.z = cluster size <= 8).  Each leaves its partial sums in its own
+//                   shared memory; after a cluster barrier every CTA sums one slice of the tile over all CTAs, in
+//                   increasing split index, through distributed shared memory, applies alpha / beta and writes C.
+//                   No workspace, no second launch; the hardware co-schedules a cluster, so the barrier cannot hang.
+//   stride*         strided batch (batched kernel only): blockIdx.y is the problem index
+struct SimtExtra {
+    TailSplit tail;
+    int cluster_reduce;
+    int64_t strideA, strideB, strideC;
+};
+constexpr int CLUSTER_REDUCE_MAX_SPLITS = 8;      // portable cluster size
+
 // Tile order shared by the kernels: groups of `group` tile rows, all tile columns inside a group, rows fastest,
 // so that the CTAs resident at one time share their A and B panels in L2.
 constexpr int SIMT_GROUP = 16;
@@ -90,16 +104,25 @@ __host__ __device__ inline void decode_tile(int tile, int tiles_m, int tiles_n, 
 inline int elem_size(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }      // of A and B
 
 // C <- beta*C  (beta == 0: store +0 without reading)
-cudaError_t launch_scale(const GemmArgs& a);
+cudaError_t launch_scale(const GemmArgs& a, int64_t strideC = 0, int64_t batch = 1);
 
 // generic bounds-checked SIMT kernel, any dtype / trans / alignment
-cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg);
+cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg, int64_t strideA = 0, int64_t strideB = 0,
+                                int64_t strideC = 0, int64_t batch = 1);
+
+// fp32 without operand staging (tiny problems; a strided batch of them): every thread reads its operands from global memory
+cudaError_t launch_simt_direct(const GemmArgs& a, int64_t strideA, int64_t strideB, int64_t strideC, int64_t batch,
+                               gemm_config_t* cfg);
 
 // fast fp32 SIMT kernel.  tile: 0 = 128x128, 1 = 128x64, 2 = 64x128, 3 = 64x64.
 // ks.splits > 1: raw partial sums go to `partials` ([split][n][m], fp32), no epilogue.
 bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb);
+bool simt_fast_can_cluster_reduce(int tile);      // can this CTA tile finish a split of k inside the kernel?
 cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg,
-                             TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr});
+                             TailSplit tail = TailSplit{0x7FFFFFFF, 1, 0, nullptr}, bool cluster_reduce = false);
+// batch problems of identical shape, operands strideA / strideB / strideC elements apart (no split of k)
+cudaError_t launch_simt_fast_batched(const GemmArgs& a, int tile, int64_t strideA, int64_t strideB, int64_t strideC,
+                                     int64_t batch, gemm_config_t* cfg);
 // finishes the tail tiles (bm x bn, tile order with groups of `group` rows):
 // C <- alpha * sum_z slot[(t - first) * splits + z] + beta*C for tiles t >= first
 cudaError_t launch_tail_reduce(const GemmArgs& a, int bm, int bn, int group, TailSplit tail);

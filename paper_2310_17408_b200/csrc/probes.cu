@@ -1,5 +1,5 @@
 // Peak-confirmation probes: the three rates the GEMM kernels are judged against, measured by this library's own
-// code on the device it runs on.  They are the counterpart of the paper's "solo mode" (Section IV-B: the micro-kernel
+// code on the device it runs on.  They are the counterpart of the paper's "solo mode" (Section IV-A: the micro-kernel
 // called on its own, operands resident in the fastest memory), one per unit that bounds a kernel here:
 //   gemm_probe_copy   HBM: a streaming copy (bytes read + bytes written per second)
 //   gemm_probe_ffma   CUDA cores: register-only fp32 FMA loops, as independent chains and in the 8 x 8 outer-product
@@ -15,16 +15,23 @@ __device__ float g_probe_sink[32];      // results land here only under a condit
 
 // ---------------------------------------------------------------- HBM copy
 
-__global__ void __launch_bounds__(512)
+// Each block walks whole 32 KB pieces (256 threads x 8 x 16 bytes), all eight loads of a thread issued before its
+// first store, so that a block keeps 32 KB in flight and touches DRAM in long contiguous runs.
+constexpr int COPY_THREADS = 256, COPY_UNROLL = 8;
+__global__ void __launch_bounds__(COPY_THREADS)
 probe_copy_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n) {
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    for (; i + 3 * stride < n; i += 4 * stride) {       // four independent 16-byte loads in flight per thread
-        const uint4 a = __ldcs(src + i), b = __ldcs(src + i + stride), c = __ldcs(src + i + 2 * stride),
-                    d = __ldcs(src + i + 3 * stride);
-        __stcs(dst + i, a); __stcs(dst + i + stride, b); __stcs(dst + i + 2 * stride, c); __stcs(dst + i + 3 * stride, d);
+    constexpr size_t PIECE = (size_t)COPY_THREADS * COPY_UNROLL;
+    const size_t pieces = n / PIECE;
+    for (size_t p = blockIdx.x; p < pieces; p += gridDim.x) {
+        const size_t base = p * PIECE + threadIdx.x;
+        uint4 v[COPY_UNROLL];
+#pragma unroll
+        for (int u = 0; u < COPY_UNROLL; ++u) v[u] = __ldcs(src + base + (size_t)u * COPY_THREADS);
+#pragma unroll
+        for (int u = 0; u < COPY_UNROLL; ++u) __stcs(dst + base + (size_t)u * COPY_THREADS, v[u]);
     }
-    for (; i < n; i += stride) __stcs(dst + i, __ldcs(src + i));
+    for (size_t i = pieces * PIECE + (size_t)blockIdx.x * COPY_THREADS + threadIdx.x; i < n; i += (size_t)gridDim.x * COPY_THREADS)
+        __stcs(dst + i, __ldcs(src + i));
 }
 
 // ---------------------------------------------------------------- fp32 FMA, registers only
@@ -252,10 +259,10 @@ int gemm_probe_copy(void* dst, const void* src, size_t bytes, double* gbs, doubl
     if (gbs == nullptr) return -4;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n = bytes / 16;
-    const int blocks = sm_count() * 4;
+    const int blocks = sm_count() * 8;
     double t = 0.0;
     const cudaError_t e = timed(s, [&]() {
-        probe_copy_kernel<<<blocks, 512, 0, s>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst), n);
+        probe_copy_kernel<<<blocks, COPY_THREADS, 0, s>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst), n);
         return cudaGetLastError();
     }, &t);
     if (e != cudaSuccess) { note_launch_error(e); return GEMM_ERR_LAUNCH; }

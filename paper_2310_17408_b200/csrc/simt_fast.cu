@@ -9,6 +9,8 @@
 //   loops L4/L5 + L6       -> each warp owns a 64 x 32 sub-tile, each thread an 8 x 8 register block that
 //                             receives one outer product per k (the role of the mr x nr micro-kernel)
 //   alpha / beta (Fig. 3)  -> applied once, when the register block is stored
+#include <atomic>
+
 #include "internal.cuh"
 
 namespace b200gemm {
@@ -267,20 +269,45 @@ __device__ __forceinline__ void unpack_block(const Acc2& p, float (&acc)[8][8]) 
         }
 }
 
+// Whether the kernel with this CTA tile can finish a split of k itself, as a thread-block cluster: every CTA then
+// parks its BM x BN partial sums in shared memory, which the operand stages are reused for (64 KB for 128 x 128:
+// more than a statically allocated array may have, so that tile keeps the workspace and the reduction pass).
+template <int BM, int BN> struct ClusterReduce { static constexpr bool value = !(BM == 128 && BN == 128); };
+
+__device__ __forceinline__ uint32_t map_shared_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(cluster_addr));
+    return v;
+}
+__device__ __forceinline__ void cluster_barrier() {      // all threads of all CTAs of the cluster
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB, bool CONV>
 __device__ __forceinline__ void
 simt_fast_body(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
                const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
-               int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, const TailSplit& tail,
+               int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, const SimtExtra& ex,
                const ConvIndex& cv) {
+    const TailSplit& tail = ex.tail;
+
     constexpr int NT = WARPS_M * WARPS_N * 32;
     static_assert(BM == WARPS_M * 64 && BN == WARPS_N * 32, "warp tile is 64 x 32");
     using LA = Loader<BM, NT, A_KCONT, VA>;
     using LB = Loader<BN, NT, B_KCONT, VB>;
     using LC = ConvLoader<BN, NT, VB>;
 
-    __shared__ __align__(16) float As[2][BK * (BM + PAD)];
-    __shared__ __align__(16) float Bs[2][BK * (BN + PAD)];
+    constexpr int A_STAGE = BK * (BM + PAD), B_STAGE = BK * (BN + PAD);
+    constexpr int STAGE_FLOATS = 2 * A_STAGE + 2 * B_STAGE;
+    constexpr int SMEM_FLOATS = (ClusterReduce<BM, BN>::value && BM * BN > STAGE_FLOATS) ? BM * BN : STAGE_FLOATS;
+    __shared__ __align__(16) float smem[SMEM_FLOATS];      // operand stages; at the end the tile's partial sums (cluster reduction)
+    float (*As)[A_STAGE] = reinterpret_cast<float (*)[A_STAGE]>(smem);
+    float (*Bs)[B_STAGE] = reinterpret_cast<float (*)[B_STAGE]>(smem + 2 * A_STAGE);
 
     // programmatic dependent launch: the next kernel of the stream may be scheduled once every CTA of this one
     // has started; it waits (griddepcontrol.wait) before it touches global memory, as this kernel does below
@@ -394,6 +421,64 @@ simt_fast_body(int64_t m, int64_t n, int64_t k, float alpha, const float* __rest
                 }
         return;
     }
+    if constexpr (ClusterReduce<BM, BN>::value) {
+        if (ex.cluster_reduce) {
+            // Split k finished by the cluster that holds this tile's k ranges (cluster rank = split index = blockIdx.z).
+            // Park the register block in shared memory as a dense [BN][BM] tile, ...
+            const int splits = (int)gridDim.z, rank = (int)blockIdx.z;
+#pragma unroll
+            for (int jh = 0; jh < 2; ++jh)
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                    for (int ih = 0; ih < 2; ++ih) {
+                        const float* v = &acc[jh * 4 + jj][ih * 4];
+                        *reinterpret_cast<float4*>(smem + (am + ih * 32) + (bn + jh * 16 + jj) * BM) = make_float4(v[0], v[1], v[2], v[3]);
+                    }
+            cluster_barrier();
+            // ... then this CTA sums its share of the tile (a contiguous run of its columns) over all CTAs, in
+            // increasing split index whoever does the summing, reading the others' shared memory
+            const bool cvec = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && (ldc % 4 == 0);
+            const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem);
+            constexpr int VECS = BM * BN / 4;
+            const int share = (VECS + splits - 1) / splits;
+            const int v_end = min(VECS, (rank + 1) * share);
+            for (int v4 = rank * share + t; v4 < v_end; v4 += NT) {
+                const int e = v4 * 4, r = e % BM, c = e / BM;
+                float4 q[CLUSTER_REDUCE_MAX_SPLITS];
+#pragma unroll
+                for (int z = 0; z < CLUSTER_REDUCE_MAX_SPLITS; ++z)
+                    if (z < splits) q[z] = ld_cluster_f4(map_shared_to_cta(base + (uint32_t)e * 4u, (uint32_t)z));
+                float4 s4 = q[0];
+#pragma unroll
+                for (int z = 1; z < CLUSTER_REDUCE_MAX_SPLITS; ++z)
+                    if (z < splits) { s4.x += q[z].x; s4.y += q[z].y; s4.z += q[z].z; s4.w += q[z].w; }
+                const int64_t gi = i0 + r, gj = j0 + c;
+                if (gi >= m || gj >= n) continue;
+                float* cp = C + gi + gj * ldc;
+                if (cvec && gi + 3 < m) {
+                    float4 o = make_float4(alpha * s4.x, alpha * s4.y, alpha * s4.z, alpha * s4.w);
+                    if (beta != 0.0f) {
+                        const float4 c0 = *reinterpret_cast<const float4*>(cp);
+                        o.x = fmaf(beta, c0.x, o.x); o.y = fmaf(beta, c0.y, o.y);
+                        o.z = fmaf(beta, c0.z, o.z); o.w = fmaf(beta, c0.w, o.w);
+                    }
+                    *reinterpret_cast<float4*>(cp) = o;
+                } else {
+                    const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4)
+                        if (gi + q4 < m) {
+                            float o = alpha * sv[q4];
+                            if (beta != 0.0f) o = fmaf(beta, cp[q4], o);
+                            cp[q4] = o;
+                        }
+                }
+            }
+            cluster_barrier();      // nobody leaves while its shared memory may still be read
+            return;
+        }
+    }
     const bool raw = partials != nullptr;
     float* out = raw ? partials + (int64_t)blockIdx.z * m * n : C;
     const int64_t ldo = raw ? m : ldc;
@@ -433,15 +518,29 @@ simt_fast_body(int64_t m, int64_t n, int64_t k, float alpha, const float* __rest
                 }
             }
         }
+
 }
 
 template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB>
 __global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
 simt_fast_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
                  const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
-                 int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, TailSplit tail) {
+                 int tiles_m, int tiles_n, int64_t kchunk, float* __restrict__ partials, SimtExtra ex) {
     simt_fast_body<BM, BN, WARPS_M, WARPS_N, MINB, A_KCONT, B_KCONT, VA, VB, false>(
-        m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, tiles_m, tiles_n, kchunk, partials, tail, ConvIndex{});
+        m, n, k, alpha, A, lda, B, ldb, beta, C, ldc, tiles_m, tiles_n, kchunk, partials, ex, ConvIndex{});
+}
+
+// a strided batch of problems of one shape: blockIdx.y is the problem (instantiated for the 64 x 64 and 128 x 128 CTA
+// tiles; a kernel of its own, because the three extra pointer offsets cost the single-problem kernel registers it
+// does not have)
+template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, bool B_KCONT, int VA, int VB>
+__global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
+simt_batched_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
+                    const float* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
+                    int tiles_m, int tiles_n, int64_t kchunk, SimtExtra ex) {
+    simt_fast_body<BM, BN, WARPS_M, WARPS_N, MINB, A_KCONT, B_KCONT, VA, VB, false>(
+        m, n, k, alpha, A + (int64_t)blockIdx.y * ex.strideA, lda, B + (int64_t)blockIdx.y * ex.strideB, ldb, beta,
+        C + (int64_t)blockIdx.y * ex.strideC, ldc, tiles_m, tiles_n, kchunk, nullptr, ex, ConvIndex{});
 }
 
 // the same kernel with operand B read through the im2row index map (n = output pixels, k = kh*kw*C_in)
@@ -449,12 +548,14 @@ template <int BM, int BN, int WARPS_M, int WARPS_N, int MINB, bool A_KCONT, int 
 __global__ void __launch_bounds__(WARPS_M* WARPS_N * 32, MINB)
 simt_conv_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda,
                  float beta, float* __restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int64_t kchunk,
-                 float* __restrict__ partials, TailSplit tail, const ConvIndex cv) {
+                 float* __restrict__ partials, SimtExtra ex, const ConvIndex cv) {
     simt_fast_body<BM, BN, WARPS_M, WARPS_N, MINB, A_KCONT, true, VA, VB, true>(
-        m, n, k, alpha, A, lda, nullptr, k, beta, C, ldc, tiles_m, tiles_n, kchunk, partials, tail, cv);
+        m, n, k, alpha, A, lda, nullptr, k, beta, C, ldc, tiles_m, tiles_n, kchunk, partials, ex, cv);
 }
 
 // ---------------------------------------------------------------- host side
+
+bool simt_fast_can_cluster_reduce(int tile) { return tile != 0; }      // see ClusterReduce
 
 bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb) {
     if (a.dtype != GEMM_F32) return false;
@@ -465,73 +566,140 @@ bool simt_fast_eligible(const GemmArgs& a, int* va, int* vb) {
 }
 
 template <int BM, int BN, int WM, int WN, int MINB, bool AK, bool BKC, int VA, int VB>
-static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
+static cudaError_t launch_one(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg, const SimtExtra& ex, int64_t batch) {
+    const TailSplit& tail = ex.tail;
     int64_t tiles_m = (a.m + BM - 1) / BM, tiles_n = (a.n + BN - 1) / BN;
     if (tiles_m * tiles_n > 0x7FFFFFFFLL || tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF / 16)
         return cudaErrorInvalidConfiguration;       // tile indices are 32-bit in the kernel (groups of 16 tile rows)
     int64_t items = tiles_m * tiles_n;
     if (tail.first < items) items = tail.first + (items - tail.first) * tail.splits;      // tail tiles count once per k range
-    if (items > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    dim3 grid((unsigned)items, 1, (unsigned)ks.splits);
+    if (items > 0x7FFFFFFFLL || batch < 1 || batch > 65535) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)items, (unsigned)batch, (unsigned)ks.splits);
     cfg->tile_m = BM; cfg->tile_n = BN; cfg->tile_k = BK; cfg->stages = 2;
-    cfg->grid = (int32_t)(items * ks.splits);
+    const int64_t ctas = items * ks.splits * batch;
+    cfg->grid = (int32_t)(ctas > 0x7FFFFFFF ? 0x7FFFFFFF : ctas);
     cudaLaunchConfig_t lc = {};
     lc.gridDim = grid;
     lc.blockDim = dim3(WM * WN * 32);
     lc.stream = a.stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // pairs with griddepcontrol.wait in the kernel
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
+    if (ex.cluster_reduce) {      // the k ranges of one tile form a cluster along z
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 1;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = (unsigned)ks.splits;
+        lc.numAttrs = 2;
+        // The CTAs of a cluster are placed close together, several to an SM where they fit, which leaves SMs idle
+        // when the whole grid is small.  Unused dynamic shared memory is requested so that no more CTAs fit on an
+        // SM than an even spread over all SMs needs (a cluster launch is split-k: always a small grid).
+        if constexpr (!BKC || true) {
+            auto kern = simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB>;
+            static std::atomic<int> static_smem[64];      // per device: static shared memory of this kernel, 0 = not asked yet
+            int dev = 0;
+            cudaGetDevice(&dev);
+            const int sms = sm_count();
+            int per_sm = (int)((ctas + sms - 1) / sms);
+            if (dev >= 0 && dev < 64 && per_sm < MINB && a.conv == nullptr) {
+                int st = static_smem[dev].load();
+                if (st == 0) {
+                    cudaFuncAttributes fa;
+                    if (cudaFuncGetAttributes(&fa, kern) == cudaSuccess &&
+                        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 190 * 1024) == cudaSuccess) {
+                        st = (int)fa.sharedSizeBytes + 1024;      // + what the system reserves per CTA
+                        static_smem[dev].store(st);
+                    } else {
+                        (void)cudaGetLastError();
+                    }
+                }
+                if (st > 0) {
+                    const int total = 228 * 1024 / (per_sm + 1) + 2048;      // per CTA: per_sm fit on an SM, per_sm + 1 do not
+                    if (total > st && total * per_sm <= 228 * 1024) lc.dynamicSmemBytes = (size_t)(total - st);
+                }
+            }
+        }
+    }
     cudaError_t le;
     if constexpr (BKC) {
         if (a.conv != nullptr) {      // operand B through the im2row index map (its memory layout is k-contiguous by construction)
             le = cudaLaunchKernelEx(&lc, simt_conv_kernel<BM, BN, WM, WN, MINB, AK, VA, VB>, a.m, a.n, a.k, a.alpha,
                                     (const float*)a.A, a.lda, a.beta, a.C, a.ldc, (int)tiles_m, (int)tiles_n, ks.chunk,
-                                    ks.splits > 1 ? partials : (float*)nullptr, tail, *a.conv);
+                                    ks.splits > 1 ? partials : (float*)nullptr, ex, *a.conv);
             return le != cudaSuccess ? le : cudaGetLastError();
+        }
+    }
+    if (batch > 1 || ex.strideA != 0 || ex.strideB != 0 || ex.strideC != 0) {
+        if constexpr ((BM == 64 && BN == 64) || (BM == 128 && BN == 128)) {
+            le = cudaLaunchKernelEx(&lc, simt_batched_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB>, a.m, a.n, a.k, a.alpha,
+                                    (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
+                                    (int)tiles_m, (int)tiles_n, ks.chunk, ex);
+            return le != cudaSuccess ? le : cudaGetLastError();
+        } else {
+            return cudaErrorInvalidConfiguration;      // batches run on the 64 x 64 and 128 x 128 tiles only
         }
     }
     le = cudaLaunchKernelEx(&lc, simt_fast_kernel<BM, BN, WM, WN, MINB, AK, BKC, VA, VB>, a.m, a.n, a.k, a.alpha,
                             (const float*)a.A, a.lda, (const float*)a.B, a.ldb, a.beta, a.C, a.ldc,
                             (int)tiles_m, (int)tiles_n, ks.chunk,
-                            ks.splits > 1 ? partials : (float*)nullptr, tail);
+                            ks.splits > 1 ? partials : (float*)nullptr, ex);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <bool AK, bool BKC, int VA, int VB>
-static cudaError_t launch_tile(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
+static cudaError_t launch_tile(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg, const SimtExtra& ex, int64_t batch) {
     switch (tile) {
-        case 0: return launch_one<128, 128, 2, 4, 2, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
-        case 1: return launch_one<128, 64, 2, 2, 3, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
-        case 2: return launch_one<64, 128, 1, 4, 3, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
-        default: return launch_one<64, 64, 1, 2, 6, AK, BKC, VA, VB>(a, ks, partials, cfg, tail);
+        case 0: return launch_one<128, 128, 2, 4, 2, AK, BKC, VA, VB>(a, ks, partials, cfg, ex, batch);
+        case 1: return launch_one<128, 64, 2, 2, 3, AK, BKC, VA, VB>(a, ks, partials, cfg, ex, batch);
+        case 2: return launch_one<64, 128, 1, 4, 3, AK, BKC, VA, VB>(a, ks, partials, cfg, ex, batch);
+        default: return launch_one<64, 64, 1, 2, 6, AK, BKC, VA, VB>(a, ks, partials, cfg, ex, batch);
     }
 }
 
 template <bool AK, bool BKC>
 static cudaError_t launch_vec(const GemmArgs& a, int va, int vb, int tile, KSplit ks, float* partials,
-                              gemm_config_t* cfg, TailSplit tail) {
-    if (va == 4 && vb == 4) return launch_tile<AK, BKC, 4, 4>(a, tile, ks, partials, cfg, tail);
-    if (va == 4) return launch_tile<AK, BKC, 4, 1>(a, tile, ks, partials, cfg, tail);
-    if (vb == 4) return launch_tile<AK, BKC, 1, 4>(a, tile, ks, partials, cfg, tail);
-    return launch_tile<AK, BKC, 1, 1>(a, tile, ks, partials, cfg, tail);
+                              gemm_config_t* cfg, const SimtExtra& ex, int64_t batch) {
+    if (va == 4 && vb == 4) return launch_tile<AK, BKC, 4, 4>(a, tile, ks, partials, cfg, ex, batch);
+    if (va == 4) return launch_tile<AK, BKC, 4, 1>(a, tile, ks, partials, cfg, ex, batch);
+    if (vb == 4) return launch_tile<AK, BKC, 1, 4>(a, tile, ks, partials, cfg, ex, batch);
+    return launch_tile<AK, BKC, 1, 1>(a, tile, ks, partials, cfg, ex, batch);
 }
 
-cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail) {
-    int va, vb;
-    simt_fast_eligible(a, &va, &vb);
-    if (a.conv != nullptr)      // 128-bit loads need whole groups of four channels on 16-byte boundaries
-        vb = ((reinterpret_cast<uintptr_t>(a.conv->X) & 15) == 0 && a.conv->c_in % 4 == 0) ? 4 : 1;
+static cudaError_t launch_simt_any(const GemmArgs& a, int va, int vb, int tile, KSplit ks, float* partials, gemm_config_t* cfg,
+                                   const SimtExtra& ex, int64_t batch) {
     cfg->kernel = GEMM_KERNEL_SIMT_FAST;
     cfg->split_k = ks.splits;
     cfg->vector_a = va; cfg->vector_b = vb;
     // A is contiguous along k when transposed; B is contiguous along k when not transposed
-    if (!a.ta && (!a.tb || a.conv)) return launch_vec<false, true>(a, va, vb, tile, ks, partials, cfg, tail);
-    if (a.ta && (!a.tb || a.conv)) return launch_vec<true, true>(a, va, vb, tile, ks, partials, cfg, tail);
-    if (!a.ta && a.tb) return launch_vec<false, false>(a, va, vb, tile, ks, partials, cfg, tail);
-    return launch_vec<true, false>(a, va, vb, tile, ks, partials, cfg, tail);
+    if (!a.ta && (!a.tb || a.conv)) return launch_vec<false, true>(a, va, vb, tile, ks, partials, cfg, ex, batch);
+    if (a.ta && (!a.tb || a.conv)) return launch_vec<true, true>(a, va, vb, tile, ks, partials, cfg, ex, batch);
+    if (!a.ta && a.tb) return launch_vec<false, false>(a, va, vb, tile, ks, partials, cfg, ex, batch);
+    return launch_vec<true, false>(a, va, vb, tile, ks, partials, cfg, ex, batch);
+}
+
+cudaError_t launch_simt_fast(const GemmArgs& a, int tile, KSplit ks, float* partials, gemm_config_t* cfg, TailSplit tail,
+                             bool cluster_reduce) {
+    int va, vb;
+    simt_fast_eligible(a, &va, &vb);
+    if (a.conv != nullptr)      // 128-bit loads need whole groups of four channels on 16-byte boundaries
+        vb = ((reinterpret_cast<uintptr_t>(a.conv->X) & 15) == 0 && a.conv->c_in % 4 == 0) ? 4 : 1;
+    const bool cluster = cluster_reduce && ks.splits > 1 && ks.splits <= CLUSTER_REDUCE_MAX_SPLITS && simt_fast_can_cluster_reduce(tile);
+    if (cluster_reduce && !cluster) return cudaErrorInvalidConfiguration;
+    const SimtExtra ex{tail, cluster ? 1 : 0, 0, 0, 0};
+    return launch_simt_any(a, va, vb, tile, ks, cluster ? nullptr : partials, cfg, ex, 1);
+}
+
+cudaError_t launch_simt_fast_batched(const GemmArgs& a, int tile, int64_t strideA, int64_t strideB, int64_t strideC,
+                                     int64_t batch, gemm_config_t* cfg) {
+    int va, vb;
+    simt_fast_eligible(a, &va, &vb);
+    if (strideA % 4 != 0) va = 1;      // every problem's operands must keep the 16-byte alignment of the first
+    if (strideB % 4 != 0) vb = 1;
+    const SimtExtra ex{TailSplit{0x7FFFFFFF, 1, 0, nullptr}, 0, strideA, strideB, strideC};
+    const KSplit whole{1, ((a.k > 0 ? a.k : 1) + BK - 1) / BK * BK};
+    return launch_simt_any(a, va, vb, tile, whole, nullptr, cfg, ex, batch);
 }
 
 }  // namespace b200gemm

@@ -31,9 +31,14 @@ template <typename T, bool TA, bool TB>
 __global__ void __launch_bounds__(256)
 simt_generic_kernel(int64_t m, int64_t n, int64_t k, float alpha, const T* __restrict__ A, int64_t lda,
                     const T* __restrict__ B, int64_t ldb, float beta, float* __restrict__ C, int64_t ldc,
-                    int64_t tiles_m, int out16) {
+                    int64_t tiles_m, int out16, int64_t strideA, int64_t strideB, int64_t strideC) {
     __shared__ float As[GK][GT + 1];
     __shared__ float Bs[GK][GT + 1];
+    // strided batch: blockIdx.y is the problem; strideC counts elements of C's type
+    A += (int64_t)blockIdx.y * strideA;
+    B += (int64_t)blockIdx.y * strideB;
+    C = out16 ? reinterpret_cast<float*>(reinterpret_cast<uint16_t*>(C) + (int64_t)blockIdx.y * strideC)
+              : C + (int64_t)blockIdx.y * strideC;
     const int t = threadIdx.x;
     const int tx = t & 15, ty = t >> 4;
     const int64_t tile = blockIdx.x;
@@ -92,16 +97,16 @@ simt_generic_kernel(int64_t m, int64_t n, int64_t k, float alpha, const T* __res
 }
 
 template <typename T>
-static cudaError_t launch_generic_t(const GemmArgs& a) {
+static cudaError_t launch_generic_t(const GemmArgs& a, int64_t sA, int64_t sB, int64_t sC, int64_t batch) {
     int64_t tiles_m = (a.m + GT - 1) / GT, tiles_n = (a.n + GT - 1) / GT;
     int64_t tiles = tiles_m * tiles_n;
-    if (tiles > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
-    dim3 grid((unsigned)tiles), block(256);
+    if (tiles > 0x7FFFFFFFLL || batch < 1 || batch > 65535) return cudaErrorInvalidConfiguration;
+    dim3 grid((unsigned)tiles, (unsigned)batch), block(256);
     const T* A = (const T*)a.A;
     const T* B = (const T*)a.B;
 #define LAUNCH(TA_, TB_)                                                                              \
     simt_generic_kernel<T, TA_, TB_><<<grid, block, 0, a.stream>>>(a.m, a.n, a.k, a.alpha, A, a.lda, B, \
-                                                                   a.ldb, a.beta, a.C, a.ldc, tiles_m, a.out16)
+                                                                   a.ldb, a.beta, a.C, a.ldc, tiles_m, a.out16, sA, sB, sC)
     if (!a.ta && !a.tb) LAUNCH(false, false);
     else if (a.ta && !a.tb) LAUNCH(true, false);
     else if (!a.ta && a.tb) LAUNCH(false, true);
@@ -110,21 +115,24 @@ static cudaError_t launch_generic_t(const GemmArgs& a) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg) {
+cudaError_t launch_simt_generic(const GemmArgs& a, gemm_config_t* cfg, int64_t strideA, int64_t strideB, int64_t strideC,
+                                int64_t batch) {
     cfg->kernel = GEMM_KERNEL_SIMT_GENERIC;
     cfg->tile_m = GT; cfg->tile_n = GT; cfg->tile_k = GK; cfg->split_k = 1; cfg->stages = 1;
     cfg->grid = (int32_t)(((a.m + GT - 1) / GT) * ((a.n + GT - 1) / GT));
     cfg->vector_a = cfg->vector_b = 1;
     cfg->launches = 1;
-    if (a.dtype == GEMM_F32) return launch_generic_t<float>(a);
-    if (a.dtype == GEMM_F16) return launch_generic_t<__half>(a);
-    return launch_generic_t<__nv_bfloat16>(a);
+    if (a.dtype == GEMM_F32) return launch_generic_t<float>(a, strideA, strideB, strideC, batch);
+    if (a.dtype == GEMM_F16) return launch_generic_t<__half>(a, strideA, strideB, strideC, batch);
+    return launch_generic_t<__nv_bfloat16>(a, strideA, strideB, strideC, batch);
 }
 
 // ---------------------------------------------------------------- C <- beta*C
 
 __global__ void __launch_bounds__(256)
-scale_kernel(int64_t m, int64_t n, float beta, float* __restrict__ C, int64_t ldc, int out16) {
+scale_kernel(int64_t m, int64_t n, float beta, float* __restrict__ C, int64_t ldc, int out16, int64_t strideC) {
+    C = out16 ? reinterpret_cast<float*>(reinterpret_cast<uint16_t*>(C) + (int64_t)blockIdx.z * strideC)
+              : C + (int64_t)blockIdx.z * strideC;
     for (int64_t j = blockIdx.y; j < n; j += gridDim.y)
         for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (int64_t)gridDim.x * blockDim.x) {
             const int64_t e = i + j * ldc;
@@ -132,10 +140,11 @@ scale_kernel(int64_t m, int64_t n, float beta, float* __restrict__ C, int64_t ld
         }
 }
 
-cudaError_t launch_scale(const GemmArgs& a) {
+cudaError_t launch_scale(const GemmArgs& a, int64_t strideC, int64_t batch) {
+    if (batch < 1 || batch > 65535) return cudaErrorInvalidConfiguration;
     unsigned gx = (unsigned)((a.m + 255) / 256 > 1024 ? 1024 : (a.m + 255) / 256);
     unsigned gy = (unsigned)(a.n > 32768 ? 32768 : a.n);
-    scale_kernel<<<dim3(gx, gy), 256, 0, a.stream>>>(a.m, a.n, a.beta, a.C, a.ldc, a.out16);
+    scale_kernel<<<dim3(gx, gy, (unsigned)batch), 256, 0, a.stream>>>(a.m, a.n, a.beta, a.C, a.ldc, a.out16, strideC);
     return cudaGetLastError();
 }
 
