@@ -21,7 +21,7 @@ _SO = _HERE / "liboracle.so"
 _SRC = [_HERE / "gemm_oracle.c", _HERE / "gemm_l1_body.inc", _HERE / "conv_oracle.c"]
 
 OR_F32, OR_F16, OR_BF16 = 0, 1, 2
-ACC_F32, ACC_F32FMA, ACC_F64 = 0, 1, 2
+ACC_F32, ACC_F32FMA, ACC_F64, ACC_F16 = 0, 1, 2, 3
 
 # default blocking of the L1 layer: the 8 x 12 micro-kernel of Section III and kc = 512 (Section IV-A);
 # mc and nc are free parameters (the paper takes them from a cache model it only cites)
@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_decode_f16.argtypes = [ctypes.c_uint16]
         L.oracle_decode_bf16.restype = dbl
         L.oracle_decode_bf16.argtypes = [ctypes.c_uint16]
+        L.oracle_round_f16.restype = dbl
+        L.oracle_round_f16.argtypes = [dbl]
         L.oracle_gemm_l0.restype = ci
         L.oracle_gemm_l0.argtypes = [ci, ci, ci, ci, i64, i64, i64, dbl, vp, i64, vp, i64,
                                      dbl, vp, i64, vp, vp, i64]
@@ -126,10 +128,12 @@ def decode_bf16(bits: int) -> float:
 
 def gemm_l0(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C0, ldc0, acc=ACC_F64):
     """Definition of the operation, one dot product per entry.  Returns an m x n array
-    (float64 for ACC_F64, float32 otherwise), F-ordered with leading dimension max(1, m)."""
+    (float64 for ACC_F64 and ACC_F16, float32 otherwise), F-ordered with leading dimension max(1, m).
+    ACC_F16: the dot products are accumulated in binary16 (one fused multiply-add and one rounding per k: the
+    paper's f16 arithmetic), then alpha*sum + beta*C0 is formed in double."""
     _check_buf(A, dtype), _check_buf(B, dtype)
     ldc = max(1, m)
-    if acc == ACC_F64:
+    if acc in (ACC_F64, ACC_F16):
         out = np.zeros(ldc * n, dtype=np.float64)
         c64, c32 = out, None
     else:
@@ -142,6 +146,11 @@ def gemm_l0(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C0, ldc
     if rc != 0:
         raise RuntimeError(f"oracle_gemm_l0 failed: {rc}")
     return out.reshape(n, ldc).T[:m, :]
+
+
+def round_f16(x: float) -> float:
+    """Nearest binary16 number to x (ties to even), as a float; the rounding step of the ACC_F16 accumulation."""
+    return float(lib().oracle_round_f16(float(x)))
 
 
 def gemm_l1(dtype, transA, transB, m, n, k, alpha, A, lda, B, ldb, beta, C0, ldc0, acc=ACC_F32,

@@ -25,7 +25,7 @@
 #endif
 
 enum { OR_F32 = 0, OR_F16 = 1, OR_BF16 = 2 };
-enum { ACC_F32 = 0, ACC_F32FMA = 1, ACC_F64 = 2 };
+enum { ACC_F32 = 0, ACC_F32FMA = 1, ACC_F64 = 2, ACC_F16 = 3 };
 
 /* ---------------------------------------------------------------- element decoding */
 
@@ -53,6 +53,24 @@ double oracle_decode_bf16(uint16_t h) {
     return sign ? -v : v;
 }
 
+/*
+ * Nearest IEEE binary16 number to x, ties to even, returned as a double (from the format's definition: 11
+ * significant bits, exponents -14 .. 15, subnormals in steps of 2^-24, overflow to infinity from 65520 on).
+ */
+double oracle_round_f16(double x) {
+    if (isnan(x) || isinf(x) || x == 0.0) return x;
+    double ax = fabs(x);
+    int e;
+    frexp(ax, &e);                    /* ax = f * 2^e, 0.5 <= f < 1: the leading bit has weight 2^(e-1) */
+    int lsb = e - 11;                 /* weight of the last of 11 significant bits */
+    if (lsb < -24) lsb = -24;         /* subnormal range: fixed spacing 2^-24 */
+    double q = ldexp(ax, -lsb);       /* in units of the last place: exact scaling */
+    double r = nearbyint(q);          /* default rounding mode: to nearest, ties to even */
+    double v = ldexp(r, lsb);
+    if (v >= 65520.0) v = INFINITY;   /* 65504 is the largest finite value; halfway to 2^16 rounds up */
+    return x < 0 ? -v : v;
+}
+
 static inline double elem(const void* X, int dtype, int64_t idx) {
     if (dtype == OR_F32) return (double)((const float*)X)[idx];
     if (dtype == OR_F16) return oracle_decode_f16(((const uint16_t*)X)[idx]);
@@ -72,7 +90,8 @@ static inline double opB(const void* B, int dtype, int tb, int64_t ldb, int64_t 
 
 /*
  * Brute force.  acc in {ACC_F32, ACC_F32FMA}: result written to C32 (C64 ignored);
- * ACC_F64: result written to C64 and, if C32 != NULL, rounded once to float there.
+ * ACC_F64: result written to C64 and, if C32 != NULL, rounded once to float there;
+ * ACC_F16: the dot product is accumulated in binary16, then alpha*sum + beta*C0 is formed in double and written like ACC_F64.
  * C0 (fp32, ldc0) is read only when beta != 0.
  */
 int oracle_gemm_l0(int dtype, int acc, int ta, int tb, int64_t m, int64_t n, int64_t k,
@@ -83,10 +102,18 @@ int oracle_gemm_l0(int dtype, int acc, int ta, int tb, int64_t m, int64_t n, int
 #pragma omp parallel for schedule(static)
     for (int64_t j = 0; j < n; ++j) {
         for (int64_t i = 0; i < m; ++i) {
-            if (acc == ACC_F64) {
+            if (acc == ACC_F64 || acc == ACC_F16) {
                 double s = 0.0;
-                for (int64_t p = 0; p < k; ++p)
-                    s += opA(A, dtype, ta, lda, i, p) * opB(B, dtype, tb, ldb, p, j);
+                if (acc == ACC_F64) {
+                    for (int64_t p = 0; p < k; ++p)
+                        s += opA(A, dtype, ta, lda, i, p) * opB(B, dtype, tb, ldb, p, j);
+                } else {
+                    /* the paper's f16 arithmetic (Section III-D): the running sum is a binary16 number, updated by one
+                     * fused multiply-add per k (the product of two binary16 numbers and its sum with a third are exact
+                     * in double; one rounding to binary16) */
+                    for (int64_t p = 0; p < k; ++p)
+                        s = oracle_round_f16(s + opA(A, dtype, ta, lda, i, p) * opB(B, dtype, tb, ldb, p, j));
+                }
                 double r = alpha * s;
                 if (beta != 0.0) r += beta * (double)C0[i + j * ldc0];
                 if (C64) C64[i + j * ldc] = r;

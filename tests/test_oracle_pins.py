@@ -12,7 +12,7 @@ import oracle
 from oracle import ACC_F32, ACC_F32FMA, ACC_F64, OR_BF16, OR_F16, OR_F32
 from workloads import (DTYPE_BF16, DTYPE_F16, DTYPE_F32, RESNET50_V15_BATCH1, VGG16_BATCH1,
                        encode_bf16, encode_f16, im2row_shapes, make_matrix)
-from workloads.generators import decode_16
+from workloads.generators import Matrix, decode_16, encode_f16
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -474,3 +474,62 @@ def test_vgg16_shapes_reproduce_paper_table():
     table = read_table("vgg16_im2row_batch1.txt")
     got = im2row_shapes(VGG16_BATCH1, batch=1, weights_as_A=False)
     assert [(i + 1, *s) for i, s in enumerate(got)] == table
+
+
+# ---------------------------------------------------------------- binary16 accumulation (the paper's f16 arithmetic)
+
+def test_round_f16_fixed_points_ties_and_library_conversion():
+    # every binary16 number is its own rounding; the midpoint of two neighbours goes to the one with an even last bit
+    pats = np.arange(0, 0x7C00, dtype=np.uint16)                       # all non-negative finite patterns, in increasing order
+    vals = pats.view(np.float16).astype(np.float64)
+    for step in (1, 37, 401):                                           # a few thousand of them, spread over all exponents
+        for i in range(0, len(vals) - 1, step):
+            assert oracle.round_f16(vals[i]) == vals[i]
+            mid = 0.5 * (vals[i] + vals[i + 1])                         # exact in double
+            even = vals[i] if (int(pats[i]) & 1) == 0 else vals[i + 1]
+            assert oracle.round_f16(mid) == even, (i, mid)
+            assert oracle.round_f16(-mid) == -even
+    # against the library's conversion (other code) on random values of all magnitudes, overflow included
+    rng = np.random.default_rng(3)
+    x = np.concatenate([rng.standard_normal(4000) * 10.0 ** rng.integers(-9, 6, 4000), [65519.9, 65520.0, 70000.0, 1e-8, 2.0 ** -25, 3 * 2.0 ** -26]])
+    with np.errstate(over="ignore"):
+        want = x.astype(np.float16).astype(np.float64)
+    got = np.array([oracle.round_f16(v) for v in x])
+    assert np.array_equal(got, want)
+
+
+def test_l0_binary16_accumulation_rounds_the_running_sum():
+    # 2048 + 1 + 1: in binary16 the spacing at 2048 is 2, so each +1 is a tie that goes back to 2048 (even); fp32 gives 2050
+    A = Matrix(encode_f16(np.array([2048.0, 1.0, 1.0])), 1, 3, 1, DTYPE_F16)
+    B = Matrix(encode_f16(np.array([1.0, 1.0, 1.0])), 3, 1, 3, DTYPE_F16)
+    C0 = np.zeros(1, dtype=np.float32)
+    args = (DTYPE_F16, "N", "N", 1, 1, 3, 1.0, A.buf, 1, B.buf, 3, 0.0, C0, 1)
+    assert oracle.gemm_l0(*args, acc=oracle.ACC_F16)[0, 0] == 2048.0
+    assert oracle.gemm_l0(*args, acc=ACC_F32)[0, 0] == 2050.0
+    # the same sum started from the small terms is exact: 1 + 1 + 2048 = 2050
+    A2 = Matrix(encode_f16(np.array([1.0, 1.0, 2048.0])), 1, 3, 1, DTYPE_F16)
+    assert oracle.gemm_l0(DTYPE_F16, "N", "N", 1, 1, 3, 1.0, A2.buf, 1, B.buf, 3, 0.0, C0, 1, acc=oracle.ACC_F16)[0, 0] == 2050.0
+    # random data against a scalar loop in the library's binary16 type (its conversion from double rounds once, to nearest even)
+    rng = np.random.default_rng(5)
+    m, n, k = 7, 5, 300
+    a = rng.standard_normal((m, k)).astype(np.float16)
+    b = rng.standard_normal((k, n)).astype(np.float16)
+    c0 = rng.standard_normal((m, n)).astype(np.float32)
+    want = np.zeros((m, n))
+    for i in range(m):
+        for j in range(n):
+            s = np.float16(0)
+            for p in range(k):
+                s = np.float16(np.float64(s) + np.float64(a[i, p]) * np.float64(b[p, j]))
+            want[i, j] = 1.5 * np.float64(s) + 0.5 * np.float64(c0[i, j])
+    got = oracle.gemm_l0(DTYPE_F16, "N", "N", m, n, k, 1.5, np.ascontiguousarray(a.T).ravel().view(np.uint16), m,
+                         np.ascontiguousarray(b.T).ravel().view(np.uint16), k, 0.5, np.ascontiguousarray(c0.T).ravel(), m,
+                         acc=oracle.ACC_F16)
+    assert np.array_equal(got, want)
+    # integer data whose partial sums are all binary16 numbers: identical to the fp64 mode
+    ai = rng.integers(-4, 5, (m, 64)).astype(np.float16)
+    bi = rng.integers(-4, 5, (64, n)).astype(np.float16)
+    pa, pb = np.ascontiguousarray(ai.T).ravel().view(np.uint16), np.ascontiguousarray(bi.T).ravel().view(np.uint16)
+    z = np.zeros(m * n, dtype=np.float32)
+    assert np.array_equal(oracle.gemm_l0(DTYPE_F16, "N", "N", m, n, 64, 1.0, pa, m, pb, 64, 0.0, z, m, acc=oracle.ACC_F16),
+                          oracle.gemm_l0(DTYPE_F16, "N", "N", m, n, 64, 1.0, pa, m, pb, 64, 0.0, z, m, acc=ACC_F64))
