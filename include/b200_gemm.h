@@ -31,7 +31,24 @@ typedef enum {
      * alpha*acc + beta*C is rounded once, to nearest even, when it is stored.  Wherever this header says that C
      * is fp32, read "of the 16-bit type" for these two; ldc counts elements of that type. */
     GEMM_F16_C16  = 3,
-    GEMM_BF16_C16 = 4
+    GEMM_BF16_C16 = 4,
+    /* fp32 A, B and C multiplied on the tensor cores: every operand entry is split into three bfloat16 pieces
+     * (x = x1 + x2 + x3 to within the last bit or two of x), and the six piece products that matter,
+     * A1 B1 + A1 B2 + A2 B1 + A2 B2 + A1 B3 + A3 B1, are accumulated in fp32, smallest first.  Not the exact IEEE
+     * fp32 arithmetic of GEMM_F32 (the dropped products are of relative size 2^-24; results stay within the same
+     * error bound 4 k 2^-24 max|A| max|B| and are exact on small integers), but several times faster on large
+     * problems.  Needs a registered workspace of gemm_workspace_bytes(); without one, and for problems too small to
+     * gain, the call runs as GEMM_F32.  Operands must be finite.  (The paper's data-type section, III-D, only
+     * narrows the type; this mode goes the other way and keeps fp32 data on the narrow-type unit.) */
+    GEMM_F32_TC   = 5,
+    /* The paper's f16 arithmetic (Section III-D "Data types": with the precision set to f16 the generated micro-kernel
+     * holds A, B, C and the accumulator registers in binary16).  A, B and C are binary16 and the products are
+     * accumulated in binary16 on the tensor cores (tcgen05.mma with a binary16 accumulator); alpha*acc + beta*C is
+     * formed in fp32 from the binary16 sum and rounded once, to nearest even, at the store.  The running sum is
+     * rounded as the hardware rounds it, which need not be after every product as a scalar fp16 loop would: results
+     * agree with such a loop to within 2 k 2^-11 sum_p |a_ip b_pj| and exactly while every partial sum is a
+     * binary16 number.  Sums beyond 65504 overflow to infinity, as in any binary16 accumulation.  k is never split. */
+    GEMM_F16_ACC16 = 6
 } gemm_dtype_t;
 
 /* return codes (0 = success; -1 .. -15 = the 1-based position of the first invalid argument of gemm()) */

@@ -11,7 +11,7 @@ from pathlib import Path
 
 _LIB_PATH = Path(__file__).resolve().parent / "libb200gemm.so"
 
-GEMM_F32, GEMM_F16, GEMM_BF16, GEMM_F16_C16, GEMM_BF16_C16 = 0, 1, 2, 3, 4
+GEMM_F32, GEMM_F16, GEMM_BF16, GEMM_F16_C16, GEMM_BF16_C16, GEMM_F32_TC, GEMM_F16_ACC16 = 0, 1, 2, 3, 4, 5, 6
 GEMM_OK = 0
 GEMM_ERR_WORKSPACE, GEMM_ERR_LAUNCH, GEMM_ERR_ARCH, GEMM_ERR_DEVICE, GEMM_ERR_TOO_LARGE = -100, -101, -102, -103, -104
 GEMM_KERNEL_AUTO, GEMM_KERNEL_SIMT_GENERIC, GEMM_KERNEL_SIMT_FAST, GEMM_KERNEL_TENSOR = 0, 1, 2, 3

@@ -260,7 +260,8 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         for (int cand = bn_lo; cand <= bn_hi; cand *= 2)
             for (int so : split_opts) {
                 if (g_force_split > 0 && so != 1) continue;
-                const int sp = g_force_split > 0 ? g_force_split : so;
+                if (a.acc16 && so != 1) continue;      // a binary16 accumulator is never split along k
+                const int sp = (g_force_split > 0 && !a.acc16) ? g_force_split : so;
                 if (sp > 1 && g_force_split == 0) {
                     if (a.k / sp < 256) continue;
                     if (ws_repack + (size_t)sp * a.m * a.n * sizeof(float) > ws_avail) continue;
@@ -281,7 +282,7 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         p->pair = bn == 256 && want == 1 && a.m > 128 && pair_tiles >= sms / 2 && main_us >= 10.0;
     }
     if (g_force_tile_m == 256) p->pair = bn == 256;
-    if (g_force_tile_m == 128) p->pair = false;
+    if (g_force_tile_m == 128 || a.acc16) p->pair = false;      // the binary16 accumulator exists in the single-CTA kernel only
     p->ks = make_split(a.k, want, 64);
     p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
     if (ws_repack + p->ws_partials > ws_avail) {
@@ -341,7 +342,8 @@ static int validate(int dtype, char ta, char tb, int64_t m, int64_t n, int64_t k
             default: return false;
         }
     };
-    if (dtype != GEMM_F32 && dtype != GEMM_F16 && dtype != GEMM_BF16 && dtype != GEMM_F16_C16 && dtype != GEMM_BF16_C16)
+    if (dtype != GEMM_F32 && dtype != GEMM_F16 && dtype != GEMM_BF16 && dtype != GEMM_F16_C16 && dtype != GEMM_BF16_C16 &&
+        dtype != GEMM_F32_TC && dtype != GEMM_F16_ACC16)
         return -1;
     if (!tr(ta, tA)) return -2;
     if (!tr(tb, tB)) return -3;
@@ -368,7 +370,63 @@ static int fail_launch(cudaError_t e) {
     return GEMM_ERR_LAUNCH;
 }
 
-static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
+static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0);
+
+// ---------------------------------------------------------------- fp32 on the tensor cores (GEMM_F32_TC)
+
+// Workspace for the bfloat16 pieces of A and B: three copies each, leading dimension rounded up to 8 elements.
+struct Split3Layout {
+    int64_t a_rows, a_cols, b_rows, b_cols, lda_p, ldb_p;
+    size_t a_piece, b_piece, total;      // bytes
+};
+static Split3Layout split3_layout(const GemmArgs& a) {
+    Split3Layout L;
+    L.a_rows = a.ta ? a.k : a.m; L.a_cols = a.ta ? a.m : a.k;
+    L.b_rows = a.tb ? a.n : a.k; L.b_cols = a.tb ? a.k : a.n;
+    L.lda_p = round_up(L.a_rows, 8);
+    L.ldb_p = round_up(L.b_rows, 8);
+    L.a_piece = (size_t)round_up(L.lda_p * L.a_cols * 2, 256);
+    L.b_piece = (size_t)round_up(L.ldb_p * L.b_cols * 2, 256);
+    L.total = 3 * (L.a_piece + L.b_piece);
+    return L;
+}
+// worth it from about here on (below, the exact kernel is as fast and the six launches cost more than they save)
+static bool split3_worthwhile(const GemmArgs& a) {
+    return (double)a.m * (double)a.n * (double)a.k >= 512.0 * 512.0 * 512.0 && a.m >= 128 && a.n >= 128 && a.k >= 64;
+}
+
+// C <- alpha * sum of the six piece products + beta*C: six bfloat16 GEMMs accumulating into C, smallest terms first
+static int run_f32_split3(const GemmArgs& a, DeviceState* st, void* ws, size_t ws_bytes) {
+    const Split3Layout L = split3_layout(a);
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    void* ap[3] = {base, base + L.a_piece, base + 2 * L.a_piece};
+    void* bp[3] = {base + 3 * L.a_piece, base + 3 * L.a_piece + L.b_piece, base + 3 * L.a_piece + 2 * L.b_piece};
+    cudaError_t e = launch_split3(static_cast<const float*>(a.A), L.a_rows, L.a_cols, a.lda, ap[0], ap[1], ap[2], L.lda_p, a.stream);
+    if (e == cudaSuccess)
+        e = launch_split3(static_cast<const float*>(a.B), L.b_rows, L.b_cols, a.ldb, bp[0], bp[1], bp[2], L.ldb_p, a.stream);
+    if (e != cudaSuccess) return fail_launch(e);
+    static const int order[6][2] = {{2, 0}, {0, 2}, {1, 1}, {1, 0}, {0, 1}, {0, 0}};      // (piece of A, piece of B)
+    int launches = 2;
+    gemm_config_t last{};
+    for (int t = 0; t < 6; ++t) {
+        GemmArgs g = a;
+        g.dtype = GEMM_BF16;
+        g.split3 = 0;
+        g.A = ap[order[t][0]]; g.lda = L.lda_p;
+        g.B = bp[order[t][1]]; g.ldb = L.ldb_p;
+        if (t > 0) g.beta = 1.0f;               // later products accumulate onto the earlier ones
+        const int rc = run_gemm(g, st, L.total + (size_t)0);
+        if (rc != GEMM_OK) return rc;
+        launches += t_last_cfg.launches;
+        last = t_last_cfg;
+    }
+    last.launches = launches;
+    t_last_cfg = last;
+    (void)ws_bytes;
+    return GEMM_OK;
+}
+
+static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip) {
     GemmArgs a = a0;
     gemm_config_t cfg{};
     cfg.split_k = 1;
@@ -382,6 +440,17 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0) {
         t_last_cfg = cfg;
         return e == cudaSuccess ? GEMM_OK : fail_launch(e);
     }
+
+    if (a.split3 && a.dtype == GEMM_F32 && !a.conv && ws_skip == 0 && g_force_kernel != GEMM_KERNEL_SIMT_FAST &&
+        g_force_kernel != GEMM_KERNEL_SIMT_GENERIC && g_force_kernel != GEMM_KERNEL_SIMT_DIRECT &&
+        (split3_worthwhile(a) || g_force_kernel == GEMM_KERNEL_TENSOR) &&
+        a.m <= 0x7FFFFFFFLL && a.n <= 0x7FFFFFFFLL && a.k <= 0x7FFFFFFFLL) {
+        void* ws3;
+        size_t ws3_bytes;
+        workspace_for(st, a.stream, &ws3, &ws3_bytes);
+        if (ws3 != nullptr && ws3_bytes >= split3_layout(a).total) return run_f32_split3(a, st, ws3, ws3_bytes);
+    }
+    a.split3 = 0;      // from here on: the exact fp32 path
 
     void* ws;
     size_t ws_bytes;
@@ -488,6 +557,8 @@ int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, f
     GemmArgs a{input_dtype(dtype), ta, tb, m, n, k, alpha, beta, A, B, static_cast<float*>(C), lda, ldb, ldc,
                static_cast<cudaStream_t>(stream), st->status};
     a.out16 = output16(dtype);
+    a.split3 = dtype == GEMM_F32_TC ? 1 : 0;
+    a.acc16 = dtype == GEMM_F16_ACC16 ? 1 : 0;
     return run_gemm(a, st);
 }
 
@@ -514,6 +585,7 @@ int gemm_strided_batched(int dtype, char transA, char transB, int64_t m, int64_t
     GemmArgs a{input_dtype(dtype), ta, tb, m, n, k, alpha, beta, A, B, static_cast<float*>(C), lda, ldb, ldc,
                static_cast<cudaStream_t>(stream), st->status};
     a.out16 = output16(dtype);
+    a.acc16 = dtype == GEMM_F16_ACC16 ? 1 : 0;
     const int es = elem_size(dtype), es_c = c_elem_size(dtype);
     auto at = [&](int64_t b0) {      // the call's arguments moved to problem b0
         GemmArgs x = a;
@@ -742,6 +814,14 @@ size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int6
     // judged for 16-byte aligned pointers and minimal leading dimensions (lda = rows of the stored A, ...)
     GemmArgs a{input_dtype(dtype), ta, tb, m, n, k, 1.0f, 0.0f, (const void*)16, (const void*)16, nullptr,
                ta ? k : m, tb ? n : k, m, nullptr, nullptr};
+    if (dtype == GEMM_F32_TC && split3_worthwhile(a)) {      // the pieces, then what the bfloat16 products would like
+        const Split3Layout L = split3_layout(a);
+        GemmArgs b = a;
+        b.dtype = GEMM_BF16;
+        b.lda = L.lda_p; b.ldb = L.ldb_p;
+        Plan pb = make_plan(b, sms, ~(size_t)0);
+        return L.total + (pb.kernel < 0 ? 0 : pb.ws_total);
+    }
     Plan p = make_plan(a, sms, ~(size_t)0);
     return p.kernel < 0 ? 0 : p.ws_total;
 }

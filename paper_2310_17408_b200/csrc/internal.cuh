@@ -31,12 +31,19 @@ struct GemmArgs {
     uint32_t* status;      // device status word (bounded waits report here)
     const ConvIndex* conv = nullptr;   // non-null: op(B) is the lowered activation matrix of this layer (B, ldb, tb unused)
     int out16 = 0;                     // element type of C: 0 = fp32, GEMM_F16 / GEMM_BF16 = that 16-bit type (C then points to it)
+    int acc16 = 0;                     // binary16 inputs, binary16 accumulation on the tensor cores, binary16 result (GEMM_F16_ACC16)
+    int split3 = 0;                    // fp32 operands: multiply on the tensor cores as three bfloat16 pieces each (GEMM_F32_TC)
 };
 
 // The all-16-bit data types (GEMM_F16_C16, GEMM_BF16_C16) are a 16-bit input type plus a 16-bit result:
 // inside the library dtype is always the input type and out16 names the result's type.
-inline int input_dtype(int dtype) { return dtype == GEMM_F16_C16 ? GEMM_F16 : (dtype == GEMM_BF16_C16 ? GEMM_BF16 : dtype); }
-inline int output16(int dtype) { return dtype == GEMM_F16_C16 ? GEMM_F16 : (dtype == GEMM_BF16_C16 ? GEMM_BF16 : 0); }
+inline int input_dtype(int dtype) {
+    return (dtype == GEMM_F16_C16 || dtype == GEMM_F16_ACC16) ? GEMM_F16
+           : (dtype == GEMM_BF16_C16 ? GEMM_BF16 : (dtype == GEMM_F32_TC ? GEMM_F32 : dtype));
+}
+inline int output16(int dtype) {
+    return (dtype == GEMM_F16_C16 || dtype == GEMM_F16_ACC16) ? GEMM_F16 : (dtype == GEMM_BF16_C16 ? GEMM_BF16 : 0);
+}
 inline int c_elem_size(int dtype) { return output16(dtype) ? 2 : 4; }
 
 // fp32 <-> the 16-bit result types, round to nearest even (device)
@@ -101,7 +108,7 @@ __host__ __device__ inline void decode_tile(int tile, int tiles_m, int tiles_n, 
     *tn = (tile % per_group) / gsz;
 }
 
-inline int elem_size(int dtype) { return dtype == GEMM_F32 ? 4 : 2; }      // of A and B
+inline int elem_size(int dtype) { return (dtype == GEMM_F32 || dtype == GEMM_F32_TC) ? 4 : 2; }      // of A and B
 
 // C <- beta*C  (beta == 0: store +0 without reading)
 cudaError_t launch_scale(const GemmArgs& a, int64_t strideC = 0, int64_t batch = 1);
@@ -139,6 +146,11 @@ cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, ge
 // copy op-independent stored matrix (rows x cols, ld) of 16-bit elements into an aligned layout (ld_out)
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,
                             cudaStream_t stream);
+
+// fp32 stored matrix (rows x cols, ld) -> three bfloat16 matrices p1, p2, p3 (leading dimension ld_p) with
+// x = p1 + p2 + p3 up to the last bit or two of x: p1 = bf16(x), p2 = bf16(x - p1), p3 = bf16(x - p1 - p2)
+cudaError_t launch_split3(const float* src, int64_t rows, int64_t cols, int64_t ld, void* p1, void* p2, void* p3,
+                          int64_t ld_p, cudaStream_t stream);
 
 // launches a one-warp kernel whose bounded wait is certain to expire (nothing arrives at its barrier)
 cudaError_t launch_wait_expiry_probe(uint32_t* status, cudaStream_t stream);

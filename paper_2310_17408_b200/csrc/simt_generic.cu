@@ -234,6 +234,62 @@ cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------- fp32 -> three bfloat16 pieces
+
+// One thread per four consecutive rows of a column.  Each piece is rounded to nearest even from what the earlier
+// pieces left over; the subtractions are exact in fp32 (the piece shares the leading bits of what it was rounded from).
+__global__ void __launch_bounds__(256)
+split3_kernel(const float* __restrict__ src, int64_t rows, int64_t cols, int64_t ld, __nv_bfloat16* __restrict__ p1,
+              __nv_bfloat16* __restrict__ p2, __nv_bfloat16* __restrict__ p3, int64_t ld_p, int vec) {
+    const int64_t quads = (rows + 3) / 4;
+    for (int64_t j = blockIdx.y; j < cols; j += gridDim.y)
+        for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < quads; q += (int64_t)gridDim.x * blockDim.x) {
+            const int64_t i = q * 4;
+            float x[4] = {0.f, 0.f, 0.f, 0.f};
+            const float* s = src + i + j * ld;
+            if (vec && i + 3 < rows) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(s));
+                x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (i + e < rows) x[e] = __ldg(s + e);
+            }
+            uint16_t h[3][4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float r = x[e];
+#pragma unroll
+                for (int t = 0; t < 3; ++t) {
+                    const __nv_bfloat16 b = __float2bfloat16_rn(r);
+                    h[t][e] = __bfloat16_as_ushort(b);
+                    r -= __bfloat162float(b);
+                }
+            }
+            // ld_p is a multiple of 8 and the pieces are 16-byte aligned: the four values of a piece go out as one 8-byte store
+            // (rows past the matrix, inside its last quad, are written as zeros: they lie in the padding of the copy)
+            __nv_bfloat16* out[3] = {p1, p2, p3};
+#pragma unroll
+            for (int t = 0; t < 3; ++t) {
+                const uint2 w = make_uint2((uint32_t)h[t][0] | ((uint32_t)h[t][1] << 16), (uint32_t)h[t][2] | ((uint32_t)h[t][3] << 16));
+                *reinterpret_cast<uint2*>(out[t] + i + j * ld_p) = w;
+            }
+        }
+}
+
+cudaError_t launch_split3(const float* src, int64_t rows, int64_t cols, int64_t ld, void* p1, void* p2, void* p3,
+                          int64_t ld_p, cudaStream_t stream) {
+    if (rows == 0 || cols == 0) return cudaSuccess;
+    const int64_t quads = (rows + 3) / 4;
+    int64_t gx = (quads + 255) / 256, gy = cols;
+    if (gx > 1024) gx = 1024;
+    if (gy > 32768) gy = 32768;
+    const int vec = ((reinterpret_cast<uintptr_t>(src) & 15) == 0 && ld % 4 == 0) ? 1 : 0;
+    split3_kernel<<<dim3((unsigned)gx, (unsigned)gy), 256, 0, stream>>>(src, rows, cols, ld, (__nv_bfloat16*)p1, (__nv_bfloat16*)p2,
+                                                                     (__nv_bfloat16*)p3, ld_p, vec);
+    return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------- tail reduction
 
 // One block row per tail tile (blockIdx.x) and a quarter of its entries per blockIdx.y: sums the tile's k ranges in

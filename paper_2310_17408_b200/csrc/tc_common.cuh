@@ -139,6 +139,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
+// 32 columns of a binary16 accumulator (one 16-bit value in the low half of each 32-bit TMEM column), two columns
+// packed into each of 16 registers: low half = even column, high half = odd column
+__device__ __forceinline__ void tmem_ld16_packed(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.pack::16b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---- CTA pairs (clusters of two CTAs, tcgen05 cta_group::2)
@@ -253,7 +263,8 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int64_t row0, i
 // (j, j+1) into one packed word, neighbouring lanes exchange these words, and a byte permute leaves the even lane with
 // rows (2i, 2i+1) of column j and the odd lane with those of column j+1 (per two entries: one packed conversion,
 // one shuffle, one permute, one shared-memory store).
-template <int BN, int STORE_BUFS, typename Release>
+// ACC16: the accumulator itself is binary16 (tcgen05.mma with a binary16 D): its values are widened to fp32 for the scaling.
+template <int BN, int STORE_BUFS, bool ACC16 = false, typename Release>
 __device__ __forceinline__ void epilogue_tile16(uint32_t tmem_acc, int64_t row0, int64_t n0, int half, int lane,
                                                 int64_t m, int64_t n, float alpha, float beta, float* out, int64_t ldo,
                                                 bool via_tma, const CUtensorMap* tmC, float* stage, uint32_t& sbuf,
@@ -268,9 +279,21 @@ __device__ __forceinline__ void epilogue_tile16(uint32_t tmem_acc, int64_t row0,
             if (col0 >= n) break;
             const bool last_chunk = (c + 2 >= BN / 32) || (col0 + 64 >= n);
             uint32_t v[32];
-            tmem_ld32(tmem_acc + c * 32, v);
             const int64_t e0 = row + col0 * ldo;
-            tmem_ld_wait();
+            if (ACC16) {
+                uint32_t h[16];
+                tmem_ld16_packed(tmem_acc + c * 32, h);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h[j]));
+                    v[2 * j] = __float_as_uint(f.x);
+                    v[2 * j + 1] = __float_as_uint(f.y);
+                }
+            } else {
+                tmem_ld32(tmem_acc + c * 32, v);
+                tmem_ld_wait();
+            }
             if (last_chunk) { release_acc(); released = true; }
             float* r = reinterpret_cast<float*>(v);       // scaled in place
             if (alpha != 1.0f || beta != 0.0f) {
@@ -343,7 +366,7 @@ inline ConvTma conv_tma_params(const ConvIndex* cv) {
     if (!cv) return ConvTma{1, 1, 1, 0, 1, 1};
     return ConvTma{cv->ho, cv->wo, cv->sh, cv->ph, cv->kw, (int32_t)(cv->c_in / 64)};
 }
-// instruction descriptor of tcgen05.mma kind::f16 with fp32 accumulation: mma_m x mma_n, operand majorness
-uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n);
+// instruction descriptor of tcgen05.mma kind::f16: mma_m x mma_n, operand majorness, fp32 (or binary16) accumulator
+uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n, bool acc16 = false);
 
 }  // namespace b200gemm

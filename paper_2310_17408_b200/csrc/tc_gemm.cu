@@ -36,7 +36,9 @@ template <int BN> struct TcCfg {
 // A_MN: op(A) is contiguous along m in memory (transA = N); B_MN: op(B) contiguous along n (transB = T).
 // CONV: op(B) is the im2row-lowered activation matrix of a convolution layer, fetched by TMA in im2col mode
 // straight from the NHWC tensor (tmB is then an im2col map); the lowered matrix never exists in memory.
-template <int BN, bool A_MN, bool B_MN, bool CONV, bool OUT16>
+// OUT: 0 = fp32 result; 1 = 16-bit result (fp32 accumulator, one rounding at the store); 2 = binary16 accumulator
+// and binary16 result (the paper's all-f16 arithmetic, Section III-D)
+template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
@@ -44,6 +46,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                uint32_t idesc, uint32_t* status, const ConvTma conv, int out16) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
+    constexpr bool OUT16 = OUT != 0, ACC16 = OUT == 2;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -224,7 +227,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool done = false;
             if constexpr (OUT16) {
                 if (!raw) {      // 16-bit result: one rounding at the store (split-k partial sums stay fp32)
-                    epilogue_tile16<BN, Cfg::STORE_BUFS>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, out, ldc,
+                    epilogue_tile16<BN, Cfg::STORE_BUFS, ACC16>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, out, ldc,
                                                 store_via_tma == 1, &tmC, stage, sbuf, out16, release);
                     done = true;
                 }
@@ -382,10 +385,10 @@ bool tensor_eligible(const GemmArgs& a) {
     return encode_fn() != nullptr;
 }
 
-uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n) {
+uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n, bool acc16) {
     const uint32_t fmt = dtype == GEMM_F16 ? 0u : 1u;    // input format: 0 = f16, 1 = bf16
     uint32_t d = 0;
-    d |= 1u << 4;                    // accumulator format: f32
+    d |= (acc16 ? 0u : 1u) << 4;     // accumulator format: 1 = f32, 0 = f16
     d |= fmt << 7;                   // A format
     d |= fmt << 10;                  // B format
     d |= (a_mn ? 1u : 0u) << 15;     // A is MN-major
@@ -395,13 +398,13 @@ uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n) {
     return d;
 }
 
-template <int BN, bool A_MN, bool B_MN, bool CONV, bool OUT16>
+template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
                              const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
     static std::atomic<bool> attr_set[64];      // zero-initialised; set once per device
-    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV, OUT16>;
+    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV, OUT>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev].load()) {
@@ -427,7 +430,7 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN), a.status, conv_tma_params(a.conv), a.out16);
+                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN, OUT == 2), a.status, conv_tma_params(a.conv), a.out16);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
@@ -453,13 +456,22 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
     if (ks.splits > 1 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && a.m % 4 == 0 &&
         a.m * a.n * 4 < (1LL << 40))
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
+    if constexpr (!CONV) {
+        if (a.acc16) {      // binary16 accumulator (never split along k: partial sums would need a wider type)
+            switch (tile_n) {
+                case 256: return launch_tc<256, A_MN, B_MN, false, 2>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+                case 128: return launch_tc<128, A_MN, B_MN, false, 2>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+                default:  return launch_tc<64, A_MN, B_MN, false, 2>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+            }
+        }
+    }
     switch (tile_n) {
-        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, CONV, true>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
-                                  : launch_tc<256, A_MN, B_MN, CONV, false>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, CONV, true>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
-                                  : launch_tc<128, A_MN, B_MN, CONV, false>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, CONV, true>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
-                                  : launch_tc<64, A_MN, B_MN, CONV, false>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
+                                  : launch_tc<256, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
+                                  : launch_tc<128, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
+                                  : launch_tc<64, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
     }
 }
 

@@ -29,13 +29,15 @@ def to_device(mat: Matrix) -> torch.Tensor:
     return torch.from_numpy(mat.buf.view(np.int16) if mat.buf.dtype == np.uint16 else mat.buf).cuda()
 
 
-def run_problem(p: Problem, A: Matrix, B: Matrix, C0: Matrix, *, workspace=True, check_inputs=True):
+def run_problem(p: Problem, A: Matrix, B: Matrix, C0: Matrix, *, workspace=True, check_inputs=True, api_dtype=None):
     """Returns (C as Matrix on the host, config dict).  Asserts rc == 0, padding rows of C untouched,
-    A and B unmodified, and the device status word clean."""
+    A and B unmodified, and the device status word clean.  api_dtype: the library's data-type code when it is not
+    the element type of the operands (GEMM_F32_TC)."""
+    code = p.dtype if api_dtype is None else api_dtype
     if workspace:
-        ensure_workspace(g.gemm_workspace_bytes(p.dtype, p.transA, p.transB, p.m, p.n, p.k) + (64 << 20))
+        ensure_workspace(g.gemm_workspace_bytes(code, p.transA, p.transB, p.m, p.n, p.k) + (64 << 20))
     dA, dB, dC = to_device(A), to_device(B), to_device(C0)
-    rc = g.gemm(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), A.ld, dB.data_ptr(), B.ld,
+    rc = g.gemm(code, p.transA, p.transB, p.m, p.n, p.k, p.alpha, dA.data_ptr(), A.ld, dB.data_ptr(), B.ld,
                 p.beta, dC.data_ptr(), C0.ld, torch.cuda.current_stream().cuda_stream)
     assert rc == 0, g.gemm_status_string(rc)
     cfg = g.gemm_last_config()
