@@ -34,7 +34,7 @@ def test_argument_checks_run_without_a_device():
     assert g.gemm(g.GEMM_F16_C16, "N", "N", 4, 4, 4, 1.0, 16, 4, 16, 4, 0.0, 16, 2) == -14
     assert g.gemm(g.GEMM_BF16_C16, "N", "N", 4, 4, 4, 1.0, 16, 4, 16, 4, 0.0, 17, 4) == -13
     assert g.gemm(g.GEMM_BF16, "N", "N", 4, 4, 4, 1.0, 16, 4, 16, 4, 0.0, 18, 4) == -13       # fp32 C at a 2-byte boundary
-    assert g.gemm(5, "N", "N", 4, 4, 4, 1.0, 16, 4, 16, 4, 0.0, 16, 4) == -1
+    assert g.gemm(9, "N", "N", 4, 4, 4, 1.0, 16, 4, 16, 4, 0.0, 16, 4) == -1
     assert "lda" in g.gemm_status_string(-9)
     assert g.gemm_force_kernel(99) == -1 and g.gemm_force_kernel(0) == 0
 
