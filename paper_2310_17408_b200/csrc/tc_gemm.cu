@@ -67,6 +67,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     // let the next kernel of the stream start its own set-up as soon as SMs free up (it waits before touching memory)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 32) {      // descriptors into the TMA unit's cache while the barriers are set up
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+        if (store_via_tma) prefetch_tensormap(&tmC);
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < NACC; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), EPI_WARPS); }
@@ -287,49 +292,91 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// Tensor maps are pure functions of what they describe (address, type, extents, stride, box), and encoding one costs
+// the host about a microsecond.  Each host thread keeps the last few it built: a caller that multiplies the same
+// buffers again (the usual case: a layer's weights, a pre-allocated activation buffer) gets its maps from here.
+struct MapKey {
+    uint64_t v[7];
+    bool operator==(const MapKey& o) const {
+        for (int i = 0; i < 7; ++i)
+            if (v[i] != o.v[i]) return false;
+        return true;
+    }
+};
+struct MapCache {
+    static constexpr int N = 32;
+    MapKey key[N];
+    CUtensorMap map[N];
+    bool used[N] = {};
+    int next = 0;
+};
+template <typename Encode>
+static bool cached_map(CUtensorMap* tm, const MapKey& k, Encode&& encode) {
+    static thread_local MapCache cache;
+    for (int i = 0; i < MapCache::N; ++i)
+        if (cache.used[i] && cache.key[i] == k) { *tm = cache.map[i]; return true; }
+    if (!encode(tm)) return false;
+    const int slot = cache.next;
+    cache.next = (cache.next + 1) % MapCache::N;
+    cache.key[slot] = k;
+    cache.map[slot] = *tm;
+    cache.used[slot] = true;
+    return true;
+}
+
 // 2-D map over a stored column-major matrix: dim0 = contiguous dimension (rows), dim1 = columns (stride ld)
 bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_t cols, int64_t ld,
                      uint32_t box_rows, uint32_t box_cols) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)rows, (cuuint64_t)cols};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {box_rows, box_cols};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, dtype == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
-                    const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    const MapKey k{{1, (uint64_t)dtype, (uint64_t)(uintptr_t)base, (uint64_t)rows, (uint64_t)cols, (uint64_t)ld,
+                    ((uint64_t)box_rows << 32) | box_cols}};
+    return cached_map(tm, k, [&](CUtensorMap* out) {
+        cuuint64_t dims[2] = {(cuuint64_t)rows, (cuuint64_t)cols};
+        cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+        cuuint32_t box[2] = {box_rows, box_cols};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = fn(out, dtype == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r == CUDA_SUCCESS;
+    });
 }
 
 // map over the split-k partial sums [split][n][m] (fp32, dense): 32 x 32 x 1 boxes
 bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)m, (cuuint64_t)n, (cuuint64_t)splits};
-    cuuint64_t strides[2] = {(cuuint64_t)m * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
-    cuuint32_t box[3] = {32, 32, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    const MapKey k{{2, 0, (uint64_t)(uintptr_t)base, (uint64_t)m, (uint64_t)n, (uint64_t)splits, 0}};
+    return cached_map(tm, k, [&](CUtensorMap* out) {
+        cuuint64_t dims[3] = {(cuuint64_t)m, (cuuint64_t)n, (cuuint64_t)splits};
+        cuuint64_t strides[2] = {(cuuint64_t)m * 4, (cuuint64_t)m * (cuuint64_t)n * 4};
+        cuuint32_t box[3] = {32, 32, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r == CUDA_SUCCESS;
+    });
 }
 
-// map over the fp32 result for the epilogue's tile stores: 32 x 32 boxes, no swizzle
+// map over the result (fp32 or a 16-bit type) for the epilogue's tile stores: 32 x 32 boxes, no swizzle
 bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc, int out16) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)n};
-    cuuint64_t strides[1] = {(cuuint64_t)ldc * (out16 ? 2 : 4)};
-    const CUtensorMapDataType dt = out16 == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
-                                   : out16 == GEMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-    cuuint32_t box[2] = {32, 32};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, dt, 2, const_cast<float*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
+    const MapKey k{{3, (uint64_t)out16, (uint64_t)(uintptr_t)base, (uint64_t)m, (uint64_t)n, (uint64_t)ldc, 0}};
+    return cached_map(tm, k, [&](CUtensorMap* out) {
+        cuuint64_t dims[2] = {(cuuint64_t)m, (cuuint64_t)n};
+        cuuint64_t strides[1] = {(cuuint64_t)ldc * (out16 ? 2 : 4)};
+        const CUtensorMapDataType dt = out16 == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                       : out16 == GEMM_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+        cuuint32_t box[2] = {32, 32};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = fn(out, dt, 2, const_cast<float*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r == CUDA_SUCCESS;
+    });
 }
 
 typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

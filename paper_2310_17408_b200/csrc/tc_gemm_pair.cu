@@ -60,6 +60,11 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const bool leader = rank == 0;
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 32) {      // descriptors into the TMA unit's cache while the barriers are set up
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+        if (store_via_tma) prefetch_tensormap(&tmC);
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int a = 0; a < NACC; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * EPI_WARPS); }
