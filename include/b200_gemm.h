@@ -136,11 +136,14 @@ int gemm_strided_batched(int dtype, char transA, char transB, int64_t m, int64_t
 
 /*
  * gemm_host — the same operation on HOST buffers (pinned memory for full speed; pageable works but serialises).
- * Allocates device buffers from the stream-ordered pool, then moves column panels of op(B) and C through a
- * three-stream pipeline (copy in / multiply on `stream` / copy out), so that transfers overlap the arithmetic,
- * and synchronises `stream` before returning.  Only the m x n window of C is transferred: C is copied in only when
- * beta != 0, and rows m..ldc-1 of the host array are never touched.  Leading dimensions and layout as for gemm().
- * Calls from several host threads on one device share the copy streams and are therefore serialised by them.
+ * Takes device buffers from a memory pool of the library's own (kept between calls; the application's default pool
+ * is not touched), then moves column panels of op(B) and C through a three-stream pipeline (copy in / multiply on
+ * `stream` / copy out), so that transfers overlap the arithmetic, and synchronises `stream` before returning.  While A
+ * itself is still on its way the first panel is multiplied k panel by k panel, each step adding onto C (the order of
+ * the paper's loop L2, Fig. 1): a large result is therefore summed in a different order than gemm() sums it, inside
+ * the same error bound (identical on integer-valued data).  Only the m x n window of C is transferred: C is copied
+ * in only when beta != 0, and rows m..ldc-1 of the host array are never touched.  Leading dimensions and layout as for
+ * gemm().  Calls from several host threads are serialised.
  */
 int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k,
               float alpha, const void* A_host, int64_t lda, const void* B_host, int64_t ldb,

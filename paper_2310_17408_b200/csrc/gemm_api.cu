@@ -234,7 +234,11 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
     //   - all SMs together fill shared memory from L2 at ~10 TB/s; HBM moves 6.5 TB/s
     //   - the epilogue moves 32 columns of a tile in ~0.45 us
     //   - splitting k adds a reduction pass: ~4 us + (splits + 1) * m * n * 4 bytes at ~5 TB/s
-    auto cost_us = [&](int bn, int splits) {
+    //   - or, for up to 8 k ranges, the ranges of a tile run as a thread-block cluster and sum the tile through
+    //     distributed shared memory: ~2.5 us, no partial sums in memory, but one tile per CTA (no persistent loop), so
+    //     only while all CTAs fit the GPU at once (measured: 512 x 1568 x 4608 on 28 tiles of 128 x 256, 4 ranges = 112
+    //     CTAs 17.0 us, 6 ranges = 168 CTAs 28.1 us; one launch with a reduction pass 18.9; unsplit 31.0)
+    auto cost_us = [&](int bn, int splits, bool cluster) {
         const double tiles = (double)ceil_div(a.m, 128) * (double)ceil_div(a.n, bn);
         const double items = tiles * splits;
         const double rounds = (double)ceil_div((int64_t)items, sms);
@@ -244,12 +248,13 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         const double main_us = rounds * kb * t_kb + rounds * (bn / 32) * 0.45;
         const double fill_us = items * kb * stage / 1e7;
         const double mn = (double)a.m * (double)a.n;
-        const double hbm_us = (2.0 * ((double)a.m * a.k + (double)a.k * a.n) + 4.0 * mn * splits) / 6.5e6;
+        const double hbm_us = (2.0 * ((double)a.m * a.k + (double)a.k * a.n) + 4.0 * mn * (cluster ? 1 : splits)) / 6.5e6;
         double t = 7.0 + std::max(main_us, std::max(fill_us, hbm_us));
-        if (splits > 1) t += 4.0 + (splits + 1) * mn * 4.0 / 5e6;
+        if (splits > 1) t += cluster ? 2.5 : 4.0 + (splits + 1) * mn * 4.0 / 5e6;
         return t;
     };
     int bn = 256, want = 1;
+    bool want_cluster = false;
     {
         const int bn_lo = (g_force_tile_n == 64 || g_force_tile_n == 128 || g_force_tile_n == 256) ? g_force_tile_n
                           : (a.n <= 64 ? 64 : 128);
@@ -258,17 +263,22 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         const int split_opts[] = {1, 2, 3, 4, 6, 8};
         double best = 1e300;
         for (int cand = bn_lo; cand <= bn_hi; cand *= 2)
-            for (int so : split_opts) {
-                if (g_force_split > 0 && so != 1) continue;
-                if (a.acc16 && so != 1) continue;      // a binary16 accumulator is never split along k
-                const int sp = (g_force_split > 0 && !a.acc16) ? g_force_split : so;
-                if (sp > 1 && g_force_split == 0) {
-                    if (a.k / sp < 256) continue;
-                    if (ws_repack + (size_t)sp * a.m * a.n * sizeof(float) > ws_avail) continue;
+            for (int so : split_opts)
+                for (int cl = 0; cl < 2; ++cl) {
+                    if (g_force_split > 0 && so != 1) continue;
+                    if (a.acc16 && so != 1) continue;      // a binary16 accumulator is never split along k
+                    const int sp = (g_force_split > 0 && !a.acc16) ? g_force_split : so;
+                    const bool cluster = cl == 1;
+                    if (cluster && (sp < 2 || sp > 8 || g_force_reduction == 1)) continue;
+                    if (cluster && g_force_split == 0 && ceil_div(a.m, 128) * ceil_div(a.n, cand) * sp > sms) continue;
+                    if (!cluster && sp > 1 && g_force_reduction == 2 && sp <= 8) continue;
+                    if (sp > 1 && g_force_split == 0 && a.k / sp < 256) continue;
+                    if (sp > 1 && !cluster && ws_repack + (size_t)sp * a.m * a.n * sizeof(float) > ws_avail) {
+                        if (g_force_split == 0) continue;
+                    }
+                    const double c = cost_us(cand, sp, cluster);
+                    if (c < best) { best = c; bn = cand; want = sp; want_cluster = cluster; }
                 }
-                const double c = cost_us(cand, sp);
-                if (c < best) { best = c; bn = cand; want = sp; }
-            }
     }
     p->tile = bn;
     // CTA pairs (256 x 256 tiles) fill a third less shared memory per flop, which is what limits the 128 x 256
@@ -280,11 +290,13 @@ static void plan_tensor(const GemmArgs& a, int sms, size_t ws_avail, bool a_ok, 
         const double rounds = (double)ceil_div(ceil_div(a.m, 128) * ceil_div(a.n, 256), sms);
         const double main_us = rounds * (double)ceil_div(a.k, 64) * 0.27;
         p->pair = bn == 256 && want == 1 && a.m > 128 && pair_tiles >= sms / 2 && main_us >= 10.0;
+        if (want_cluster) p->pair = false;
     }
     if (g_force_tile_m == 256) p->pair = bn == 256;
     if (g_force_tile_m == 128 || a.acc16) p->pair = false;      // the binary16 accumulator exists in the single-CTA kernel only
     p->ks = make_split(a.k, want, 64);
-    p->ws_partials = p->ks.splits > 1 ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
+    p->cluster_reduce = want_cluster && !p->pair && p->ks.splits >= 2 && p->ks.splits <= 8;      // single-CTA kernel only
+    p->ws_partials = (p->ks.splits > 1 && !p->cluster_reduce) ? (size_t)p->ks.splits * a.m * a.n * sizeof(float) : 0;
     if (ws_repack + p->ws_partials > ws_avail) {
         if (g_force_split > 0) { p->kernel = -1; return; }
         p->ks = make_split(a.k, 1, 64);
@@ -495,7 +507,8 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip) {
     }
     float* partials = p.ks.splits > 1 ? reinterpret_cast<float*>(wsp) : nullptr;
     if (p.kernel == GEMM_KERNEL_TENSOR) {
-        e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg) : launch_tensor(a, p.tile, p.ks, partials, &cfg);
+        e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg)
+                   : launch_tensor(a, p.tile, p.ks, partials, &cfg, p.cluster_reduce);
     } else if (p.tail_splits > 1) {
         TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
         e = launch_simt_fast(a, p.tile, p.ks, nullptr, &cfg, tail);
@@ -657,11 +670,32 @@ static cudaError_t copy_window(void* dst, const void* src, int64_t rows, int64_t
     return cudaMemcpy2DAsync(dst, (size_t)ld * es, src, (size_t)ld * es, (size_t)rows * es, (size_t)cols, kind, s);
 }
 
-struct HostPipe {          // per device: the two copy streams of gemm_host
+struct HostPipe {          // per device: what gemm_host keeps between calls
     bool init = false;
-    cudaStream_t in = nullptr, out = nullptr;
+    cudaStream_t in = nullptr, out = nullptr;      // the two copy streams
+    cudaMemPool_t pool = nullptr;                   // the library's own pool for the staging buffers of A, B and C
+    std::vector<cudaEvent_t> events;                // grown on demand, reused by every call
 };
 static HostPipe g_pipe[MAX_DEVICES];
+static std::mutex g_host_mutex;                     // one gemm_host per process at a time (they share the pipe)
+
+// columns per panel of C: a multiple of the CTA tile such that the panel's tiles fill whole waves of the GPU as nearly as
+// possible (a panel is one gemm() call), among the widths that cut C into 4 .. 12 panels
+static int64_t host_panel_columns(int dtype, int64_t m, int64_t n, int sms) {
+    const int tile = dtype == GEMM_F32 ? 128 : 256;                 // fp32: 128 x 128 CTA tiles; 16-bit: 256 x 256 on CTA pairs
+    const int64_t slots = dtype == GEMM_F32 ? 2 * (int64_t)sms : sms / 2;
+    const int64_t tiles_m = ceil_div(m, tile), tiles_n = ceil_div(n, tile);
+    int64_t best = tiles_n;
+    double best_eff = -1.0;
+    for (int64_t c = 1; c <= tiles_n; ++c) {
+        const int64_t panels = ceil_div(tiles_n, c);
+        if (panels < 4 || panels > 12) continue;
+        const int64_t tiles = tiles_m * c;
+        const double eff = (double)tiles / (double)(ceil_div(tiles, slots) * slots);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = c; }
+    }
+    return best * tile;
+}
 
 int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k, float alpha, const void* A_host,
               int64_t lda, const void* B_host, int64_t ldb, float beta, void* C_host, int64_t ldc, void* stream) {
@@ -672,21 +706,24 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return GEMM_ERR_LAUNCH;
+    DeviceState* st = device_state();
+    if (!st) return GEMM_ERR_LAUNCH;
+    std::lock_guard<std::mutex> host_lock(g_host_mutex);
     HostPipe* pipe = &g_pipe[dev];
-    {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        if (!pipe->init) {
-            // keep freed staging buffers in the stream-ordered pool instead of returning them at every synchronise
-            cudaMemPool_t pool;
-            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
-                uint64_t keep = ~0ull;
-                cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
-            }
-            if (cudaStreamCreateWithFlags(&pipe->in, cudaStreamNonBlocking) != cudaSuccess ||
-                cudaStreamCreateWithFlags(&pipe->out, cudaStreamNonBlocking) != cudaSuccess)
-                return fail_launch(cudaGetLastError());
-            pipe->init = true;
-        }
+    if (!pipe->init) {
+        // a pool of the library's own, so that keeping freed staging buffers for the next call changes nothing for
+        // the application's default pool
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        if (cudaMemPoolCreate(&pipe->pool, &props) != cudaSuccess) return fail_launch(cudaGetLastError());
+        uint64_t keep = ~0ull;
+        cudaMemPoolSetAttribute(pipe->pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        if (cudaStreamCreateWithFlags(&pipe->in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&pipe->out, cudaStreamNonBlocking) != cudaSuccess)
+            return fail_launch(cudaGetLastError());
+        pipe->init = true;
     }
     const int es = elem_size(dtype);       // of A and B
     const bool needs_ab = (k > 0 && alpha != 0.0f);
@@ -700,48 +737,41 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     // is multiplied and panel p-1 is copied out.  Small problems use one panel.
     const double traffic = (double)b_bytes + (double)m * n * es_c * (beta != 0.0f ? 2.0 : 1.0);
     int64_t panel = n;
-    if (traffic > 32e6 && n >= 1024) {
-        int64_t panels = (int64_t)(traffic / 48e6) + 1;
-        if (panels > 16) panels = 16;
-        panel = round_up(ceil_div(n, panels), 256);
-    }
+    if (traffic > 32e6 && n >= 1024) panel = host_panel_columns(input_dtype(dtype), m, n, st->sms);
+    if (panel > n) panel = n;
     const int np = (int)ceil_div(n, panel);
-    // While A itself is still arriving, the first column panel is computed in row panels of op(A): each needs
-    // only its own rows of A, so the multiplication starts long before the whole of A is on the device.
-    int64_t rpanel = m;
-    if (np > 1 && needs_ab && (double)a_bytes > 32e6 && m >= 1024) {
-        int64_t rp = (int64_t)((double)a_bytes / 32e6) + 1;
-        if (rp > 8) rp = 8;
-        rpanel = round_up(ceil_div(m, rp), 256);
+    // While A itself is still arriving, the first column panel is computed k panel by k panel (the order of the
+    // paper's loop L2 around the packing of A, Fig. 1: C accumulates over blocks of k): each step needs only the part
+    // of A that has arrived, runs on whole tiles of C, and adds onto what the earlier steps left in C.
+    int64_t kpanel = k;
+    // (not for 16-bit results: every step would round C to 16 bits again)
+    if (np > 1 && needs_ab && (double)a_bytes > 32e6 && k >= 2048 && es_c == 4) {
+        int64_t kp = (int64_t)((double)a_bytes / 32e6) + 1;
+        if (kp > 8) kp = 8;
+        kpanel = round_up(ceil_div(k, kp), 256);
     }
-    const int nr = (int)ceil_div(m, rpanel);
+    const int nk = (int)ceil_div(k > 0 ? k : 1, kpanel);
 
     void *dA = nullptr, *dB = nullptr, *dC = nullptr;
     cudaError_t e = cudaSuccess;
     int rc = GEMM_OK;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess && r != cudaSuccess) e = r; return r == cudaSuccess; };
-    const int nev = 2 * np + 3 + nr;
-    cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[nev];
-    if (!ev) return GEMM_ERR_LAUNCH;
-    int made = 0;
-    for (; made < nev; ++made)
-        if (!chk(cudaEventCreateWithFlags(&ev[made], cudaEventDisableTiming))) break;
+    const size_t nev = (size_t)(2 * np + 3 + nk);
+    while (pipe->events.size() < nev && e == cudaSuccess) {
+        cudaEvent_t ev_new;
+        if (chk(cudaEventCreateWithFlags(&ev_new, cudaEventDisableTiming))) pipe->events.push_back(ev_new);
+    }
+    if (e != cudaSuccess) return fail_launch(e);
+    cudaEvent_t* ev = pipe->events.data();
     cudaEvent_t ev_alloc = ev[0], ev_a = ev[1], ev_done = ev[2];
 
-    if (e == cudaSuccess) {
-        if (a_bytes) chk(cudaMallocAsync(&dA, a_bytes, s));
-        if (b_bytes) chk(cudaMallocAsync(&dB, b_bytes, s));
-        chk(cudaMallocAsync(&dC, c_bytes, s));
-    }
+    if (a_bytes) chk(cudaMallocFromPoolAsync(&dA, a_bytes, pipe->pool, s));
+    if (b_bytes) chk(cudaMallocFromPoolAsync(&dB, b_bytes, pipe->pool, s));
+    chk(cudaMallocFromPoolAsync(&dC, c_bytes, pipe->pool, s));
     if (e == cudaSuccess) {
         chk(cudaEventRecord(ev_alloc, s));                       // the copy streams start after the allocations
         chk(cudaStreamWaitEvent(pipe->in, ev_alloc, 0));
         chk(cudaStreamWaitEvent(pipe->out, ev_alloc, 0));
-        if (a_bytes && nr == 1) {
-            chk(copy_window(dA, A_host, a_rows, a_cols, lda, es, cudaMemcpyHostToDevice, pipe->in));
-            chk(cudaEventRecord(ev_a, pipe->in));
-            chk(cudaStreamWaitEvent(s, ev_a, 0));
-        }
     }
     for (int p = 0; p < np && e == cudaSuccess && rc == GEMM_OK; ++p) {
         const int64_t j0 = (int64_t)p * panel, cols = (n - j0 < panel) ? n - j0 : panel;
@@ -761,21 +791,24 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
         chk(cudaEventRecord(ev_in, pipe->in));
         chk(cudaStreamWaitEvent(s, ev_in, 0));
         if (e != cudaSuccess) break;
-        if (p == 0 && nr > 1) {
-            for (int r = 0; r < nr && e == cudaSuccess && rc == GEMM_OK; ++r) {
-                const int64_t i0 = (int64_t)r * rpanel, rows = (m - i0 < rpanel) ? m - i0 : rpanel;
-                // rows i0.. of op(A): a row window of the stored matrix (transA = N) or whole columns of it (T)
-                const size_t a_off = ta ? (size_t)i0 * lda * es : (size_t)i0 * es;
+        if (p == 0 && needs_ab) {
+            // A follows the first panel of B and C; the first panel is multiplied k panel by k panel as A arrives
+            for (int q = 0; q < nk && e == cudaSuccess && rc == GEMM_OK; ++q) {
+                const int64_t p0 = (int64_t)q * kpanel, kk = (k - p0 < kpanel) ? k - p0 : kpanel;
+                // columns p0.. of op(A): whole columns of the stored matrix (transA = N) or a row window of it (T)
+                const size_t a_off = ta ? (size_t)p0 * es : (size_t)p0 * lda * es;
                 char* dAp = static_cast<char*>(dA) + a_off;
                 const char* hAp = static_cast<const char*>(A_host) + a_off;
-                if (ta) chk(copy_window(dAp, hAp, k, rows, lda, es, cudaMemcpyHostToDevice, pipe->in));
-                else chk(copy_window(dAp, hAp, rows, k, lda, es, cudaMemcpyHostToDevice, pipe->in));
-                cudaEvent_t ev_row = ev[3 + 2 * np + r];
-                chk(cudaEventRecord(ev_row, pipe->in));
-                chk(cudaStreamWaitEvent(s, ev_row, 0));
+                if (ta) chk(copy_window(dAp, hAp, kk, m, lda, es, cudaMemcpyHostToDevice, pipe->in));
+                else chk(copy_window(dAp, hAp, m, kk, lda, es, cudaMemcpyHostToDevice, pipe->in));
+                cudaEvent_t ev_k = ev[3 + 2 * np + q];
+                chk(cudaEventRecord(ev_k, pipe->in));
+                chk(cudaStreamWaitEvent(s, ev_k, 0));
                 if (e != cudaSuccess) break;
-                rc = gemm(dtype, transA, transB, rows, cols, k, alpha, dAp, lda, dBp + b_off, ldb, beta,
-                          static_cast<char*>(dC) + c_off + (size_t)i0 * es_c, ldc, stream);
+                // rows p0.. of op(B) inside this panel: a row window of the stored matrix (transB = N) or whole columns (T)
+                const size_t bk_off = tb ? (size_t)p0 * ldb * es : (size_t)p0 * es;
+                rc = gemm(dtype, transA, transB, m, cols, kk, alpha, dAp, lda, dBp + b_off + bk_off, ldb, q == 0 ? beta : 1.0f,
+                          static_cast<char*>(dC) + c_off, ldc, stream);
             }
         } else {
             rc = gemm(dtype, transA, transB, m, cols, k, alpha, dA, lda, needs_ab ? dBp + b_off : nullptr, ldb, beta,
@@ -787,18 +820,14 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
         chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols, ldc, es_c,
                         cudaMemcpyDeviceToHost, pipe->out));
     }
-    if (made > 2) {
-        cudaEventRecord(ev_done, pipe->out);                     // the caller's stream rejoins both copy streams
-        cudaStreamWaitEvent(s, ev_done, 0);
-        cudaEventRecord(ev_a, pipe->in);
-        cudaStreamWaitEvent(s, ev_a, 0);
-    }
+    cudaEventRecord(ev_done, pipe->out);                     // the caller's stream rejoins both copy streams
+    cudaStreamWaitEvent(s, ev_done, 0);
+    cudaEventRecord(ev_a, pipe->in);
+    cudaStreamWaitEvent(s, ev_a, 0);
     if (dA) cudaFreeAsync(dA, s);
     if (dB) cudaFreeAsync(dB, s);
     if (dC) cudaFreeAsync(dC, s);
     chk(cudaStreamSynchronize(s));
-    for (int i = 0; i < made; ++i) cudaEventDestroy(ev[i]);
-    delete[] ev;
     if (e != cudaSuccess) return fail_launch(e);
     return rc;
 }

@@ -139,7 +139,9 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 
 // tcgen05 tensor-core kernel (fp16 / bf16).  tile_n in {64, 128, 256}; tile_m is 128.
 bool tensor_eligible(const GemmArgs& a);
-cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg);
+// cluster: the ks.splits (2 .. 8) k ranges of a tile run as one thread-block cluster and sum the tile themselves through
+// distributed shared memory (no partials, no reduction pass)
+cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg, bool cluster = false);
 // the same on CTA pairs (tcgen05 cta_group::2): 256 x 256 tiles, two SMs per tile
 cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg);
 

@@ -36,6 +36,55 @@ template <int BN> struct TcCfg {
 // A_MN: op(A) is contiguous along m in memory (transA = N); B_MN: op(B) contiguous along n (transB = T).
 // CONV: op(B) is the im2row-lowered activation matrix of a convolution layer, fetched by TMA in im2col mode
 // straight from the NHWC tensor (tmB is then an im2col map); the lowered matrix never exists in memory.
+// Split k summed by the cluster (see the kernel): this CTA's share of the BN-column tile whose partial sums lie, as dense
+// [BN][128] fp32 tiles, at shared-memory offset `park_addr` of every CTA of the cluster.  Kept out of line so that its
+// registers do not count against the main loop and the epilogue.
+template <int BN>
+__device__ __noinline__ void cluster_sum_tile(uint32_t park_addr, int S, int64_t row0, int64_t col0, int64_t m, int64_t n,
+                                              float alpha, float beta, float* __restrict__ C, int64_t ldc, int out16) {
+    const uint32_t rank = cluster_ctarank();
+    constexpr int VECS = TBM * BN / 4;
+    const int share = (VECS + S - 1) / S;
+    const int v_end = min(VECS, (int)(rank + 1) * share);
+    const bool cvec = !out16 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 && ldc % 4 == 0;
+    for (int v4 = (int)rank * share + (int)threadIdx.x; v4 < v_end; v4 += TC_THREADS) {
+        const int e = v4 * 4, r = e % TBM, c = e / TBM;
+        float4 q[8];
+#pragma unroll
+        for (int z = 0; z < 8; ++z)
+            if (z < S) {
+                const uint32_t ra = map_to_cta(park_addr + (uint32_t)e * 4u, (uint32_t)z);
+                asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(q[z].x), "=f"(q[z].y), "=f"(q[z].z), "=f"(q[z].w) : "r"(ra));
+            }
+        float4 s4 = q[0];
+#pragma unroll
+        for (int z = 1; z < 8; ++z)
+            if (z < S) { s4.x += q[z].x; s4.y += q[z].y; s4.z += q[z].z; s4.w += q[z].w; }
+        const int64_t gi = row0 + r, gj = col0 + c;
+        if (gi >= m || gj >= n) continue;
+        const int64_t e0 = gi + gj * ldc;
+        if (cvec && gi + 3 < m) {
+            float4 o = make_float4(alpha * s4.x, alpha * s4.y, alpha * s4.z, alpha * s4.w);
+            if (beta != 0.0f) {
+                const float4 c0 = *reinterpret_cast<const float4*>(C + e0);
+                o.x = fmaf(beta, c0.x, o.x); o.y = fmaf(beta, c0.y, o.y);
+                o.z = fmaf(beta, c0.z, o.z); o.w = fmaf(beta, c0.w, o.w);
+            }
+            *reinterpret_cast<float4*>(C + e0) = o;
+        } else {
+            const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (gi + u < m) {
+                    float o = alpha * sv[u];
+                    if (beta != 0.0f) o = fmaf(beta, load_c(C, out16, e0 + u), o);
+                    store_c(C, out16, e0 + u, o);
+                }
+        }
+    }
+}
+
 // OUT: 0 = fp32 result; 1 = 16-bit result (fp32 accumulator, one rounding at the store); 2 = binary16 accumulator
 // and binary16 result (the paper's all-f16 arithmetic, Section III-D)
 template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
@@ -43,7 +92,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
-               uint32_t idesc, uint32_t* status, const ConvTma conv, int out16) {
+               uint32_t idesc, uint32_t* status, const ConvTma conv, int out16, int cluster_k) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr bool OUT16 = OUT != 0, ACC16 = OUT == 2;
@@ -93,6 +142,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int64_t items = (int64_t)tiles_m * tiles_n * splits;
+    // Work items of this CTA.  Ordinarily: blockIdx.x, blockIdx.x + gridDim.x, ...  With cluster_k (split k finished
+    // inside the kernel) every CTA has exactly one item: the cluster is the tile, the rank in the cluster the k range.
+    int64_t item_first = blockIdx.x, item_step = gridDim.x;
+    if (cluster_k) {
+        item_first = (int64_t)(blockIdx.x % cluster_k) * ((int64_t)tiles_m * tiles_n) + blockIdx.x / cluster_k;
+        item_step = items;
+    }
     constexpr int GROUP = 16;
     auto decode = [&](int64_t item, int& tm, int& tn, int& sp) {
         const int64_t tiles = (int64_t)tiles_m * tiles_n;
@@ -115,7 +171,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             uint32_t cnt = 0;
             bool ok = true;
-            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+            for (int64_t item = item_first; item < items && ok; item += item_step) {
                 int tm, tn, sp;
                 decode(item, tm, tn, sp);
                 int64_t kbeg;
@@ -166,7 +222,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             uint32_t cnt = 0, it = 0;
             bool ok = true;
-            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
+            for (int64_t item = item_first; item < items && ok; item += item_step, ++it) {
                 int tm, tn, sp;
                 decode(item, tm, tn, sp);
                 int64_t kbeg;
@@ -211,7 +267,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         float* stage = store_stage + (warp - 2) * (Cfg::STORE_BUFS * 32 * 32);
         uint32_t it = 0, sbuf = 0;
         bool ok = true;
-        for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x, ++it) {
+        for (int64_t item = item_first; item < items && ok; item += item_step, ++it) {
             int tm, tn, sp;
             decode(item, tm, tn, sp);
             const uint32_t acc = it % NACC, aph = (it / NACC) & 1;
@@ -229,6 +285,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (lane == 0) mbar_arrive(tempty_bar(acc));
             };
             const uint32_t tacc = tmem_base + acc * BN + ((uint32_t)(q * 32) << 16);
+            if (cluster_k) {
+                // park the raw accumulator in shared memory as a dense [BN][128] fp32 tile (the operand stages are free:
+                // every MMA that read them has completed); the cluster sums it below
+                float* park = reinterpret_cast<float*>(smem_al);
+#pragma unroll 1
+                for (int c = half; c < BN / 32; c += 2) {
+                    uint32_t v[32];
+                    tmem_ld32(tacc + c * 32, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) park[(c * 32 + j) * TBM + q * 32 + lane] = __uint_as_float(v[j]);
+                }
+                release();
+                continue;
+            }
             bool done = false;
             if constexpr (OUT16) {
                 if (!raw) {      // 16-bit result: one rounding at the store (split-k partial sums stay fp32)
@@ -242,6 +313,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                           raw, via_tma, &tmC, sp, stage, sbuf, release);
         }
         if (lane == 0) bulk_wait_all();       // staging tiles must outlive the stores that read them
+    }
+
+    if (cluster_k) {
+        // ------------------------------------------------ split k summed by the cluster (every thread of every CTA)
+        // Each CTA of the cluster holds the partial sums of its k range in shared memory.  After a cluster barrier this
+        // CTA sums a contiguous share of the tile over all CTAs, in increasing k range whoever does the summing,
+        // through distributed shared memory, applies alpha / beta and writes C.  The barrier is the hardware's (a
+        // cluster is co-scheduled); a role that gave up a bounded wait arrives here as well, so nobody waits in vain.
+        __syncthreads();
+        __syncwarp();
+        cluster_sync_all();
+        if (*abort_flag == 0) {
+            int tm, tn, sp;
+            decode(item_first, tm, tn, sp);
+            cluster_sum_tile<BN>(smem_base, cluster_k, (int64_t)tm * TBM, (int64_t)tn * BN, m, n, alpha, beta, C, ldc, out16);
+        }
+        __syncwarp();
+        cluster_sync_all();      // nobody leaves while its shared memory may still be read
     }
 
     // ------------------------------------------------ teardown: every thread arrives here on every path
@@ -447,7 +536,8 @@ uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n, bool 
 
 template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
-                             const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma) {
+                             const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma,
+                             bool cluster = false) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
     static std::atomic<bool> attr_set[64];      // zero-initialised; set once per device
@@ -462,27 +552,37 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
     const int64_t tiles_m = (a.m + TBM - 1) / TBM, tiles_n = (a.n + BN - 1) / BN;
     if (tiles_m > 0x7FFFFFFF || tiles_n > 0x7FFFFFFF || tiles_m * tiles_n > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     const int64_t items = tiles_m * tiles_n * ks.splits;
-    const int grid = (int)(items < sm_count() ? items : sm_count());
+    if (cluster && (ks.splits < 2 || ks.splits > 8 || items > 0x7FFFFFFFLL)) return cudaErrorInvalidConfiguration;
+    // cluster: one CTA per item, the k ranges of a tile forming a cluster; otherwise a persistent grid
+    const int grid = cluster ? (int)items : (int)(items < sm_count() ? items : sm_count());
     cfg->tile_m = TBM; cfg->tile_n = BN; cfg->tile_k = TBK; cfg->stages = Cfg::STAGES; cfg->grid = grid;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)grid);
     lc.blockDim = dim3(TC_THREADS);
     lc.dynamicSmemBytes = Cfg::SMEM_BYTES;
     lc.stream = a.stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // pairs with griddepcontrol.wait in the kernel
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
+    if (cluster) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)ks.splits;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        lc.numAttrs = 2;
+    }
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
-                                        ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN, OUT == 2), a.status, conv_tma_params(a.conv), a.out16);
+                                        (ks.splits > 1 && !cluster) ? partials : (float*)nullptr,
+                                        instr_desc(a.dtype, A_MN, B_MN, TBM, BN, OUT == 2), a.status, conv_tma_params(a.conv), a.out16,
+                                        cluster ? ks.splits : 0);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template <bool A_MN, bool B_MN, bool CONV>
-static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg) {
+static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg, bool cluster) {
     CUtensorMap tmA, tmB;
     // stored A: (m x k) if transA = N [contiguous m], (k x m) otherwise [contiguous k]
     bool ok = A_MN ? make_map(&tmA, a.dtype, a.A, a.m, a.k, a.lda, 64, TBK)
@@ -500,7 +600,7 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
     int store_via_tma = 0;
     if (ks.splits == 1 && c_tma_addressable(a.C, a.m, a.ldc, a.out16))
         store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc, a.out16) ? 1 : 0;
-    if (ks.splits > 1 && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && a.m % 4 == 0 &&
+    if (ks.splits > 1 && !cluster && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && a.m % 4 == 0 &&
         a.m * a.n * 4 < (1LL << 40))
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
     if constexpr (!CONV) {
@@ -513,27 +613,27 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
         }
     }
     switch (tile_n) {
-        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
-                                  : launch_tc<256, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
-                                  : launch_tc<128, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
-        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma)
-                                  : launch_tc<64, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);
+        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, cluster)
+                                  : launch_tc<256, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, cluster);
+        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, cluster)
+                                  : launch_tc<128, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, cluster);
+        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, CONV, 1>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, cluster)
+                                  : launch_tc<64, A_MN, B_MN, CONV, 0>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma, cluster);
     }
 }
 
-cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg) {
+cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg, bool cluster) {
     cfg->kernel = GEMM_KERNEL_TENSOR;
     cfg->split_k = ks.splits;
     cfg->vector_a = cfg->vector_b = 1;
     const bool a_mn = !a.ta, b_mn = a.tb;
     if (a.conv != nullptr)
-        return a_mn ? launch_tc_bn<true, false, true>(a, tile_n, ks, partials, cfg)
-                    : launch_tc_bn<false, false, true>(a, tile_n, ks, partials, cfg);
-    if (a_mn && b_mn) return launch_tc_bn<true, true, false>(a, tile_n, ks, partials, cfg);
-    if (a_mn && !b_mn) return launch_tc_bn<true, false, false>(a, tile_n, ks, partials, cfg);
-    if (!a_mn && b_mn) return launch_tc_bn<false, true, false>(a, tile_n, ks, partials, cfg);
-    return launch_tc_bn<false, false, false>(a, tile_n, ks, partials, cfg);
+        return a_mn ? launch_tc_bn<true, false, true>(a, tile_n, ks, partials, cfg, cluster)
+                    : launch_tc_bn<false, false, true>(a, tile_n, ks, partials, cfg, cluster);
+    if (a_mn && b_mn) return launch_tc_bn<true, true, false>(a, tile_n, ks, partials, cfg, cluster);
+    if (a_mn && !b_mn) return launch_tc_bn<true, false, false>(a, tile_n, ks, partials, cfg, cluster);
+    if (!a_mn && b_mn) return launch_tc_bn<false, true, false>(a, tile_n, ks, partials, cfg, cluster);
+    return launch_tc_bn<false, false, false>(a, tile_n, ks, partials, cfg, cluster);
 }
 
 }  // namespace b200gemm
