@@ -68,11 +68,17 @@ CONV_WORKLOADS = {
 # kernel and problem, with the hash of the kernel's source file at capture time: a changed kernel reports null.
 TRAFFIC = {
     ("simt_fast_kernel", "8192x8192x8192", "f32"): {
-        "bytes": 3470697216 + 265491968, "source": "paper_2310_17408_b200/csrc/simt_fast.cu",
-        "sha256": "03a90bb8978a54edffb191d8a450eb031ac71995c0342240b444043f0a35874e"},
+        "bytes": 3953546752 + 265748224, "source": "paper_2310_17408_b200/csrc/simt_fast.cu",
+        "sha256": "2fe44e48407d403c605326b6e6d9841e5eab96f818a2308ef116e323c3a5cd47"},
     ("tc_gemm_pair_kernel", "8192x8192x8192", "bf16"): {
-        "bytes": 1123555584 + 260218368, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
-        "sha256": "3f6a7f0db8a5cf9085ad9289a0e93d1bfa8610df8a362df4d565033b16a993bf"},
+        "bytes": 1101455104 + 261325312, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
+        "sha256": "8d1968c394593bfd009d17f5e7fd973d9745ffc862c1a1d0bf45dbe54b790fbb"},
+    ("tc_gemm_pair_kernel", "16384x16384x16384", "bf16"): {
+        "bytes": 14162072320 + 1103334144, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
+        "sha256": "8d1968c394593bfd009d17f5e7fd973d9745ffc862c1a1d0bf45dbe54b790fbb"},
+    ("tc_gemm_pair_kernel", "16384x16384x16384", "f16"): {
+        "bytes": 18260333568 + 1103571712, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
+        "sha256": "8d1968c394593bfd009d17f5e7fd973d9745ffc862c1a1d0bf45dbe54b790fbb"},
 }
 
 

@@ -198,38 +198,47 @@ cudaError_t launch_splitk_reduce(const GemmArgs& a, int splits, const float* par
 
 // ---------------------------------------------------------------- 16-bit operand repack (aligned leading dimension)
 
-// One warp per column segment of up to 2048 elements: lanes walk it two elements at a time (two 2-byte loads, one
-// 4-byte store), so both the unaligned source column and the aligned destination column are touched in contiguous
-// 64 / 128-byte pieces.  Rows rows..ld_out-1 of the copy are zero.
-constexpr int REPACK_SEG = 2048;
-
+// One thread per 16-byte chunk (8 elements) of the aligned copy.  A chunk that lies wholly inside its column is read
+// as 32-bit words: four when its first source element sits on a 4-byte boundary, otherwise five, shifted by one
+// element with byte permutes (columns of odd length alternate between the two cases).  Chunks at the end of a column,
+// the last column (whose fifth word could lie beyond the matrix) and the very first chunk go element by element; rows rows..ld_out-1 of
+// the copy are zero.
 __global__ void __launch_bounds__(256)
 repack16_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld, uint16_t* __restrict__ dst,
                 int64_t ld_out) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const int64_t segs = (ld_out + REPACK_SEG - 1) / REPACK_SEG;
-    for (int64_t u = warp; u < cols * segs; u += nwarps) {
-        const int64_t j = u / segs, i0 = (u % segs) * REPACK_SEG;
-        const int64_t i1 = min(ld_out, i0 + REPACK_SEG);
-        const uint16_t* sp = src + j * ld;
-        uint32_t* dp = reinterpret_cast<uint32_t*>(dst + j * ld_out);      // ld_out is a multiple of 8 elements
-        for (int64_t i = i0 + 2 * lane; i < i1; i += 64) {
-            const uint32_t lo = (i < rows) ? sp[i] : 0u;
-            const uint32_t hi = (i + 1 < rows) ? sp[i + 1] : 0u;
-            dp[i >> 1] = lo | (hi << 16);
+    const int64_t chunks = ld_out / 8;                      // per column (ld_out is a multiple of 8)
+    const int64_t total = chunks * cols;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t j = u / chunks, i0 = (u - j * chunks) * 8;
+        const uint16_t* sp = src + j * ld + i0;
+        uint4 out;
+        if (i0 + 8 <= rows && j + 1 < cols && u > 0) {      // (u == 0: the word below the first element may lie before the matrix)
+            const uintptr_t addr = reinterpret_cast<uintptr_t>(sp);
+            const uint32_t* w = reinterpret_cast<const uint32_t*>(addr & ~(uintptr_t)3);
+            if ((addr & 2) == 0) {
+                out = make_uint4(__ldg(w), __ldg(w + 1), __ldg(w + 2), __ldg(w + 3));
+            } else {                                        // the chunk starts in the upper half of w[0]
+                const uint32_t a = __ldg(w), b = __ldg(w + 1), c = __ldg(w + 2), d = __ldg(w + 3), e = __ldg(w + 4);
+                out = make_uint4(__byte_perm(a, b, 0x5432), __byte_perm(b, c, 0x5432), __byte_perm(c, d, 0x5432),
+                                 __byte_perm(d, e, 0x5432));
+            }
+        } else {
+            uint32_t h[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) h[t] = (i0 + t < rows) ? (uint32_t)sp[t] : 0u;
+            out = make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16));
         }
+        *reinterpret_cast<uint4*>(dst + j * ld_out + i0) = out;
     }
 }
 
 cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t ld, void* dst, int64_t ld_out,
                             cudaStream_t stream) {
-    const int64_t units = cols * ((ld_out + REPACK_SEG - 1) / REPACK_SEG);
-    int64_t blocks = (units + 7) / 8;                   // 8 warps per block
-    const int64_t cap = (int64_t)sm_count() * 64;
+    const int64_t total = (ld_out / 8) * cols;
+    if (total <= 0) return cudaSuccess;
+    int64_t blocks = (total + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 32;
     if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
     repack16_kernel<<<(unsigned)blocks, 256, 0, stream>>>((const uint16_t*)src, rows, cols, ld, (uint16_t*)dst, ld_out);
     return cudaGetLastError();
 }
