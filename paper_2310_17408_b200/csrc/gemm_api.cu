@@ -740,7 +740,7 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     if (traffic > 32e6 && n >= 1024) panel = host_panel_columns(input_dtype(dtype), m, n, st->sms);
     if (panel > n) panel = n;
     const int np = (int)ceil_div(n, panel);
-    // While A itself is still arriving, the first column panel is computed k panel by k panel (the order of the
+    // While A itself is still arriving, the leading column panels are computed k panel by k panel (the order of the
     // paper's loop L2 around the packing of A, Fig. 1: C accumulates over blocks of k): each step needs only the part
     // of A that has arrived, runs on whole tiles of C, and adds onto what the earlier steps left in C.
     int64_t kpanel = k;
@@ -773,52 +773,93 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
         chk(cudaStreamWaitEvent(pipe->in, ev_alloc, 0));
         chk(cudaStreamWaitEvent(pipe->out, ev_alloc, 0));
     }
-    for (int p = 0; p < np && e == cudaSuccess && rc == GEMM_OK; ++p) {
-        const int64_t j0 = (int64_t)p * panel, cols = (n - j0 < panel) ? n - j0 : panel;
-        cudaEvent_t ev_in = ev[3 + 2 * p], ev_mul = ev[4 + 2 * p];
-        const char* hB = static_cast<const char*>(B_host);
-        char* dBp = static_cast<char*>(dB);
-        const size_t b_off = needs_ab ? (tb ? (size_t)j0 * es : (size_t)j0 * ldb * es) : 0;
+    const char* hB = static_cast<const char*>(B_host);
+    char* dBp = static_cast<char*>(dB);
+    auto cols_of = [&](int p) { const int64_t j0 = (int64_t)p * panel; return (n - j0 < panel) ? n - j0 : panel; };
+    auto b_off_of = [&](int p) { const int64_t j0 = (int64_t)p * panel; return needs_ab ? (tb ? (size_t)j0 * es : (size_t)j0 * ldb * es) : (size_t)0; };
+    auto c_off_of = [&](int p) { return (size_t)((int64_t)p * panel) * ldc * es_c; };
+    // panel p of op(B) and (if it is read) of C to the device; ev[3 + 2p] marks their arrival
+    auto send_panel = [&](int p) {
+        const int64_t cols = cols_of(p);
+        const size_t b_off = b_off_of(p), c_off = c_off_of(p);
         if (needs_ab) {
             if (tb) chk(copy_window(dBp + b_off, hB + b_off, cols, k, ldb, es, cudaMemcpyHostToDevice, pipe->in));
             else chk(copy_window(dBp + b_off, hB + b_off, k, cols, ldb, es, cudaMemcpyHostToDevice, pipe->in));
         }
-        const size_t c_off = (size_t)j0 * ldc * es_c;
         // only the m x cols window of C travels: the host's padding rows are never touched
         if (beta != 0.0f)
             chk(copy_window(static_cast<char*>(dC) + c_off, static_cast<const char*>(C_host) + c_off, m, cols, ldc, es_c,
                             cudaMemcpyHostToDevice, pipe->in));
-        chk(cudaEventRecord(ev_in, pipe->in));
-        chk(cudaStreamWaitEvent(s, ev_in, 0));
-        if (e != cudaSuccess) break;
-        if (p == 0 && needs_ab) {
-            // A follows the first panel of B and C; the first panel is multiplied k panel by k panel as A arrives
-            for (int q = 0; q < nk && e == cudaSuccess && rc == GEMM_OK; ++q) {
-                const int64_t p0 = (int64_t)q * kpanel, kk = (k - p0 < kpanel) ? k - p0 : kpanel;
-                // columns p0.. of op(A): whole columns of the stored matrix (transA = N) or a row window of it (T)
-                const size_t a_off = ta ? (size_t)p0 * es : (size_t)p0 * lda * es;
-                char* dAp = static_cast<char*>(dA) + a_off;
-                const char* hAp = static_cast<const char*>(A_host) + a_off;
-                if (ta) chk(copy_window(dAp, hAp, kk, m, lda, es, cudaMemcpyHostToDevice, pipe->in));
-                else chk(copy_window(dAp, hAp, m, kk, lda, es, cudaMemcpyHostToDevice, pipe->in));
-                cudaEvent_t ev_k = ev[3 + 2 * np + q];
-                chk(cudaEventRecord(ev_k, pipe->in));
-                chk(cudaStreamWaitEvent(s, ev_k, 0));
-                if (e != cudaSuccess) break;
-                // rows p0.. of op(B) inside this panel: a row window of the stored matrix (transB = N) or whole columns (T)
-                const size_t bk_off = tb ? (size_t)p0 * ldb * es : (size_t)p0 * es;
-                rc = gemm(dtype, transA, transB, m, cols, kk, alpha, dAp, lda, dBp + b_off + bk_off, ldb, q == 0 ? beta : 1.0f,
-                          static_cast<char*>(dC) + c_off, ldc, stream);
-            }
-        } else {
-            rc = gemm(dtype, transA, transB, m, cols, k, alpha, dA, lda, needs_ab ? dBp + b_off : nullptr, ldb, beta,
-                      static_cast<char*>(dC) + c_off, ldc, stream);
-        }
-        if (rc != GEMM_OK || e != cudaSuccess) break;
-        chk(cudaEventRecord(ev_mul, s));
-        chk(cudaStreamWaitEvent(pipe->out, ev_mul, 0));
-        chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols, ldc, es_c,
+        chk(cudaEventRecord(ev[3 + 2 * p], pipe->in));
+    };
+    // panel p back to the host once the multiplications enqueued so far are done
+    auto return_panel = [&](int p) {
+        const size_t c_off = c_off_of(p);
+        chk(cudaEventRecord(ev[4 + 2 * p], s));
+        chk(cudaStreamWaitEvent(pipe->out, ev[4 + 2 * p], 0));
+        chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols_of(p), ldc, es_c,
                         cudaMemcpyDeviceToHost, pipe->out));
+    };
+    // k panel q of A times the matching rows of panel p of op(B), added onto panel p of C
+    auto k_step = [&](int q, int p) {
+        const int64_t p0 = (int64_t)q * kpanel, kk = (k - p0 < kpanel) ? k - p0 : kpanel;
+        const size_t a_off = ta ? (size_t)p0 * es : (size_t)p0 * lda * es;          // columns p0.. of op(A)
+        const size_t bk_off = tb ? (size_t)p0 * ldb * es : (size_t)p0 * es;          // rows p0.. of op(B)
+        chk(cudaStreamWaitEvent(s, ev[3 + 2 * np + q], 0));
+        chk(cudaStreamWaitEvent(s, ev[3 + 2 * p], 0));
+        if (e != cudaSuccess || rc != GEMM_OK) return;
+        rc = gemm(dtype, transA, transB, m, cols_of(p), kk, alpha, static_cast<char*>(dA) + a_off, lda,
+                  dBp + b_off_of(p) + bk_off, ldb, q == 0 ? beta : 1.0f, static_cast<char*>(dC) + c_off_of(p), ldc, stream);
+    };
+
+    // Phase 1, while A arrives (k panel by k panel, after the first panel of B and C): the first `lead` column panels
+    // are multiplied k panel by k panel, enough of them that the arithmetic lasts about as long as A's transfer; the
+    // later ones of them join when their B and C have arrived, catching up on the k panels that are already there.
+    int lead = 0;
+    if (needs_ab) {
+        lead = 1;
+        if (nk > 1) {
+            const double t_a = (double)a_bytes / 50e9;
+            const double rate = input_dtype(dtype) == GEMM_F32 ? 5.0e13 : 1.2e15;
+            const double t_panel = 2.0 * (double)m * (double)panel * (double)k / rate;
+            lead = (int)(t_a / t_panel + 0.999);
+            if (lead > np - 1) lead = np - 1;
+            if (lead > nk) lead = nk;
+            if (lead < 1) lead = 1;
+        }
+        send_panel(0);
+        int joined = 1;
+        for (int q = 0; q < nk && e == cudaSuccess && rc == GEMM_OK; ++q) {
+            const int64_t p0 = (int64_t)q * kpanel, kk = (k - p0 < kpanel) ? k - p0 : kpanel;
+            const size_t a_off = ta ? (size_t)p0 * es : (size_t)p0 * lda * es;
+            char* dAp = static_cast<char*>(dA) + a_off;
+            const char* hAp = static_cast<const char*>(A_host) + a_off;
+            if (ta) chk(copy_window(dAp, hAp, kk, m, lda, es, cudaMemcpyHostToDevice, pipe->in));
+            else chk(copy_window(dAp, hAp, m, kk, lda, es, cudaMemcpyHostToDevice, pipe->in));
+            chk(cudaEventRecord(ev[3 + 2 * np + q], pipe->in));
+            for (int p = 0; p < joined; ++p) k_step(q, p);
+            // the next lead panel follows this k panel on the wire when its turn has come (evenly spread over A's transfer)
+            if (joined < lead && (q + 1) * lead >= joined * nk) {
+                send_panel(joined);
+                for (int qq = 0; qq <= q; ++qq) k_step(qq, joined);
+                ++joined;
+            }
+        }
+        for (int p = joined; p < lead && e == cudaSuccess && rc == GEMM_OK; ++p) {      // (only if nk < lead, which the clamp rules out)
+            send_panel(p);
+            for (int q = 0; q < nk; ++q) k_step(q, p);
+        }
+        for (int p = 0; p < lead && e == cudaSuccess && rc == GEMM_OK; ++p) return_panel(p);
+    }
+    // Phase 2: A is resident; the remaining panels flow through copy in / multiply / copy out
+    for (int p = lead; p < np && e == cudaSuccess && rc == GEMM_OK; ++p) {
+        send_panel(p);
+        chk(cudaStreamWaitEvent(s, ev[3 + 2 * p], 0));
+        if (e != cudaSuccess) break;
+        rc = gemm(dtype, transA, transB, m, cols_of(p), k, alpha, dA, lda, needs_ab ? dBp + b_off_of(p) : nullptr, ldb, beta,
+                  static_cast<char*>(dC) + c_off_of(p), ldc, stream);
+        if (rc != GEMM_OK) break;
+        return_panel(p);
     }
     cudaEventRecord(ev_done, pipe->out);                     // the caller's stream rejoins both copy streams
     cudaStreamWaitEvent(s, ev_done, 0);
