@@ -472,6 +472,41 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip) {
         ws = static_cast<uint8_t*>(ws) + ws_skip;
         ws_bytes -= ws_skip;
     }
+    // 16-bit inputs with at most 64 rows of C and many columns (the C_out = 64 layers): a 128-row MMA would run half
+    // empty and only half of the epilogue warps would have rows to store.  Exchange the roles of the operands instead:
+    // C^T = op(B)^T op(A)^T, the columns of C (pixels) become the 128 rows of the MMA, its 64 rows the MMA's N, and a
+    // lane of the epilogue writes consecutive floats of its column of C.
+    if (a.dtype != GEMM_F32 && !a.conv && !a.out16 && !a.acc16 && a.m <= 64 && a.n >= 1024 && g_force_tile_m == 0 &&
+        g_force_tile_n == 0 && g_force_split == 0 && g_force_kernel != GEMM_KERNEL_SIMT_GENERIC) {
+        GemmArgs x = a;
+        x.m = a.n; x.n = a.m;
+        x.A = a.B; x.lda = a.ldb; x.ta = !a.tb;
+        x.B = a.A; x.ldb = a.lda; x.tb = !a.ta;
+        x.ct = 1;
+        Plan px = make_plan(x, st->sms, ws_bytes);
+        if (px.kernel == GEMM_KERNEL_TENSOR && px.tile == 64 && px.ks.splits == 1 && !px.pair) {
+            uint8_t* w = static_cast<uint8_t*>(ws);
+            if (px.repack_a) {
+                const int64_t rows = x.ta ? x.k : x.m, cols = x.ta ? x.m : x.k;
+                e = launch_repack16(x.A, rows, cols, x.lda, w, px.lda_p, x.stream);
+                if (e != cudaSuccess) return fail_launch(e);
+                x.A = w; x.lda = px.lda_p;
+                w += round_up(px.lda_p * cols * 2, 256);
+                cfg.repacked |= 2; cfg.launches++;      // (the caller's B)
+            }
+            if (px.repack_b) {
+                const int64_t rows = x.tb ? x.n : x.k, cols = x.tb ? x.k : x.n;
+                e = launch_repack16(x.B, rows, cols, x.ldb, w, px.ldb_p, x.stream);
+                if (e != cudaSuccess) return fail_launch(e);
+                x.B = w; x.ldb = px.ldb_p;
+                cfg.repacked |= 1; cfg.launches++;      // (the caller's A)
+            }
+            e = launch_tensor(x, 64, px.ks, nullptr, &cfg, false);
+            std::swap(cfg.tile_m, cfg.tile_n);           // reported in the caller's orientation
+            t_last_cfg = cfg;
+            return e == cudaSuccess ? GEMM_OK : fail_launch(e);
+        }
+    }
     Plan p = make_plan(a, st->sms, ws_bytes);
     if (p.kernel < 0) return GEMM_ERR_WORKSPACE;
 
@@ -509,6 +544,13 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip) {
     if (p.kernel == GEMM_KERNEL_TENSOR) {
         e = p.pair ? launch_tensor_pair(a, p.ks, partials, &cfg)
                    : launch_tensor(a, p.tile, p.ks, partials, &cfg, p.cluster_reduce);
+        if (e != cudaSuccess && p.cluster_reduce) {      // as below for the fp32 kernel: without the cluster, k unsplit
+            (void)cudaGetLastError();
+            p.cluster_reduce = false;
+            p.ks = make_split(a.k, 1, 64);
+            partials = nullptr;
+            e = launch_tensor(a, p.tile, p.ks, nullptr, &cfg, false);
+        }
     } else if (p.tail_splits > 1) {
         TailSplit tail{p.tail_first, p.tail_splits, p.tail_chunk, reinterpret_cast<float*>(wsp)};
         e = launch_simt_fast(a, p.tile, p.ks, nullptr, &cfg, tail);
@@ -517,6 +559,13 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip) {
         cfg.tail_split = p.tail_splits;
     } else {
         e = launch_simt_fast(a, p.tile, p.ks, partials, &cfg, TailSplit{0x7FFFFFFF, 1, 0, nullptr}, p.cluster_reduce);
+        if (e != cudaSuccess && p.cluster_reduce) {
+            // the device would not take the cluster (a restricted context, say): the same tile, k unsplit
+            (void)cudaGetLastError();
+            p.cluster_reduce = false;
+            p.ks = make_split(a.k, 1, 16);
+            e = launch_simt_fast(a, p.tile, p.ks, nullptr, &cfg);
+        }
     }
     if (e == cudaSuccess && p.ks.splits > 1 && !p.cluster_reduce) {
         e = launch_splitk_reduce(a, p.ks.splits, partials);

@@ -32,6 +32,8 @@ struct GemmArgs {
     const ConvIndex* conv = nullptr;   // non-null: op(B) is the lowered activation matrix of this layer (B, ldb, tb unused)
     int out16 = 0;                     // element type of C: 0 = fp32, GEMM_F16 / GEMM_BF16 = that 16-bit type (C then points to it)
     int acc16 = 0;                     // binary16 inputs, binary16 accumulation on the tensor cores, binary16 result (GEMM_F16_ACC16)
+    int ct = 0;                        // tensor kernels: the roles of the operands were exchanged; C (m x n here) is stored as its
+                                       // transpose: element (i, j) at C[j + i*ldc]
     int split3 = 0;                    // fp32 operands: multiply on the tensor cores as three bfloat16 pieces each (GEMM_F32_TC)
 };
 

@@ -262,6 +262,81 @@ __device__ __forceinline__ void epilogue_tile(uint32_t tmem_acc, int64_t row0, i
     if (!released) release_acc();
 }
 
+// The epilogue when the roles of the operands were exchanged (C^T = op(B)^T op(A)^T is what the kernel computes: its
+// rows are the columns of the caller's C).  Lane = tile row = one column of C, so the 32 tile columns of a chunk are 32
+// consecutive floats of that column: each lane scales and stores them itself, four at a time, without staging.
+// `m`, `n` are the kernel's extents (rows = columns of C); element (row, col) of the tile lives at out[col + row*ldo].
+template <int BN, int STORE_BUFS, typename Release>
+__device__ __forceinline__ void epilogue_tile_ct(uint32_t tmem_acc, int64_t row0, int64_t n0, int half, int lane,
+                                                 int64_t m, int64_t n, float alpha, float beta, float* out, int64_t ldo,
+                                                 bool via_tma, const CUtensorMap* tmC, float* stage, uint32_t& sbuf,
+                                                 Release&& release_acc) {
+    const int64_t row = row0 + lane;
+    bool released = false;
+    if (row0 < m) {
+        const bool vec = (reinterpret_cast<uintptr_t>(out) & 15) == 0 && ldo % 4 == 0;
+#pragma unroll 1
+        for (int c = half; c < BN / 32; c += 2) {
+            const int64_t col0 = n0 + c * 32;
+            if (col0 >= n) break;
+            const bool last_chunk = (c + 2 >= BN / 32) || (col0 + 64 >= n);
+            uint32_t v[32];
+            tmem_ld32(tmem_acc + c * 32, v);
+            tmem_ld_wait();
+            if (last_chunk) { release_acc(); released = true; }
+            float* r = reinterpret_cast<float*>(v);
+            float* cp = out + col0 + row * ldo;
+            if (alpha != 1.0f || beta != 0.0f) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    r[j] *= alpha; r[j + 1] *= alpha; r[j + 2] *= alpha; r[j + 3] *= alpha;
+                    if (beta != 0.0f && row < m) {
+                        if (vec && col0 + j + 4 <= n) {
+                            const float4 c0 = *reinterpret_cast<const float4*>(cp + j);
+                            r[j] = fmaf(beta, c0.x, r[j]); r[j + 1] = fmaf(beta, c0.y, r[j + 1]);
+                            r[j + 2] = fmaf(beta, c0.z, r[j + 2]); r[j + 3] = fmaf(beta, c0.w, r[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                if (col0 + j + u < n) r[j + u] = fmaf(beta, cp[j + u], r[j + u]);
+                        }
+                    }
+                }
+            }
+            if (via_tma) {
+                // staging tile [32 tile rows][32 floats] in the 128-byte-swizzled layout the store's tensor map names:
+                // 16-byte chunk q of row l sits at chunk position q ^ (l % 8), which also spreads a warp's 16-byte
+                // stores over all banks; the bulk store writes 32 columns of C x 32 floats and clips at the edges
+                if (lane == 0) bulk_wait_read<STORE_BUFS - 1>();
+                __syncwarp();
+                uint8_t* st = reinterpret_cast<uint8_t*>(stage + sbuf * (32 * 32));
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<float4*>(st + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                        make_float4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(tmC, smem_u32(st), (int32_t)col0, (int32_t)row0);
+                    bulk_commit();
+                }
+                sbuf = (sbuf + 1 == (uint32_t)STORE_BUFS) ? 0 : sbuf + 1;
+            } else if (row < m) {
+                if (vec && col0 + 32 <= n) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4*>(cp + j) = make_float4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (col0 + j < n) cp[j] = r[j];
+                }
+            }
+        }
+    }
+    if (!released) release_acc();
+}
+
 // The same for a 16-bit result (out16 = GEMM_F16 or GEMM_BF16; never for split-k partial sums): `out` and tmC are
 // in that type and alpha*acc + beta*C0 is rounded once, to nearest even, at the store.  Two rows of one column are
 // packed into a 32-bit word before they go to the staging tile: every lane converts its values of a column pair
@@ -356,6 +431,9 @@ bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_
 bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits);
 // map over the result (fp32, or the 16-bit type out16) for the epilogue's tile stores: 32 x 32 boxes, no swizzle
 bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_t ldc, int out16);
+// map over an fp32 C for the tile stores of the exchanged-roles epilogue: dim0 = rows of C (contiguous), dim1 = columns
+// (stride ldc), boxes of 32 x 32 in the 128-byte-swizzled shared-memory layout
+bool make_ct_map(CUtensorMap* tm, const float* base, int64_t c_rows, int64_t c_cols, int64_t ldc);
 // whether C (of either element size) can be written by TMA tile stores: 16-byte aligned base and column stride, and
 // columns whose m elements end on a 16-byte boundary.  The last condition keeps the rows m..ldc-1 untouched: a tile
 // store that is clipped at the matrix edge was seen to write the whole 16-byte unit the edge falls into (binary16

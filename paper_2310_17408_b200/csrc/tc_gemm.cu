@@ -86,7 +86,8 @@ __device__ __noinline__ void cluster_sum_tile(uint32_t park_addr, int S, int64_t
 }
 
 // OUT: 0 = fp32 result; 1 = 16-bit result (fp32 accumulator, one rounding at the store); 2 = binary16 accumulator
-// and binary16 result (the paper's all-f16 arithmetic, Section III-D)
+// and binary16 result (the paper's all-f16 arithmetic, Section III-D); 3 = fp32 result stored transposed (the host
+// exchanged the roles of the operands: C is ldc-strided along the tile's rows and contiguous along its columns)
 template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -95,7 +96,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                uint32_t idesc, uint32_t* status, const ConvTma conv, int out16, int cluster_k) {
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
-    constexpr bool OUT16 = OUT != 0, ACC16 = OUT == 2;
+    constexpr bool OUT16 = OUT == 1 || OUT == 2, ACC16 = OUT == 2, CT = OUT == 3;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -301,6 +302,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 continue;
             }
             bool done = false;
+            if constexpr (CT) {
+                epilogue_tile_ct<BN, Cfg::STORE_BUFS>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, C, ldc,
+                                                      store_via_tma == 3, &tmC, stage, sbuf, release);
+                done = true;
+            }
             if constexpr (OUT16) {
                 if (!raw) {      // 16-bit result: one rounding at the store (split-k partial sums stay fp32)
                     epilogue_tile16<BN, Cfg::STORE_BUFS, ACC16>(tacc, row0, (int64_t)tn * BN, half, lane, m, n, alpha, beta, out, ldc,
@@ -468,6 +474,22 @@ bool make_c_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int64_
     });
 }
 
+bool make_ct_map(CUtensorMap* tm, const float* base, int64_t c_rows, int64_t c_cols, int64_t ldc) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const MapKey k{{4, 0, (uint64_t)(uintptr_t)base, (uint64_t)c_rows, (uint64_t)c_cols, (uint64_t)ldc, 0}};
+    return cached_map(tm, k, [&](CUtensorMap* out) {
+        cuuint64_t dims[2] = {(cuuint64_t)c_rows, (cuuint64_t)c_cols};
+        cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+        cuuint32_t box[2] = {32, 32};
+        cuuint32_t estr[2] = {1, 1};
+        CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r == CUDA_SUCCESS;
+    });
+}
+
 typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -598,12 +620,19 @@ static cudaError_t launch_tc_bn(const GemmArgs& a, int tile_n, KSplit ks, float*
     // the result goes out through TMA tile stores when C is 16-byte addressable and this is not a split-k pass
     CUtensorMap tmC = tmA;
     int store_via_tma = 0;
-    if (ks.splits == 1 && c_tma_addressable(a.C, a.m, a.ldc, a.out16))
+    if (!a.ct && ks.splits == 1 && c_tma_addressable(a.C, a.m, a.ldc, a.out16))
         store_via_tma = make_c_map(&tmC, a.C, a.m, a.n, a.ldc, a.out16) ? 1 : 0;
     if (ks.splits > 1 && !cluster && (reinterpret_cast<uintptr_t>(partials) & 15) == 0 && a.m % 4 == 0 &&
         a.m * a.n * 4 < (1LL << 40))
         store_via_tma = make_partials_map(&tmC, partials, a.m, a.n, ks.splits) ? 2 : 0;
     if constexpr (!CONV) {
+        if (a.ct) {      // operands exchanged by the host: n (the caller's m) is at most 64, C goes out transposed
+            if (tile_n != 64 || ks.splits != 1 || a.out16) return cudaErrorInvalidConfiguration;
+            // here a.n is the row count of the caller's C and a.m its column count; tile stores when C is 16-byte addressable
+            int ct_store = 0;
+            if (c_tma_addressable(a.C, a.n, a.ldc, 0) && make_ct_map(&tmC, a.C, a.n, a.m, a.ldc)) ct_store = 3;
+            return launch_tc<64, A_MN, B_MN, false, 3>(a, ks, partials, cfg, tmA, tmB, tmC, ct_store);
+        }
         if (a.acc16) {      // binary16 accumulator (never split along k: partial sums would need a wider type)
             switch (tile_n) {
                 case 256: return launch_tc<256, A_MN, B_MN, false, 2>(a, ks, partials, cfg, tmA, tmB, tmC, store_via_tma);

@@ -391,3 +391,28 @@ def test_nothing_is_written_outside_the_m_by_n_window(api_dtype):
         assert np.array_equal(body[:, :m], want.T), (m, n, k, ldc)
         assert np.all(body[:, m:] == 7.0), "rows m..ldc-1 were written"
         assert np.all(host[:guard] == 7.0) and np.all(host[guard + ldc * n:] == 7.0), "written outside the buffer of C"
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+@pytest.mark.parametrize("ta,tb", TRANS)
+def test_few_rows_many_columns_take_the_exchanged_operand_roles(dtype, ta, tb):
+    """16-bit inputs, at most 64 rows of C, many columns (the C_out = 64 layers): the library computes C^T = op(B)^T op(A)^T
+    with the columns of C as the rows of the MMA.  Ragged sizes, padded and unaligned leading dimensions (C then takes
+    the scalar stores, the operands the aligned copy), alpha / beta, exact integers."""
+    ensure_workspace(64 << 20)
+    for (m, n, k), pad in [((64, 2048, 128), (0, 0, 0)), ((64, 1500, 200), (0, 0, 0)), ((17, 4100, 70), (8, 8, 4)),
+                           ((1, 1024, 64), (0, 0, 3)), ((40, 1100, 147), (1, 1, 1))]:
+        for kind, alpha, beta in [("int", 1.5, 0.5), ("normal", 1.0, 0.0), ("normal", -0.75, 1.25)]:
+            p = problem(dtype, m, n, k, ta, tb, alpha, beta, kind, pad, seed=n + k)
+            A, B, C0 = p.operands()
+            C, cfg = run_problem(p, A, B, C0)
+            assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and (cfg["tile_m"], cfg["tile_n"]) == (64, 128), cfg
+            check_against_oracle(p, A, B, C0, C, integer=(kind == "int"))
+    # a forced tile keeps the operands' roles: same result within the tolerance, the other kernel
+    p = problem(dtype, 64, 2048, 256, ta, tb, 1.0, 0.0, "int", (0, 0, 0), seed=5)
+    A, B, C0 = p.operands()
+    C1, cfg1 = run_problem(p, A, B, C0)
+    g.gemm_force_tile(128, 256, 0)
+    C2, cfg2 = run_problem(p, A, B, C0)
+    assert (cfg1["tile_m"], cfg1["tile_n"]) == (64, 128) and (cfg2["tile_m"], cfg2["tile_n"]) == (128, 256)
+    assert np.array_equal(C1.buf.view(np.uint32), C2.buf.view(np.uint32))
