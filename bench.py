@@ -36,6 +36,8 @@ FP32_LANES_PER_SM = 128
 WORKLOADS = {
     "cfg2_fp32_squares": lambda: config_problems(2),
     "cfg1_fp32_512": lambda: config_problems(1),
+    # config 2 through GEMM_F32_TC: fp32 data on the tensor cores as three bfloat16 pieces per entry (not IEEE fp32 arithmetic)
+    "cfg2_fp32_tc": lambda: [__import__("dataclasses").replace(p, name=p.name + "_tc", tc3=True) for p in config_problems(2)],
     "cfg3_fp32_im2row": lambda: config_problems(3),
     "cfg4_fp32_nonsquarish": lambda: config_problems(4),
     "cfg5_f16": lambda: config_problems(5, dtype=DTYPE_F16),
@@ -197,7 +199,12 @@ def aggregate_throughput(flops_per_rank_step, step_ms_max, world):
 def roofline_class(p, peaks):
     """(bound, peak, unit, algorithmic amount) of one problem: the slower of compute and HBM time decides."""
     t_hbm = p.algorithmic_bytes() / (peaks["hbm_gbs"] * 1e9)
-    if p.dtype == DTYPE_F32:
+    if getattr(p, "tc3", False):
+        # six bfloat16 products per fp32 product: the tensor peak counts a sixth in fp32-equivalent flops
+        peak_c = peaks["tensor_tflops"] / 6.0
+        if p.flops / (peak_c * 1e12) >= t_hbm:
+            return "tensor", peak_c, "TFLOP/s", p.flops / 1e12
+    elif p.dtype == DTYPE_F32:
         peak_c = fp32_alu_peak_tflops(peaks["sm_max_mhz"])
         t_cmp = p.flops / (peak_c * 1e12)
         if t_cmp >= t_hbm:

@@ -4,15 +4,16 @@
 // from global memory into registers (128-bit loads through the read-only path where alignment allows; L1 serves
 // the reuse between neighbouring threads).  No shared memory, no barrier, no workspace, no reduction pass: one
 // launch whose length is one thread's k loop, which is what matters when the whole problem is a few microseconds
-// of work.  blockIdx.y is the problem index of a strided batch.
+// of work.  The unit of work is a 32 x 16 slab of one problem's C, one warp each; the slabs of all problems of a
+// strided batch are numbered through, so that small problems share CTAs instead of leaving warps idle.
 #include "internal.cuh"
 
 namespace b200gemm {
 
 constexpr int DT = 4;                 // thread tile (DT x DT)
-constexpr int D_WARP_M = 8;           // threads of a warp along m (x 4 along n): a warp covers 32 x 16 of C
-constexpr int D_WARPS = 4;            // warps per CTA, stacked along n: CTA tile 32 x 64
-constexpr int D_TILE_M = D_WARP_M * DT, D_TILE_N = 4 * DT * D_WARPS;
+constexpr int D_WARP_M = 8;           // threads of a warp along m (x 4 along n): a warp covers a 32 x 16 slab of C
+constexpr int D_WARPS = 4;            // warps per CTA; every warp takes the next slab of the whole batch
+constexpr int D_TILE_M = D_WARP_M * DT, D_TILE_N = 4 * DT;      // slab extents
 
 // four consecutive k of one row (KCONT) or four consecutive rows at one k (!KCONT) of a stored matrix
 template <bool VEC>
@@ -34,17 +35,19 @@ template <bool TA, bool TB, bool VEC>
 __global__ void __launch_bounds__(32 * D_WARPS)
 simt_direct_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __restrict__ A, int64_t lda, int64_t strideA,
                    const float* __restrict__ B, int64_t ldb, int64_t strideB, float beta, float* __restrict__ C,
-                   int64_t ldc, int64_t strideC, int tiles_m) {
+                   int64_t ldc, int64_t strideC, int tiles_m, int64_t slabs_per_problem, int64_t total_slabs) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t tm = blockIdx.x % tiles_m, tn = blockIdx.x / tiles_m;
+    const int64_t slab = (int64_t)blockIdx.x * D_WARPS + warp;
+    const int64_t problem = slab / slabs_per_problem, within = slab - problem * slabs_per_problem;
+    const int64_t tm = within % tiles_m, tn = within / tiles_m;
     const int64_t i0 = tm * D_TILE_M + (lane % D_WARP_M) * DT;
-    const int64_t j0 = tn * D_TILE_N + (warp * 4 + lane / D_WARP_M) * DT;
-    A += (int64_t)blockIdx.y * strideA;
-    B += (int64_t)blockIdx.y * strideB;
-    C += (int64_t)blockIdx.y * strideC;
+    const int64_t j0 = tn * D_TILE_N + (lane / D_WARP_M) * DT;
+    A += problem * strideA;
+    B += problem * strideB;
+    C += problem * strideC;
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (i0 >= m || j0 >= n) return;
+    if (slab >= total_slabs || i0 >= m || j0 >= n) return;
 
     float acc[DT][DT];      // [column][row]
 #pragma unroll
@@ -169,10 +172,10 @@ simt_direct_kernel(int64_t m, int64_t n, int64_t k, float alpha, const float* __
 }
 
 template <bool TA, bool TB, bool VEC>
-static cudaError_t launch_direct_t(const GemmArgs& a, int64_t sA, int64_t sB, int64_t sC, int64_t batch, int64_t tiles_m,
-                                   int64_t tiles) {
+static cudaError_t launch_direct_t(const GemmArgs& a, int64_t sA, int64_t sB, int64_t sC, int64_t tiles_m, int64_t spp,
+                                   int64_t total) {
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3((unsigned)tiles, (unsigned)batch, 1);
+    lc.gridDim = dim3((unsigned)((total + D_WARPS - 1) / D_WARPS), 1, 1);
     lc.blockDim = dim3(32 * D_WARPS);
     lc.stream = a.stream;
     cudaLaunchAttribute attr[1];
@@ -181,26 +184,29 @@ static cudaError_t launch_direct_t(const GemmArgs& a, int64_t sA, int64_t sB, in
     lc.attrs = attr;
     lc.numAttrs = 1;
     cudaError_t le = cudaLaunchKernelEx(&lc, simt_direct_kernel<TA, TB, VEC>, a.m, a.n, a.k, a.alpha, (const float*)a.A, a.lda, sA,
-                                        (const float*)a.B, a.ldb, sB, a.beta, a.C, a.ldc, sC, (int)tiles_m);
+                                        (const float*)a.B, a.ldb, sB, a.beta, a.C, a.ldc, sC, (int)tiles_m, spp, total);
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 cudaError_t launch_simt_direct(const GemmArgs& a, int64_t strideA, int64_t strideB, int64_t strideC, int64_t batch,
                                gemm_config_t* cfg) {
     const int64_t tiles_m = (a.m + D_TILE_M - 1) / D_TILE_M, tiles_n = (a.n + D_TILE_N - 1) / D_TILE_N;
-    const int64_t tiles = tiles_m * tiles_n;
-    if (tiles > 0x7FFFFFFFLL || tiles_m > 0x7FFFFFFF || batch < 1 || batch > 65535) return cudaErrorInvalidConfiguration;
+    const int64_t spp = tiles_m * tiles_n;                    // slabs per problem
+    if (batch < 1 || tiles_m > 0x7FFFFFFF || spp > (1LL << 40) / batch) return cudaErrorInvalidConfiguration;
+    const int64_t total = spp * batch;
+    if ((total + D_WARPS - 1) / D_WARPS > 0x7FFFFFFFLL) return cudaErrorInvalidConfiguration;
     auto al = [](const void* p, int64_t ld, int64_t stride) {
         return (reinterpret_cast<uintptr_t>(p) & 15) == 0 && ld % 4 == 0 && stride % 4 == 0;
     };
     const bool vec = al(a.A, a.lda, strideA) && al(a.B, a.ldb, strideB);
     cfg->kernel = GEMM_KERNEL_SIMT_DIRECT;
     cfg->tile_m = D_TILE_M; cfg->tile_n = D_TILE_N; cfg->tile_k = 4; cfg->split_k = 1; cfg->stages = 1;
-    cfg->grid = (int32_t)(tiles * batch > 0x7FFFFFFF ? 0x7FFFFFFF : tiles * batch);
+    const int64_t ctas = (total + D_WARPS - 1) / D_WARPS;
+    cfg->grid = (int32_t)(ctas > 0x7FFFFFFF ? 0x7FFFFFFF : ctas);
     cfg->vector_a = cfg->vector_b = vec ? 4 : 1;
     cfg->launches = 1;
-#define DIRECT(TA_, TB_) (vec ? launch_direct_t<TA_, TB_, true>(a, strideA, strideB, strideC, batch, tiles_m, tiles) \
-                              : launch_direct_t<TA_, TB_, false>(a, strideA, strideB, strideC, batch, tiles_m, tiles))
+#define DIRECT(TA_, TB_) (vec ? launch_direct_t<TA_, TB_, true>(a, strideA, strideB, strideC, tiles_m, spp, total) \
+                              : launch_direct_t<TA_, TB_, false>(a, strideA, strideB, strideC, tiles_m, spp, total))
     if (!a.ta && !a.tb) return DIRECT(false, false);
     if (a.ta && !a.tb) return DIRECT(true, false);
     if (!a.ta && a.tb) return DIRECT(false, true);

@@ -118,24 +118,30 @@ def test_batched_shared_operands_and_scaling_only():
 
 
 def test_batched_beyond_one_launch():
-    # more problems than the batch dimension of one launch holds (65535): two launches.  All problems share A and B
-    # (stride 0) and start from their own C, so one oracle call per distinct C0 value gives every expected result.
+    # more problems than the batch dimension of a grid holds (65535).  All problems share A and B (stride 0) and start
+    # from their own C, so one oracle call per distinct C0 value gives every expected result.  The kernel without
+    # staging numbers its work units through the whole batch (one launch); the staged kernel runs in two launches.
     m, n, k, batch = 4, 4, 8, 70000
     A = make_matrix(m, k, kind="int", seed=1, matrix_id=0)
     B = make_matrix(k, n, kind="int", seed=1, matrix_id=1)
     c0 = (np.arange(batch, dtype=np.float32) % 5.0) - 2.0                  # problem b starts from the constant (b mod 5) - 2
     hC = np.repeat(c0, m * n).astype(np.float32)
-    dA, dB, dC = to_device(A), to_device(B), torch.from_numpy(hC).cuda()
-    rc = g.gemm_strided_batched(DTYPE_F32, "N", "N", m, n, k, 1.0, dA.data_ptr(), m, 0, dB.data_ptr(), k, 0, 0.5,
-                                dC.data_ptr(), m, m * n, batch, torch.cuda.current_stream().cuda_stream)
-    assert rc == 0
-    assert g.gemm_last_config()["launches"] == 2
-    assert g.gemm_poll_status() == 0
-    got = dC.cpu().numpy().reshape(batch, n, m)
-    for v in range(5):
-        C0 = np.full(m * n, v - 2.0, dtype=np.float32)
-        want = oracle.gemm_l0(DTYPE_F32, "N", "N", m, n, k, 1.0, A.buf, m, B.buf, k, 0.5, C0, m, acc=oracle.ACC_F32)
-        assert np.array_equal(got[v::5], np.broadcast_to(want.T, got[v::5].shape))
+    dA, dB = to_device(A), to_device(B)
+    for force, launches in ((g.GEMM_KERNEL_AUTO, 1), (g.GEMM_KERNEL_SIMT_FAST, 2)):
+        dC = torch.from_numpy(hC).cuda()
+        g.gemm_force_kernel(force)
+        rc = g.gemm_strided_batched(DTYPE_F32, "N", "N", m, n, k, 1.0, dA.data_ptr(), m, 0, dB.data_ptr(), k, 0, 0.5,
+                                    dC.data_ptr(), m, m * n, batch, torch.cuda.current_stream().cuda_stream)
+        assert rc == 0
+        cfg = g.gemm_last_config()
+        assert cfg["launches"] == launches, cfg
+        assert cfg["kernel"] == (g.GEMM_KERNEL_SIMT_DIRECT if force == g.GEMM_KERNEL_AUTO else g.GEMM_KERNEL_SIMT_FAST)
+        assert g.gemm_poll_status() == 0
+        got = dC.cpu().numpy().reshape(batch, n, m)
+        for v in range(5):
+            C0 = np.full(m * n, v - 2.0, dtype=np.float32)
+            want = oracle.gemm_l0(DTYPE_F32, "N", "N", m, n, k, 1.0, A.buf, m, B.buf, k, 0.5, C0, m, acc=oracle.ACC_F32)
+            assert np.array_equal(got[v::5], np.broadcast_to(want.T, got[v::5].shape))
 
 
 @pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])

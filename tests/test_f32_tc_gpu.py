@@ -30,7 +30,9 @@ def test_split_precision_against_the_fp64_oracle(ta, tb):
             p = Problem("tc3", DTYPE_F32, m, n, k, alpha, beta, ta, tb, kindA=kind, kindB=kind,
                         kindC=kind if kind == "int" else "uniform", seed=m + k, pad=pad)
             A, B, C0 = p.operands()
+            g.gemm_force_kernel(g.GEMM_KERNEL_TENSOR)      # these sizes are below what the selector sends to the tensor cores
             C, cfg = run_problem(p, A, B, C0, api_dtype=TC)
+            g.gemm_force_kernel(g.GEMM_KERNEL_AUTO)
             assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["launches"] >= 8, cfg      # two splitting passes + six products
             check_against_oracle(p, A, B, C0, C, integer=(kind == "int"))
 
@@ -38,7 +40,7 @@ def test_split_precision_against_the_fp64_oracle(ta, tb):
 def test_split_precision_error_is_at_the_level_of_fp32_arithmetic():
     # the same problem through the exact fp32 kernel and through the three-piece path: both errors against the fp64
     # oracle are reported; the three-piece path must stay within a small multiple of the exact kernel's error
-    p = Problem("tc3e", DTYPE_F32, 1024, 1024, 2048, 1.0, 0.0, seed=9)
+    p = Problem("tc3e", DTYPE_F32, 2048, 1024, 2048, 1.0, 0.0, seed=9)
     A, B, C0 = p.operands()
     ref = oracle.gemm_l1(DTYPE_F32, "N", "N", p.m, p.n, p.k, 1.0, A.buf, A.ld, B.buf, B.ld, 0.0, C0.buf, C0.ld, acc=oracle.ACC_F64)
     C_exact, _ = run_problem(p, A, B, C0)
@@ -53,7 +55,7 @@ def test_split_precision_error_is_at_the_level_of_fp32_arithmetic():
 
 def test_split_precision_falls_back_to_the_exact_kernel():
     # no workspace: the call runs as GEMM_F32; too small to gain: likewise
-    p = Problem("tc3f", DTYPE_F32, 512, 520, 600, 1.5, 0.5, seed=3)
+    p = Problem("tc3f", DTYPE_F32, 1536, 1600, 1700, 1.5, 0.5, seed=3)
     A, B, C0 = p.operands()
     drop_workspace()
     C, cfg = run_problem(p, A, B, C0, workspace=False, api_dtype=TC)
