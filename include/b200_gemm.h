@@ -139,7 +139,7 @@ int gemm_strided_batched(int dtype, char transA, char transB, int64_t m, int64_t
  * Takes device buffers from a memory pool of the library's own (kept between calls; the application's default pool
  * is not touched), then moves column panels of op(B) and C through a three-stream pipeline (copy in / multiply on
  * `stream` / copy out), so that transfers overlap the arithmetic, and synchronises `stream` before returning.  While A
- * itself is still on its way the first panel is multiplied k panel by k panel, each step adding onto C (the order of
+ * itself is still on its way the leading panels are multiplied k panel by k panel, each step adding onto C (the order of
  * the paper's loop L2, Fig. 1): a large result is therefore summed in a different order than gemm() sums it, inside
  * the same error bound (identical on integer-valued data).  Only the m x n window of C is transferred: C is copied
  * in only when beta != 0, and rows m..ldc-1 of the host array are never touched.  Leading dimensions and layout as for

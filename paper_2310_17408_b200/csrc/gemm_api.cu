@@ -733,7 +733,7 @@ static std::mutex g_host_mutex;                     // one gemm_host per process
 
 // columns per panel of C: a multiple of the CTA tile such that the panel's tiles fill whole waves of the GPU as nearly as
 // possible (a panel is one gemm() call), among the widths that cut C into 4 .. 12 panels
-static int64_t host_panel_columns(int dtype, int64_t m, int64_t n, int sms) {
+static int64_t host_panel_columns(int dtype, int64_t m, int64_t n, int sms, bool wire_bound) {
     const int tile = dtype == GEMM_F32 ? 128 : 256;                 // fp32: 128 x 128 CTA tiles; 16-bit: 256 x 256 on CTA pairs
     const int64_t slots = dtype == GEMM_F32 ? 2 * (int64_t)sms : sms / 2;
     const int64_t tiles_m = ceil_div(m, tile), tiles_n = ceil_div(n, tile);
@@ -743,6 +743,9 @@ static int64_t host_panel_columns(int dtype, int64_t m, int64_t n, int sms) {
         const int64_t panels = ceil_div(tiles_n, c);
         if (panels < 4 || panels > 12) continue;
         const int64_t tiles = tiles_m * c;
+        // when the transfers set the pace the arithmetic has slack: finer panels (a shorter last step after the last
+        // byte has arrived), as long as a panel still gives every SM a tile
+        if (wire_bound && panels < 6 && tiles_m * ceil_div(tiles_n, 6) * 2 >= slots) continue;
         const double eff = (double)tiles / (double)(ceil_div(tiles, slots) * slots);
         if (eff > best_eff + 1e-9) { best_eff = eff; best = c; }
     }
@@ -789,7 +792,10 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     // is multiplied and panel p-1 is copied out.  Small problems use one panel.
     const double traffic = (double)b_bytes + (double)m * n * es_c * (beta != 0.0f ? 2.0 : 1.0);
     int64_t panel = n;
-    if (traffic > 32e6 && n >= 1024) panel = host_panel_columns(input_dtype(dtype), m, n, st->sms);
+    const double wire_rate = 50e9, flop_rate = input_dtype(dtype) == GEMM_F32 ? 5.4e13 : 1.2e15;
+    const double t_wire = ((double)a_bytes + (double)b_bytes + (beta != 0.0f ? (double)m * n * es_c : 0.0)) / wire_rate;
+    const double t_flops = 2.0 * (double)m * (double)n * (double)k / flop_rate;
+    if (traffic > 32e6 && n >= 1024) panel = host_panel_columns(input_dtype(dtype), m, n, st->sms, t_wire > 1.25 * t_flops);
     if (panel > n) panel = n;
     const int np = (int)ceil_div(n, panel);
     // While A itself is still arriving, the leading column panels are computed k panel by k panel (the order of the
@@ -808,7 +814,7 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     cudaError_t e = cudaSuccess;
     int rc = GEMM_OK;
     auto chk = [&](cudaError_t r) { if (e == cudaSuccess && r != cudaSuccess) e = r; return r == cudaSuccess; };
-    const size_t nev = (size_t)(2 * np + 3 + nk);
+    const size_t nev = (size_t)(3 * np + 2 * nk + 8);
     while (pipe->events.size() < nev && e == cudaSuccess) {
         cudaEvent_t ev_new;
         if (chk(cudaEventCreateWithFlags(&ev_new, cudaEventDisableTiming))) pipe->events.push_back(ev_new);
@@ -816,6 +822,7 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     if (e != cudaSuccess) return fail_launch(e);
     cudaEvent_t* ev = pipe->events.data();
     cudaEvent_t ev_alloc = ev[0], ev_a = ev[1], ev_done = ev[2];
+    size_t ev_next = 3;
 
     if (a_bytes) chk(cudaMallocFromPoolAsync(&dA, a_bytes, pipe->pool, s));
     if (b_bytes) chk(cudaMallocFromPoolAsync(&dB, b_bytes, pipe->pool, s));
@@ -827,91 +834,111 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
     }
     const char* hB = static_cast<const char*>(B_host);
     char* dBp = static_cast<char*>(dB);
-    auto cols_of = [&](int p) { const int64_t j0 = (int64_t)p * panel; return (n - j0 < panel) ? n - j0 : panel; };
-    auto b_off_of = [&](int p) { const int64_t j0 = (int64_t)p * panel; return needs_ab ? (tb ? (size_t)j0 * es : (size_t)j0 * ldb * es) : (size_t)0; };
-    auto c_off_of = [&](int p) { return (size_t)((int64_t)p * panel) * ldc * es_c; };
-    // panel p of op(B) and (if it is read) of C to the device; ev[3 + 2p] marks their arrival
-    auto send_panel = [&](int p) {
-        const int64_t cols = cols_of(p);
-        const size_t b_off = b_off_of(p), c_off = c_off_of(p);
-        if (needs_ab) {
-            if (tb) chk(copy_window(dBp + b_off, hB + b_off, cols, k, ldb, es, cudaMemcpyHostToDevice, pipe->in));
-            else chk(copy_window(dBp + b_off, hB + b_off, k, cols, ldb, es, cudaMemcpyHostToDevice, pipe->in));
-        }
-        // only the m x cols window of C travels: the host's padding rows are never touched
+    // columns [first column of panel pa, first column of panel pb) of C and of op(B)
+    auto col0_of = [&](int p) { const int64_t j0 = (int64_t)p * panel; return j0 < n ? j0 : n; };
+    auto cols_of = [&](int pa, int pb) { return col0_of(pb) - col0_of(pa); };
+    auto b_off_of = [&](int p) { const int64_t j0 = col0_of(p); return needs_ab ? (tb ? (size_t)j0 * es : (size_t)j0 * ldb * es) : (size_t)0; };
+    auto c_off_of = [&](int p) { return (size_t)col0_of(p) * ldc * es_c; };
+    // The multiplications wait for what the inbound stream had been given when they were enqueued: the stream is in
+    // order, so its latest event covers every earlier copy.
+    auto arrived = [&]() {
+        cudaEvent_t now = ev[ev_next++];
+        chk(cudaEventRecord(now, pipe->in));
+        chk(cudaStreamWaitEvent(s, now, 0));
+    };
+    // panels [pa, pb) of C to the device, if C is read at all (only the m rows travel: the host's padding is never touched)
+    auto send_c = [&](int pa, int pb) {
         if (beta != 0.0f)
-            chk(copy_window(static_cast<char*>(dC) + c_off, static_cast<const char*>(C_host) + c_off, m, cols, ldc, es_c,
-                            cudaMemcpyHostToDevice, pipe->in));
-        chk(cudaEventRecord(ev[3 + 2 * p], pipe->in));
+            chk(copy_window(static_cast<char*>(dC) + c_off_of(pa), static_cast<const char*>(C_host) + c_off_of(pa), m,
+                            cols_of(pa, pb), ldc, es_c, cudaMemcpyHostToDevice, pipe->in));
     };
-    // panel p back to the host once the multiplications enqueued so far are done
-    auto return_panel = [&](int p) {
-        const size_t c_off = c_off_of(p);
-        chk(cudaEventRecord(ev[4 + 2 * p], s));
-        chk(cudaStreamWaitEvent(pipe->out, ev[4 + 2 * p], 0));
-        chk(copy_window(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off, m, cols_of(p), ldc, es_c,
-                        cudaMemcpyDeviceToHost, pipe->out));
+    // rows [k0, k0 + kk) of panels [pa, pb) of op(B) to the device
+    auto send_b = [&](int pa, int pb, int64_t k0, int64_t kk) {
+        if (!needs_ab) return;
+        const size_t off = b_off_of(pa) + (tb ? (size_t)k0 * ldb * es : (size_t)k0 * es);
+        if (tb) chk(copy_window(dBp + off, hB + off, cols_of(pa, pb), kk, ldb, es, cudaMemcpyHostToDevice, pipe->in));
+        else chk(copy_window(dBp + off, hB + off, kk, cols_of(pa, pb), ldb, es, cudaMemcpyHostToDevice, pipe->in));
     };
-    // k panel q of A times the matching rows of panel p of op(B), added onto panel p of C
-    auto k_step = [&](int q, int p) {
-        const int64_t p0 = (int64_t)q * kpanel, kk = (k - p0 < kpanel) ? k - p0 : kpanel;
-        const size_t a_off = ta ? (size_t)p0 * es : (size_t)p0 * lda * es;          // columns p0.. of op(A)
-        const size_t bk_off = tb ? (size_t)p0 * ldb * es : (size_t)p0 * es;          // rows p0.. of op(B)
-        chk(cudaStreamWaitEvent(s, ev[3 + 2 * np + q], 0));
-        chk(cudaStreamWaitEvent(s, ev[3 + 2 * p], 0));
+    // columns [k0, k0 + kk) of op(A) to the device
+    auto send_a = [&](int64_t k0, int64_t kk) {
+        const size_t off = ta ? (size_t)k0 * es : (size_t)k0 * lda * es;
+        char* dAp = static_cast<char*>(dA) + off;
+        const char* hAp = static_cast<const char*>(A_host) + off;
+        if (ta) chk(copy_window(dAp, hAp, kk, m, lda, es, cudaMemcpyHostToDevice, pipe->in));
+        else chk(copy_window(dAp, hAp, m, kk, lda, es, cudaMemcpyHostToDevice, pipe->in));
+    };
+    // panels [pa, pb) back to the host once the multiplications enqueued so far are done
+    auto return_panels = [&](int pa, int pb) {
+        cudaEvent_t done = ev[ev_next++];
+        chk(cudaEventRecord(done, s));
+        chk(cudaStreamWaitEvent(pipe->out, done, 0));
+        chk(copy_window(static_cast<char*>(C_host) + c_off_of(pa), static_cast<char*>(dC) + c_off_of(pa), m, cols_of(pa, pb),
+                        ldc, es_c, cudaMemcpyDeviceToHost, pipe->out));
+    };
+    // columns [k0, k0 + kk) of op(A) times the matching rows of panels [pa, pb) of op(B), onto those panels of C (as one call:
+    // the panels are neighbours); the first range of k applies beta, the later ones add
+    auto multiply = [&](int pa, int pb, int64_t k0, int64_t kk) {
         if (e != cudaSuccess || rc != GEMM_OK) return;
-        rc = gemm(dtype, transA, transB, m, cols_of(p), kk, alpha, static_cast<char*>(dA) + a_off, lda,
-                  dBp + b_off_of(p) + bk_off, ldb, q == 0 ? beta : 1.0f, static_cast<char*>(dC) + c_off_of(p), ldc, stream);
+        const size_t a_off = ta ? (size_t)k0 * es : (size_t)k0 * lda * es;
+        const size_t bk_off = tb ? (size_t)k0 * ldb * es : (size_t)k0 * es;
+        rc = gemm(dtype, transA, transB, m, cols_of(pa, pb), kk, alpha, needs_ab ? static_cast<char*>(dA) + a_off : nullptr, lda,
+                  needs_ab ? dBp + b_off_of(pa) + bk_off : nullptr, ldb, k0 == 0 ? beta : 1.0f,
+                  static_cast<char*>(dC) + c_off_of(pa), ldc, stream);
     };
 
-    // Phase 1, while A arrives (k panel by k panel, after the first panel of B and C): the first `lead` column panels
-    // are multiplied k panel by k panel, enough of them that the arithmetic lasts about as long as A's transfer; the
-    // later ones of them join when their B and C have arrived, catching up on the k panels that are already there.
+    // Phase 1, while A arrives k panel by k panel: the first `lead` column panels are multiplied k panel by k panel.  They
+    // join one after the other, a new one behind every k panel of A (its C, and the rows of its B that match the k panels
+    // already there, then one multiplication over that whole range of k to catch up), so that early on, when every byte
+    // on the wire enables little arithmetic, the work that can run grows in both directions at once.  From then on each k
+    // panel of A travels with the matching rows of B for all panels that have joined and is multiplied into them in one call.
     int lead = 0;
     if (needs_ab) {
         lead = 1;
         if (nk > 1) {
-            const double t_a = (double)a_bytes / 50e9;
-            const double rate = input_dtype(dtype) == GEMM_F32 ? 5.0e13 : 1.2e15;
-            const double t_panel = 2.0 * (double)m * (double)panel * (double)k / rate;
-            lead = (int)(t_a / t_panel + 0.999);
+            // every lead panel also puts its own B and C on the wire, so the arithmetic of L panels has to cover A's
+            // transfer plus L panels' worth of B and C; a transfer-bound problem takes a few panels for the early overlap
+            const double t_a = (double)a_bytes / wire_rate;
+            const double t_panel = 2.0 * (double)m * (double)panel * (double)k / flop_rate;
+            const double t_bc = ((double)panel * (double)k * es + (beta != 0.0f ? (double)m * (double)panel * es_c : 0.0)) / wire_rate;
+            lead = t_panel > 1.25 * t_bc ? (int)(t_a / (t_panel - t_bc) + 0.999) : 4;
             if (lead > np - 1) lead = np - 1;
             if (lead > nk) lead = nk;
             if (lead < 1) lead = 1;
         }
-        send_panel(0);
+        send_c(0, 1);
+        if (nk == 1) send_b(0, 1, 0, k);
         int joined = 1;
         for (int q = 0; q < nk && e == cudaSuccess && rc == GEMM_OK; ++q) {
-            const int64_t p0 = (int64_t)q * kpanel, kk = (k - p0 < kpanel) ? k - p0 : kpanel;
-            const size_t a_off = ta ? (size_t)p0 * es : (size_t)p0 * lda * es;
-            char* dAp = static_cast<char*>(dA) + a_off;
-            const char* hAp = static_cast<const char*>(A_host) + a_off;
-            if (ta) chk(copy_window(dAp, hAp, kk, m, lda, es, cudaMemcpyHostToDevice, pipe->in));
-            else chk(copy_window(dAp, hAp, m, kk, lda, es, cudaMemcpyHostToDevice, pipe->in));
-            chk(cudaEventRecord(ev[3 + 2 * np + q], pipe->in));
-            for (int p = 0; p < joined; ++p) k_step(q, p);
-            // the next lead panel follows this k panel on the wire when its turn has come (evenly spread over A's transfer)
-            if (joined < lead && (q + 1) * lead >= joined * nk) {
-                send_panel(joined);
-                for (int qq = 0; qq <= q; ++qq) k_step(qq, joined);
+            const int64_t k0 = (int64_t)q * kpanel, kk = (k - k0 < kpanel) ? k - k0 : kpanel;
+            const bool last = q == nk - 1;
+            send_a(k0, kk);
+            if (nk > 1) send_b(0, joined, k0, kk);
+            arrived();
+            if (!last) multiply(0, joined, k0, kk);
+            else
+                for (int p = 0; p < joined; ++p) {      // panel by panel, so that each starts home as soon as it is complete
+                    multiply(p, p + 1, k0, kk);
+                    return_panels(p, p + 1);
+                }
+            if (joined < lead) {
+                send_c(joined, joined + 1);
+                send_b(joined, joined + 1, 0, k0 + kk);
+                arrived();
+                multiply(joined, joined + 1, 0, k0 + kk);
+                if (last) return_panels(joined, joined + 1);
                 ++joined;
             }
         }
-        for (int p = joined; p < lead && e == cudaSuccess && rc == GEMM_OK; ++p) {      // (only if nk < lead, which the clamp rules out)
-            send_panel(p);
-            for (int q = 0; q < nk; ++q) k_step(q, p);
-        }
-        for (int p = 0; p < lead && e == cudaSuccess && rc == GEMM_OK; ++p) return_panel(p);
+        lead = joined;
     }
     // Phase 2: A is resident; the remaining panels flow through copy in / multiply / copy out
     for (int p = lead; p < np && e == cudaSuccess && rc == GEMM_OK; ++p) {
-        send_panel(p);
-        chk(cudaStreamWaitEvent(s, ev[3 + 2 * p], 0));
-        if (e != cudaSuccess) break;
-        rc = gemm(dtype, transA, transB, m, cols_of(p), k, alpha, dA, lda, needs_ab ? dBp + b_off_of(p) : nullptr, ldb, beta,
-                  static_cast<char*>(dC) + c_off_of(p), ldc, stream);
+        send_c(p, p + 1);
+        send_b(p, p + 1, 0, k);
+        arrived();
+        multiply(p, p + 1, 0, k);
         if (rc != GEMM_OK) break;
-        return_panel(p);
+        return_panels(p, p + 1);
     }
     cudaEventRecord(ev_done, pipe->out);                     // the caller's stream rejoins both copy streams
     cudaStreamWaitEvent(s, ev_done, 0);

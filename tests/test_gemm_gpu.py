@@ -241,7 +241,8 @@ def test_gemm_host_pipelined_panels_match_oracle(dtype):
              (260, 8200, 1100, "T", "T", 1.0, 0.0, (8, 8, 2)),     # multi-panel, strided panels of B, C write-only
              (100, 90, 70, "N", "T", -1.0, 1.0, (1, 3, 1)),        # single panel
              (4500, 3000, 2100, "N", "N", 1.0, 0.5, (4, 0, 4)),    # A large enough to arrive in row panels
-             (4400, 2900, 2050, "T", "N", 1.0, 0.0, (8, 8, 0))]    # same with A stored transposed
+             (4400, 2900, 2050, "T", "N", 1.0, 0.0, (8, 8, 0)),    # same with A stored transposed
+             (4300, 2800, 2200, "N", "T", 1.5, 0.5, (0, 8, 4))]    # k slices of a transposed B beside A's
     for (m, n, k, ta, tb, alpha, beta, pad) in cases:
         p = problem(dtype, m, n, k, ta, tb, alpha, beta, kind, pad, seed=m)
         A, B, C0 = p.operands()
