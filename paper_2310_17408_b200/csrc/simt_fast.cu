@@ -209,19 +209,20 @@ __device__ __forceinline__ void fma2(uint64_t& c, uint64_t a, uint64_t b) {
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(c) : "l"(a), "l"(b));
 }
 
-// The thread's 8 x 8 register block as 2 x 2 sub-blocks of packed pairs.  For rows (i, i+1) and columns (j, j+1):
-//   P[j/2][i/2] = ( acc(i, j),   acc(i+1, j+1) )   updated with (a_i, a_i+1) * (b_j,   b_j+1)
-//   Q[j/2][i/2] = ( acc(i, j+1), acc(i+1, j)   )   updated with (a_i, a_i+1) * (b_j+1, b_j)
-// so that the pairs of A come straight out of the 128-bit fragment load and B needs only its four swapped pairs.
+// The thread's 8 x 8 register block as packed pairs of neighbouring rows: P[j][i] = ( acc(2i, j), acc(2i+1, j) ),
+// updated with (a_2i, a_2i+1) * (b_j, b_j).  The pairs of A come straight out of the 128-bit fragment loads; every b_j
+// is duplicated into a pair once per k.  Measured on operands fed from shared memory alone (no global traffic), this
+// form runs at 66 TFLOP/s, the scalar 8 x 8 block at 60-63 and pairs along the diagonals (A pairs and swapped B pairs,
+// no duplicates) at 61.
 struct Acc2 {
-    uint64_t P[4][4], Q[4][4];
+    uint64_t P[8][4];
 };
 
 // one BK slice of outer products on the thread's 8 x 8 register block
 template <int BM, int BN>
 __device__ __forceinline__ void compute_stage(Acc2& acc, const float* __restrict__ As,
                                               const float* __restrict__ Bs, int am, int bn) {
-    uint64_t a[2][4], b[2][4], bs[2][4];
+    uint64_t a[2][4], b[2][8];
     auto frag = [&](int kk, int buf) {
         const float* ap = As + kk * (BM + PAD) + am;
         const float* bp = Bs + kk * (BN + PAD) + bn;
@@ -231,42 +232,29 @@ __device__ __forceinline__ void compute_stage(Acc2& acc, const float* __restrict
         float4 b1 = *reinterpret_cast<const float4*>(bp + 16);
         a[buf][0] = pack2(a0.x, a0.y); a[buf][1] = pack2(a0.z, a0.w);
         a[buf][2] = pack2(a1.x, a1.y); a[buf][3] = pack2(a1.z, a1.w);
-        b[buf][0] = pack2(b0.x, b0.y); b[buf][1] = pack2(b0.z, b0.w);
-        b[buf][2] = pack2(b1.x, b1.y); b[buf][3] = pack2(b1.z, b1.w);
-        bs[buf][0] = pack2(b0.y, b0.x); bs[buf][1] = pack2(b0.w, b0.z);
-        bs[buf][2] = pack2(b1.y, b1.x); bs[buf][3] = pack2(b1.w, b1.z);
+        b[buf][0] = pack2(b0.x, b0.x); b[buf][1] = pack2(b0.y, b0.y);
+        b[buf][2] = pack2(b0.z, b0.z); b[buf][3] = pack2(b0.w, b0.w);
+        b[buf][4] = pack2(b1.x, b1.x); b[buf][5] = pack2(b1.y, b1.y);
+        b[buf][6] = pack2(b1.z, b1.z); b[buf][7] = pack2(b1.w, b1.w);
     };
     frag(0, 0);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
         if (kk + 1 < BK) frag(kk + 1, (kk + 1) & 1);
-        // boustrophedon order over the 4 x 4 pairs: consecutive instructions share the A pair, and across a turn
-        // also the B pair (measured 1 % faster than row-by-row order)
+        // row pair by row pair: eight consecutive instructions share the A pair
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-                const int j = (i & 1) ? 3 - jj : jj;
-                if (i & 1) {
-                    fma2(acc.Q[j][i], a[kk & 1][i], bs[kk & 1][j]);
-                    fma2(acc.P[j][i], a[kk & 1][i], b[kk & 1][j]);
-                } else {
-                    fma2(acc.P[j][i], a[kk & 1][i], b[kk & 1][j]);
-                    fma2(acc.Q[j][i], a[kk & 1][i], bs[kk & 1][j]);
-                }
-            }
+            for (int j = 0; j < 8; ++j) fma2(acc.P[j][i], a[kk & 1][i], b[kk & 1][j]);
     }
 }
 
 // packed accumulators -> acc[column][row] of the 8 x 8 block
 __device__ __forceinline__ void unpack_block(const Acc2& p, float (&acc)[8][8]) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+    for (int j = 0; j < 8; ++j)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            unpack2(p.P[j][i], acc[2 * j][2 * i], acc[2 * j + 1][2 * i + 1]);
-            unpack2(p.Q[j][i], acc[2 * j + 1][2 * i], acc[2 * j][2 * i + 1]);
-        }
+        for (int i = 0; i < 4; ++i) unpack2(p.P[j][i], acc[j][2 * i], acc[j][2 * i + 1]);
 }
 
 // Whether the kernel with this CTA tile can finish a split of k itself, as a thread-block cluster: every CTA then
@@ -342,9 +330,9 @@ simt_fast_body(int64_t m, int64_t n, int64_t k, float alpha, const float* __rest
 
     Acc2 acc2;
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
+    for (int j = 0; j < 8; ++j)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc2.P[j][i] = acc2.Q[j][i] = 0ull;      // (+0.0f, +0.0f)
+        for (int i = 0; i < 4; ++i) acc2.P[j][i] = 0ull;      // (+0.0f, +0.0f)
 
     float ra[LA::ELEMS], rb[LB::ELEMS];
     const bool interior = (i0 + BM <= m) && (j0 + BN <= n);
