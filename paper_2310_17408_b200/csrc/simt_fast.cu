@@ -209,11 +209,13 @@ __device__ __forceinline__ void fma2(uint64_t& c, uint64_t a, uint64_t b) {
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(c) : "l"(a), "l"(b));
 }
 
-// The thread's 8 x 8 register block as packed pairs of neighbouring rows: P[j][i] = ( acc(2i, j), acc(2i+1, j) ),
-// updated with (a_2i, a_2i+1) * (b_j, b_j).  The pairs of A come straight out of the 128-bit fragment loads; every b_j
-// is duplicated into a pair once per k.  Measured on operands fed from shared memory alone (no global traffic), this
-// form runs at 66 TFLOP/s, the scalar 8 x 8 block at 60-63 and pairs along the diagonals (A pairs and swapped B pairs,
-// no duplicates) at 61.
+// The thread's 8 x 8 register block as packed pairs of neighbouring columns: P[i][j] = ( acc(i, 2j), acc(i, 2j+1) ),
+// updated with (a_i, a_i) * (b_2j, b_2j+1).  The pairs of B come straight out of the 128-bit fragment loads; every a_i
+// is duplicated into a pair once per k; column pair by column pair, so that eight consecutive instructions share the
+// B pair.  Forms measured in this kernel at 8192^3: this one 59.7 TFLOP/s; pairs of neighbouring rows with b
+// duplicated 58.1 (either order of the loops); pairs along the diagonals (A pairs and swapped B pairs, no duplicates)
+// 55.3; the scalar block 51 (at 4096^3).  On operands fed from shared memory alone, without the global loads, stores and barriers
+// around it, the same forms reach 66, 63-66, 61 and 60-63.
 struct Acc2 {
     uint64_t P[8][4];
 };
@@ -222,7 +224,7 @@ struct Acc2 {
 template <int BM, int BN>
 __device__ __forceinline__ void compute_stage(Acc2& acc, const float* __restrict__ As,
                                               const float* __restrict__ Bs, int am, int bn) {
-    uint64_t a[2][4], b[2][8];
+    uint64_t a[2][8], b[2][4];
     auto frag = [&](int kk, int buf) {
         const float* ap = As + kk * (BM + PAD) + am;
         const float* bp = Bs + kk * (BN + PAD) + bn;
@@ -230,31 +232,30 @@ __device__ __forceinline__ void compute_stage(Acc2& acc, const float* __restrict
         float4 a1 = *reinterpret_cast<const float4*>(ap + 32);
         float4 b0 = *reinterpret_cast<const float4*>(bp);
         float4 b1 = *reinterpret_cast<const float4*>(bp + 16);
-        a[buf][0] = pack2(a0.x, a0.y); a[buf][1] = pack2(a0.z, a0.w);
-        a[buf][2] = pack2(a1.x, a1.y); a[buf][3] = pack2(a1.z, a1.w);
-        b[buf][0] = pack2(b0.x, b0.x); b[buf][1] = pack2(b0.y, b0.y);
-        b[buf][2] = pack2(b0.z, b0.z); b[buf][3] = pack2(b0.w, b0.w);
-        b[buf][4] = pack2(b1.x, b1.x); b[buf][5] = pack2(b1.y, b1.y);
-        b[buf][6] = pack2(b1.z, b1.z); b[buf][7] = pack2(b1.w, b1.w);
+        b[buf][0] = pack2(b0.x, b0.y); b[buf][1] = pack2(b0.z, b0.w);
+        b[buf][2] = pack2(b1.x, b1.y); b[buf][3] = pack2(b1.z, b1.w);
+        a[buf][0] = pack2(a0.x, a0.x); a[buf][1] = pack2(a0.y, a0.y);
+        a[buf][2] = pack2(a0.z, a0.z); a[buf][3] = pack2(a0.w, a0.w);
+        a[buf][4] = pack2(a1.x, a1.x); a[buf][5] = pack2(a1.y, a1.y);
+        a[buf][6] = pack2(a1.z, a1.z); a[buf][7] = pack2(a1.w, a1.w);
     };
     frag(0, 0);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
         if (kk + 1 < BK) frag(kk + 1, (kk + 1) & 1);
-        // row pair by row pair: eight consecutive instructions share the A pair
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int j = 0; j < 8; ++j) fma2(acc.P[j][i], a[kk & 1][i], b[kk & 1][j]);
+            for (int i = 0; i < 8; ++i) fma2(acc.P[i][j], a[kk & 1][i], b[kk & 1][j]);
     }
 }
 
 // packed accumulators -> acc[column][row] of the 8 x 8 block
 __device__ __forceinline__ void unpack_block(const Acc2& p, float (&acc)[8][8]) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
+    for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) unpack2(p.P[j][i], acc[j][2 * i], acc[j][2 * i + 1]);
+        for (int j = 0; j < 4; ++j) unpack2(p.P[i][j], acc[2 * j][i], acc[2 * j + 1][i]);
 }
 
 // Whether the kernel with this CTA tile can finish a split of k itself, as a thread-block cluster: every CTA then
