@@ -288,11 +288,12 @@ int gemm_last_cuda_error(void);   /* cudaError_t of the last failed launch, 0 if
  *
  *   gemm_probe_copy   streams `bytes` (a multiple of 16, at most 64 GiB) from src to dst (device pointers, 16-byte
  *                     aligned, not overlapping; dst is overwritten).  *gbs = (bytes read + bytes written) / time, GB/s.
- *   gemm_probe_ffma   register-only fp32 fused multiply-adds on all SMs, no memory traffic.  pattern 0: 16 independent
- *                     chains per thread, 2048 threads per SM (the issue-rate ceiling); pattern 1: an 8 x 8 block of
- *                     accumulators updated by outer products, 2 x 256 threads per SM (what a thread of the SIMT
- *                     GEMM kernel does between shared-memory reads); pattern 2: the same block on packed
- *                     fma.rn.f32x2.  iters in 1..65536 loop trips of 8 steps each.  *tflops = 2 * FMAs / time.
+ *   gemm_probe_ffma   fp32 fused multiply-adds on all SMs, no global memory traffic.  pattern 0: 16 independent
+ *                     register-only chains per thread, 2048 threads per SM (the issue-rate ceiling); pattern 1: the
+ *                     micro-kernel of the SIMT GEMM kernel on its own, an 8 x 8 block of accumulators per thread updated
+ *                     by outer products whose operands are read from shared memory with the kernel's 128-bit fragment
+ *                     loads, 2 x 256 threads per SM, scalar FMAs; pattern 2: the same on packed fma.rn.f32x2 in the
+ *                     kernel's arrangement.  iters in 1..65536 loop trips of 8 steps each.  *tflops = 2 * FMAs / time.
  *   gemm_probe_umma   tcgen05.mma (kind::f16, fp32 accumulators in TMEM) on operand tiles that stay in shared memory:
  *                     one CTA per SM issuing 128 x 256 x 16 MMAs (pair = 0), or one CTA pair per two SMs issuing
  *                     256 x 256 x 16 MMAs with cta_group::2 (pair = 1); dtype GEMM_F16 or GEMM_BF16; kblocks in

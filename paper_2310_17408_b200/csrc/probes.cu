@@ -2,8 +2,8 @@
 // code on the device it runs on.  They are the counterpart of the paper's "solo mode" (Section IV-A: the micro-kernel
 // called on its own, operands resident in the fastest memory), one per unit that bounds a kernel here:
 //   gemm_probe_copy   HBM: a streaming copy (bytes read + bytes written per second)
-//   gemm_probe_ffma   CUDA cores: register-only fp32 FMA loops, as independent chains and in the 8 x 8 outer-product
-//                     register pattern of the SIMT kernel's micro-tile (scalar and packed fma.rn.f32x2 forms)
+//   gemm_probe_ffma   CUDA cores: fp32 FMA loops, as independent register-only chains and as the SIMT kernel's 8 x 8
+//                     micro-kernel fed from shared memory (scalar and packed fma.rn.f32x2 forms)
 //   gemm_probe_umma   tensor cores: tcgen05.mma on operands that stay in shared memory, accumulators in TMEM
 // Every probe has a bounded run time (iteration counts are capped), touches no caller memory except the two
 // buffers handed to the copy probe, and times itself with CUDA events on the caller's stream.
@@ -54,19 +54,27 @@ probe_ffma_chains_kernel(int iters, float x, float y) {
     if (s == 1.2345678e-30f) g_probe_sink[threadIdx.x & 31] = s;
 }
 
-// the register pattern of a GEMM thread: an 8 x 8 block of accumulators receives one outer product a (8) x b (8) per
-// step; a and b change every step (here: rotated among registers that the loop keeps alive), as they do when they
-// come from shared memory.  PACKED: two FMAs per fma.rn.f32x2, accumulators held as the diagonal / anti-diagonal
-// pairs of 2 x 2 sub-blocks, the arrangement of the SIMT kernel.
+// The micro-kernel of a GEMM thread on its own: an 8 x 8 block of accumulators receives one outer product a (8) x b (8)
+// per k, a and b read from shared memory with two 128-bit loads each, as the SIMT kernel's threads read their
+// fragments (one slice of 8 k per loop trip, the next k's fragments loaded while the current ones are used); no global
+// traffic, no stores, no barriers inside the loop.  PACKED: two FMAs per fma.rn.f32x2, accumulators held as pairs of
+// neighbouring columns and every a duplicated into a pair, the arrangement of the SIMT kernel; otherwise scalar FMAs,
+// row by row with the columns there and back.
+constexpr int PROBE_BK = 8, PROBE_LD = 132;       // rows of 128 floats + 4 of padding, as the kernel's stages
 template <bool PACKED>
 __global__ void __launch_bounds__(256, 2)
 probe_ffma_block_kernel(int iters, float x) {
-    float a[2][8], b[2][8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        a[0][i] = x * (float)(threadIdx.x + i); a[1][i] = x * (float)(threadIdx.x + 2 * i + 1);
-        b[0][i] = x * (float)(blockIdx.x + i);  b[1][i] = x * (float)(blockIdx.x + 3 * i + 2);
+    __shared__ __align__(16) float As[PROBE_BK * PROBE_LD];
+    __shared__ __align__(16) float Bs[PROBE_BK * PROBE_LD];
+    for (int i = threadIdx.x; i < PROBE_BK * PROBE_LD; i += 256) {
+        As[i] = x * (float)(i % 7);
+        Bs[i] = x * (float)(i % 5);
     }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // fragment offsets: 0..28 (+32) of a row of A, 0..76 (+16) of a row of B: inside the 128 floats of a row
+    const float* ap = As + (lane & 7) * 4;
+    const float* bp = Bs + (lane >> 3) * 4 + (warp & 1) * 64;
     float s = 0.0f;
     if (!PACKED) {
         float acc[8][8];
@@ -75,52 +83,74 @@ probe_ffma_block_kernel(int iters, float x) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) acc[j][i] = 0.0f;
         for (int it = 0; it < iters; ++it) {
+            float a[2][8], b[2][8];
+            auto frag = [&](int kk, int buf) {
+                const float4 a0 = *reinterpret_cast<const float4*>(ap + kk * PROBE_LD);
+                const float4 a1 = *reinterpret_cast<const float4*>(ap + kk * PROBE_LD + 32);
+                const float4 b0 = *reinterpret_cast<const float4*>(bp + kk * PROBE_LD);
+                const float4 b1 = *reinterpret_cast<const float4*>(bp + kk * PROBE_LD + 16);
+                a[buf][0] = a0.x; a[buf][1] = a0.y; a[buf][2] = a0.z; a[buf][3] = a0.w;
+                a[buf][4] = a1.x; a[buf][5] = a1.y; a[buf][6] = a1.z; a[buf][7] = a1.w;
+                b[buf][0] = b0.x; b[buf][1] = b0.y; b[buf][2] = b0.z; b[buf][3] = b0.w;
+                b[buf][4] = b1.x; b[buf][5] = b1.y; b[buf][6] = b1.z; b[buf][7] = b1.w;
+            };
+            frag(0, 0);
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
+            for (int kk = 0; kk < PROBE_BK; ++kk) {
+                if (kk + 1 < PROBE_BK) frag(kk + 1, (kk + 1) & 1);
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
+                for (int i = 0; i < 8; ++i)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) acc[j][i] = fmaf(a[u & 1][(i + u) & 7], b[u & 1][(j + u) & 7], acc[j][i]);
+                    for (int jj = 0; jj < 8; ++jj) {
+                        const int j = (i & 1) ? 7 - jj : jj;
+                        acc[j][i] = fmaf(a[kk & 1][i], b[kk & 1][j], acc[j][i]);
+                    }
+            }
+            asm volatile("" ::: "memory");      // the next trip reads its fragments again
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j)
 #pragma unroll
             for (int i = 0; i < 8; ++i) s += acc[j][i];
     } else {
-        uint64_t P[4][4], Q[4][4];
+        uint64_t P[8][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int i = 0; i < 8; ++i)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) P[j][i] = Q[j][i] = 0ull;
+            for (int j = 0; j < 4; ++j) P[i][j] = 0ull;
         auto pack = [](float lo, float hi) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; };
-        uint64_t ap[2][4], bp[2][4], bs[2][4];
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                ap[h][i] = pack(a[h][2 * i], a[h][2 * i + 1]);
-                bp[h][i] = pack(b[h][2 * i], b[h][2 * i + 1]);
-                bs[h][i] = pack(b[h][2 * i + 1], b[h][2 * i]);
-            }
         for (int it = 0; it < iters; ++it) {
+            uint64_t a[2][8], b[2][4];
+            auto frag = [&](int kk, int buf) {
+                const float4 a0 = *reinterpret_cast<const float4*>(ap + kk * PROBE_LD);
+                const float4 a1 = *reinterpret_cast<const float4*>(ap + kk * PROBE_LD + 32);
+                const float4 b0 = *reinterpret_cast<const float4*>(bp + kk * PROBE_LD);
+                const float4 b1 = *reinterpret_cast<const float4*>(bp + kk * PROBE_LD + 16);
+                b[buf][0] = pack(b0.x, b0.y); b[buf][1] = pack(b0.z, b0.w);
+                b[buf][2] = pack(b1.x, b1.y); b[buf][3] = pack(b1.z, b1.w);
+                a[buf][0] = pack(a0.x, a0.x); a[buf][1] = pack(a0.y, a0.y);
+                a[buf][2] = pack(a0.z, a0.z); a[buf][3] = pack(a0.w, a0.w);
+                a[buf][4] = pack(a1.x, a1.x); a[buf][5] = pack(a1.y, a1.y);
+                a[buf][6] = pack(a1.z, a1.z); a[buf][7] = pack(a1.w, a1.w);
+            };
+            frag(0, 0);
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
+            for (int kk = 0; kk < PROBE_BK; ++kk) {
+                if (kk + 1 < PROBE_BK) frag(kk + 1, (kk + 1) & 1);
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+                for (int j = 0; j < 4; ++j)
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(P[j][i]) : "l"(ap[u & 1][(i + u) & 3]), "l"(bp[u & 1][(j + u) & 3]));
-                        asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(Q[j][i]) : "l"(ap[u & 1][(i + u) & 3]), "l"(bs[u & 1][(j + u) & 3]));
-                    }
+                    for (int i = 0; i < 8; ++i)
+                        asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(P[i][j]) : "l"(a[kk & 1][i]), "l"(b[kk & 1][j]));
+            }
+            asm volatile("" ::: "memory");
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
+        for (int i = 0; i < 8; ++i)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int j = 0; j < 4; ++j) {
                 float lo, hi;
-                asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(P[j][i]));
-                s += lo + hi;
-                asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(Q[j][i]));
+                asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(P[i][j]));
                 s += lo + hi;
             }
     }
