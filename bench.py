@@ -822,7 +822,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="cfg2_fp32_squares", choices=sorted(WORKLOADS) + sorted(CONV_WORKLOADS) + sorted(BATCHED_WORKLOADS))
     ap.add_argument("--shape", default=None, help="M,N,K: time this single problem instead of a workload (alpha=1, beta=0)")
-    ap.add_argument("--dtype", default="f32", choices=["f32", "f16", "bf16"], help="operand type for --shape")
+    ap.add_argument("--dtype", default="f32", choices=["f32", "f32tc", "f16", "bf16"],
+                    help="operand type for --shape (f32tc: fp32 data through GEMM_F32_TC)")
     ap.add_argument("--kind", default=None, choices=["uniform", "normal", "int"],
                     help="value distribution for --shape (default: uniform for f32, normal for 16-bit inputs; int = integers in [-4, 4])")
     ap.add_argument("--alpha", type=float, default=1.0, help="alpha for --shape")
@@ -854,9 +855,10 @@ def main():
     if args.shape:
         from workloads import Problem
         m, n, k = (int(t) for t in args.shape.split(","))
-        dt = {"f32": DTYPE_F32, "f16": DTYPE_F16, "bf16": DTYPE_BF16}[args.dtype]
+        dt = {"f32": DTYPE_F32, "f32tc": DTYPE_F32, "f16": DTYPE_F16, "bf16": DTYPE_BF16}[args.dtype]
         kind = args.kind or ("uniform" if dt == DTYPE_F32 else "normal")
-        problems = [Problem(f"{args.dtype}_{m}x{n}x{k}", dt, m, n, k, args.alpha, args.beta, kindA=kind, kindB=kind, seed=0)]
+        problems = [Problem(f"{args.dtype}_{m}x{n}x{k}", dt, m, n, k, args.alpha, args.beta, kindA=kind, kindB=kind, seed=0,
+                            tc3=args.dtype == "f32tc")]
         args.workload = f"single:{args.dtype}:{m}x{n}x{k}"
     if args.impl == "reference":
         return run_reference(args, problems, args.workload)

@@ -36,8 +36,9 @@ typedef enum {
      * (x = x1 + x2 + x3 to within the last bit or two of x), and the six piece products that matter,
      * A1 B1 + A1 B2 + A2 B1 + A2 B2 + A1 B3 + A3 B1, are accumulated in fp32, smallest first.  Not the exact IEEE
      * fp32 arithmetic of GEMM_F32 (the dropped products are of relative size 2^-24; results stay within the same
-     * error bound 4 k 2^-24 max|A| max|B| and are exact on small integers), but 2 to 3.5 times faster from about
-     * 2048^3 on.  Needs a registered workspace of gemm_workspace_bytes(); without one, and for problems too small to
+     * error bound 4 k 2^-24 max|A| max|B| and are exact on small integers), but 1.4 to 3.4 times faster from about
+     * 1280^3 on (where C has at least 16 tiles of 256 x 256 the six products run as one multiplication whose k loop
+     * walks the pieces).  Needs a registered workspace of gemm_workspace_bytes(); without one, and for problems too small to
      * gain, the call runs as GEMM_F32.  Operands must be finite.  (The paper's data-type section, III-D, only
      * narrows the type; this mode goes the other way and keeps fp32 data on the narrow-type unit.) */
     GEMM_F32_TC   = 5,

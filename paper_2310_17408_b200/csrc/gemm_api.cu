@@ -389,7 +389,10 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip = 0);
 // Workspace for the bfloat16 pieces of A and B: three copies each, leading dimension rounded up to 8 elements.
 struct Split3Layout {
     int64_t a_rows, a_cols, b_rows, b_cols, lda_p, ldb_p;
-    size_t a_piece, b_piece, total;      // bytes
+    size_t a_piece, b_piece, total;      // bytes: three separate pieces per operand (six products, six launches)
+    // the pieces of an operand one after the other along k, k padded with zeros to a multiple of 64 (one launch)
+    int64_t seg_k, lda_f, ldb_f;
+    size_t a_fused, b_fused, a_step, b_step, total_fused;      // bytes; *_step = distance between two pieces
 };
 static Split3Layout split3_layout(const GemmArgs& a) {
     Split3Layout L;
@@ -400,17 +403,72 @@ static Split3Layout split3_layout(const GemmArgs& a) {
     L.a_piece = (size_t)round_up(L.lda_p * L.a_cols * 2, 256);
     L.b_piece = (size_t)round_up(L.ldb_p * L.b_cols * 2, 256);
     L.total = 3 * (L.a_piece + L.b_piece);
+    L.seg_k = round_up(a.k, 64);
+    // k is the row index of a stored operand (A^T, B): pieces stacked in the rows, one leading dimension of 3 * seg_k;
+    // k is the column index (A, B^T): pieces are runs of seg_k columns
+    L.lda_f = a.ta ? 3 * L.seg_k : L.lda_p;
+    L.ldb_f = a.tb ? L.ldb_p : 3 * L.seg_k;
+    L.a_step = a.ta ? (size_t)L.seg_k * 2 : (size_t)L.lda_p * L.seg_k * 2;
+    L.b_step = a.tb ? (size_t)L.ldb_p * L.seg_k * 2 : (size_t)L.seg_k * 2;
+    L.a_fused = (size_t)round_up(a.ta ? 3 * L.seg_k * a.m * 2 : L.lda_p * 3 * L.seg_k * 2, 256);
+    L.b_fused = (size_t)round_up(a.tb ? L.ldb_p * 3 * L.seg_k * 2 : 3 * L.seg_k * a.n * 2, 256);
+    L.total_fused = L.a_fused + L.b_fused;
     return L;
 }
-// worth it from about here on (measured: 1024^3 83 us against 57 us for the exact kernel, 2048^3 153 against 326 us,
-// 8192^3 5.7 against 19.9 ms; below, the two splitting passes and six launches cost more than they save)
+// worth it from about here on.  As one launch on CTA pairs (at least 16 tiles of 256 x 256), measured against the exact
+// kernel: 1024^3 51 against 53 us, 1280^3 64 against 91, 1536^3 74 against 140, 2048^3 99 against 309 us, 8192^3 5.5
+// against 18.4 ms.  As six launches (fewer tiles): 1024^3 83 against 57 us, 2048^3 153 against 326.
+static bool split3_one_launch_shape(const GemmArgs& a) {
+    return a.m > 128 && ceil_div(a.m, 256) * ceil_div(a.n, 256) >= 16;
+}
 static bool split3_worthwhile(const GemmArgs& a) {
-    return (double)a.m * (double)a.n * (double)a.k >= 1536.0 * 1536.0 * 1536.0 && a.m >= 128 && a.n >= 128 && a.k >= 64;
+    const double volume = (double)a.m * (double)a.n * (double)a.k;
+    const double from = split3_one_launch_shape(a) ? 1280.0 : 1536.0;
+    return volume >= from * from * from && a.m >= 128 && a.n >= 128 && a.k >= 64;
+}
+
+// The six piece products as ONE multiplication on CTA pairs: op(A) and op(B) hold their pieces one after the other along
+// k and every tile's k loop walks the six (piece of A, piece of B) segments, smallest products first, into one fp32
+// accumulator in TMEM; alpha and beta are applied once, in the epilogue.  For problems whose 256 x 256 tiles give
+// every CTA pair work.
+static bool split3_fused_fits(const GemmArgs& a, const Split3Layout& L, int sms, size_t ws_bytes) {
+    if (ws_bytes < L.total_fused || g_force_tile_m == 128 || g_force_tile_n == 128 || g_force_tile_n == 64) return false;
+    if (3 * L.seg_k > 0x7FFFFFFFLL) return false;
+    return split3_one_launch_shape(a);      // one k loop is six ordinary ones long: a tile per pair is not needed
+}
+static int run_f32_split3_fused(const GemmArgs& a, const Split3Layout& L, void* ws) {
+    uint8_t* pa = static_cast<uint8_t*>(ws);
+    uint8_t* pb = pa + L.a_fused;
+    // k runs along the rows of a stored A^T / B and along the columns of a stored A / B^T
+    cudaError_t e = a.ta ? launch_split3(static_cast<const float*>(a.A), L.a_rows, L.a_cols, a.lda, pa, pa + L.a_step, pa + 2 * L.a_step,
+                                         L.lda_f, a.stream, L.seg_k, 0)
+                         : launch_split3(static_cast<const float*>(a.A), L.a_rows, L.a_cols, a.lda, pa, pa + L.a_step, pa + 2 * L.a_step,
+                                         L.lda_f, a.stream, 0, L.seg_k);
+    if (e == cudaSuccess)
+        e = a.tb ? launch_split3(static_cast<const float*>(a.B), L.b_rows, L.b_cols, a.ldb, pb, pb + L.b_step, pb + 2 * L.b_step,
+                                 L.ldb_f, a.stream, 0, L.seg_k)
+                 : launch_split3(static_cast<const float*>(a.B), L.b_rows, L.b_cols, a.ldb, pb, pb + L.b_step, pb + 2 * L.b_step,
+                                 L.ldb_f, a.stream, L.seg_k, 0);
+    if (e != cudaSuccess) return fail_launch(e);
+    GemmArgs g = a;
+    g.dtype = GEMM_BF16;
+    g.split3 = 0;
+    g.A = pa; g.lda = L.lda_f;
+    g.B = pb; g.ldb = L.ldb_f;
+    g.k = 3 * L.seg_k;          // the extent of the stored operands along k
+    g.seg_k = L.seg_k;
+    gemm_config_t cfg{};
+    e = launch_tensor_pair(g, KSplit{1, g.k}, nullptr, &cfg);
+    if (e != cudaSuccess) return fail_launch(e);
+    cfg.launches = 3;
+    note_config(cfg);
+    return GEMM_OK;
 }
 
 // C <- alpha * sum of the six piece products + beta*C: six bfloat16 GEMMs accumulating into C, smallest terms first
 static int run_f32_split3(const GemmArgs& a, DeviceState* st, void* ws, size_t ws_bytes) {
     const Split3Layout L = split3_layout(a);
+    if (split3_fused_fits(a, L, st->sms, ws_bytes)) return run_f32_split3_fused(a, L, ws);
     uint8_t* base = static_cast<uint8_t*>(ws);
     void* ap[3] = {base, base + L.a_piece, base + 2 * L.a_piece};
     void* bp[3] = {base + 3 * L.a_piece, base + 3 * L.a_piece + L.b_piece, base + 3 * L.a_piece + 2 * L.b_piece};
@@ -461,7 +519,9 @@ static int run_gemm(const GemmArgs& a0, DeviceState* st, size_t ws_skip) {
         void* ws3;
         size_t ws3_bytes;
         workspace_for(st, a.stream, &ws3, &ws3_bytes);
-        if (ws3 != nullptr && ws3_bytes >= split3_layout(a).total) return run_f32_split3(a, st, ws3, ws3_bytes);
+        const Split3Layout L3 = split3_layout(a);
+        if (ws3 != nullptr && (ws3_bytes >= L3.total || split3_fused_fits(a, L3, st->sms, ws3_bytes)))
+            return run_f32_split3(a, st, ws3, ws3_bytes);
     }
     a.split3 = 0;      // from here on: the exact fp32 path
 
@@ -969,7 +1029,8 @@ size_t gemm_workspace_bytes(int dtype, char transA, char transB, int64_t m, int6
         b.dtype = GEMM_BF16;
         b.lda = L.lda_p; b.ldb = L.ldb_p;
         Plan pb = make_plan(b, sms, ~(size_t)0);
-        return L.total + (pb.kernel < 0 ? 0 : pb.ws_total);
+        const size_t separate = L.total + (pb.kernel < 0 ? 0 : pb.ws_total);      // six launches
+        return separate > L.total_fused ? separate : L.total_fused;                // one launch (pieces side by side along k)
     }
     Plan p = make_plan(a, sms, ~(size_t)0);
     return p.kernel < 0 ? 0 : p.ws_total;

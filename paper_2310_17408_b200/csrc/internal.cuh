@@ -35,6 +35,8 @@ struct GemmArgs {
     int ct = 0;                        // tensor kernels: the roles of the operands were exchanged; C (m x n here) is stored as its
                                        // transpose: element (i, j) at C[j + i*ldc]
     int split3 = 0;                    // fp32 operands: multiply on the tensor cores as three bfloat16 pieces each (GEMM_F32_TC)
+    int64_t seg_k = 0;                 // CTA-pair kernel: A and B hold three bfloat16 pieces each, one after the other along k
+                                       // (seg_k entries of k per piece, a multiple of 64, zero padded; k = 3 * seg_k)
 };
 
 // The all-16-bit data types (GEMM_F16_C16, GEMM_BF16_C16) are a 16-bit input type plus a 16-bit result:
@@ -154,7 +156,7 @@ cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t
 // fp32 stored matrix (rows x cols, ld) -> three bfloat16 matrices p1, p2, p3 (leading dimension ld_p) with
 // x = p1 + p2 + p3 up to the last bit or two of x: p1 = bf16(x), p2 = bf16(x - p1), p3 = bf16(x - p1 - p2)
 cudaError_t launch_split3(const float* src, int64_t rows, int64_t cols, int64_t ld, void* p1, void* p2, void* p3,
-                          int64_t ld_p, cudaStream_t stream);
+                          int64_t ld_p, cudaStream_t stream, int64_t rows_out = 0, int64_t cols_out = 0);
 
 // launches a one-warp kernel whose bounded wait is certain to expire (nothing arrives at its barrier)
 cudaError_t launch_wait_expiry_probe(uint32_t* status, cudaStream_t stream);

@@ -249,20 +249,24 @@ cudaError_t launch_repack16(const void* src, int64_t rows, int64_t cols, int64_t
 // pieces left over; the subtractions are exact in fp32 (the piece shares the leading bits of what it was rounded from).
 __global__ void __launch_bounds__(256)
 split3_kernel(const float* __restrict__ src, int64_t rows, int64_t cols, int64_t ld, __nv_bfloat16* __restrict__ p1,
-              __nv_bfloat16* __restrict__ p2, __nv_bfloat16* __restrict__ p3, int64_t ld_p, int vec) {
-    const int64_t quads = (rows + 3) / 4;
-    for (int64_t j = blockIdx.y; j < cols; j += gridDim.y)
+              __nv_bfloat16* __restrict__ p2, __nv_bfloat16* __restrict__ p3, int64_t ld_p, int vec, int64_t rows_out,
+              int64_t cols_out) {
+    // rows_out (a multiple of 4) x cols_out entries of every piece are written: zeros beyond the rows x cols of the source
+    const int64_t quads = rows_out / 4;
+    for (int64_t j = blockIdx.y; j < cols_out; j += gridDim.y)
         for (int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q < quads; q += (int64_t)gridDim.x * blockDim.x) {
             const int64_t i = q * 4;
             float x[4] = {0.f, 0.f, 0.f, 0.f};
-            const float* s = src + i + j * ld;
-            if (vec && i + 3 < rows) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(s));
-                x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-            } else {
+            if (j < cols && i < rows) {
+                const float* s = src + i + j * ld;
+                if (vec && i + 3 < rows) {
+                    const float4 v = __ldg(reinterpret_cast<const float4*>(s));
+                    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+                } else {
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (i + e < rows) x[e] = __ldg(s + e);
+                    for (int e = 0; e < 4; ++e)
+                        if (i + e < rows) x[e] = __ldg(s + e);
+                }
             }
             uint16_t h[3][4];
 #pragma unroll
@@ -276,7 +280,6 @@ split3_kernel(const float* __restrict__ src, int64_t rows, int64_t cols, int64_t
                 }
             }
             // ld_p is a multiple of 8 and the pieces are 16-byte aligned: the four values of a piece go out as one 8-byte store
-            // (rows past the matrix, inside its last quad, are written as zeros: they lie in the padding of the copy)
             __nv_bfloat16* out[3] = {p1, p2, p3};
 #pragma unroll
             for (int t = 0; t < 3; ++t) {
@@ -286,16 +289,20 @@ split3_kernel(const float* __restrict__ src, int64_t rows, int64_t cols, int64_t
         }
 }
 
+// rows_out / cols_out: the extent written per piece (0 = the source's own, rows rounded up to 4); ld_p >= rows_out
 cudaError_t launch_split3(const float* src, int64_t rows, int64_t cols, int64_t ld, void* p1, void* p2, void* p3,
-                          int64_t ld_p, cudaStream_t stream) {
+                          int64_t ld_p, cudaStream_t stream, int64_t rows_out, int64_t cols_out) {
     if (rows == 0 || cols == 0) return cudaSuccess;
-    const int64_t quads = (rows + 3) / 4;
-    int64_t gx = (quads + 255) / 256, gy = cols;
+    if (rows_out == 0) rows_out = (rows + 3) / 4 * 4;
+    if (cols_out == 0) cols_out = cols;
+    if (rows_out % 4 != 0 || rows_out < rows || cols_out < cols || ld_p < rows_out) return cudaErrorInvalidValue;
+    const int64_t quads = rows_out / 4;
+    int64_t gx = (quads + 255) / 256, gy = cols_out;
     if (gx > 1024) gx = 1024;
     if (gy > 32768) gy = 32768;
     const int vec = ((reinterpret_cast<uintptr_t>(src) & 15) == 0 && ld % 4 == 0) ? 1 : 0;
     split3_kernel<<<dim3((unsigned)gx, (unsigned)gy), 256, 0, stream>>>(src, rows, cols, ld, (__nv_bfloat16*)p1, (__nv_bfloat16*)p2,
-                                                                     (__nv_bfloat16*)p3, ld_p, vec);
+                                                                     (__nv_bfloat16*)p3, ld_p, vec, rows_out, cols_out);
     return cudaGetLastError();
 }
 

@@ -39,7 +39,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k,
                     float alpha, float beta, float* __restrict__ C, int64_t ldc, int tiles_m, int tiles_n, int splits,
                     int64_t kchunk, float* __restrict__ partials, uint32_t idesc, uint32_t* status, const ConvTma conv,
-                    int out16) {
+                    int out16, int seg_kblocks) {
     constexpr int STAGES = PAIR_STAGES, NACC = PAIR_NACC, BN = PAIR_BN;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -98,7 +98,11 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         tm = g * GROUP + (tile % per_group) % gsz;
         tn = (tile % per_group) / gsz;
     };
+    // seg_kblocks > 0 (fp32 data as three bfloat16 pieces each): op(A) and op(B) hold their pieces one after the other
+    // along k, seg_kblocks k blocks per piece, and a tile's k loop walks six (piece of A, piece of B) segments, the
+    // smallest products first, all into the same accumulator
     auto kblocks_of = [&](int sp, int64_t& kbeg) {
+        if (seg_kblocks > 0) { kbeg = 0; return 6 * seg_kblocks; }
         kbeg = (int64_t)sp * kchunk;
         const int64_t kend = min(k, kbeg + kchunk);
         return (int)((kend - kbeg + TBK - 1) / TBK);
@@ -125,14 +129,20 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                    STATUS_MARK | (ROLE_TMA << 16) | (BAR_EMPTY << 8) | s)) { ok = false; break; }
                     const uint32_t sa = smem_base + s * PAIR_STAGE_BYTES;
                     const uint32_t sb = sa + PAIR_A_BYTES;
-                    const int32_t k0 = (int32_t)(kbeg + (int64_t)kb * TBK);
+                    int32_t k0 = (int32_t)(kbeg + (int64_t)kb * TBK), k0a = k0;
+                    if (seg_kblocks > 0) {
+                        // segments (piece of A, piece of B): (2,0) (0,2) (1,1) (1,0) (0,1) (0,0), two bits per entry
+                        const int seg = kb / seg_kblocks, kk = kb - seg * seg_kblocks;
+                        k0a = (int32_t)((((0x052 >> (2 * seg)) & 3) * seg_kblocks + kk) * TBK);
+                        k0 = (int32_t)((((0x118 >> (2 * seg)) & 3) * seg_kblocks + kk) * TBK);
+                    }
                     if (leader) mbar_expect_tx(full_bar(s), 2 * PAIR_STAGE_BYTES);   // both CTAs' bytes
                     const uint32_t fb = map_to_cta(full_bar(s), 0);
                     if (A_MN) {
 #pragma unroll
-                        for (int c = 0; c < TBM / 64; ++c) tma_load_2d_pair(&tmA, sa + c * (64 * TBK * 2), fb, m0 + c * 64, k0);
+                        for (int c = 0; c < TBM / 64; ++c) tma_load_2d_pair(&tmA, sa + c * (64 * TBK * 2), fb, m0 + c * 64, k0a);
                     } else {
-                        tma_load_2d_pair(&tmA, sa, fb, k0, m0);
+                        tma_load_2d_pair(&tmA, sa, fb, k0a, m0);
                     }
                     if (CONV) {
                         const int kg = k0 / TBK;
@@ -301,7 +311,8 @@ static cudaError_t launch_pair(const GemmArgs& a, KSplit ks, float* partials, ge
     cudaError_t le = cudaLaunchKernelEx(&lc, kern, tmA, tmB, tmC, store_via_tma, a.m, a.n, a.k, a.alpha, a.beta, a.C, a.ldc,
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         ks.splits > 1 ? partials : (float*)nullptr,
-                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status, conv_tma_params(a.conv), a.out16);
+                                        instr_desc(a.dtype, A_MN, B_MN, 2 * TBM, PAIR_BN), a.status, conv_tma_params(a.conv), a.out16,
+                                        (int)(a.seg_k / TBK));
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 

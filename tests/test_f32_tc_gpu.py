@@ -37,6 +37,22 @@ def test_split_precision_against_the_fp64_oracle(ta, tb):
             check_against_oracle(p, A, B, C0, C, integer=(kind == "int"))
 
 
+@pytest.mark.parametrize("ta,tb", list(itertools.product("NT", "NT")))
+def test_split_precision_as_one_launch_on_cta_pairs(ta, tb):
+    # enough 256 x 256 tiles for every CTA pair: the six piece products run as one multiplication whose k loop walks the
+    # pieces (stored one after the other along k, k padded to a multiple of 64 with zeros); ragged k, m, n and padding
+    for (m, n, k), pad in [((2350, 2400, 200), (0, 0, 0)), ((2305, 2562, 333), (3, 1, 2))]:
+        for kind, alpha, beta in [("uniform", 1.5, 0.5), ("int", -1.0, 1.0), ("uniform", 1.0, 0.0)]:
+            p = Problem("tc3p", DTYPE_F32, m, n, k, alpha, beta, ta, tb, kindA=kind, kindB=kind,
+                        kindC=kind if kind == "int" else "uniform", seed=m + k, pad=pad)
+            A, B, C0 = p.operands()
+            g.gemm_force_kernel(g.GEMM_KERNEL_TENSOR)      # below the size the selector sends to the tensor cores
+            C, cfg = run_problem(p, A, B, C0, api_dtype=TC)
+            g.gemm_force_kernel(g.GEMM_KERNEL_AUTO)
+            assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["launches"] == 3 and cfg["tile_m"] == 256, cfg
+            check_against_oracle(p, A, B, C0, C, integer=(kind == "int"))
+
+
 def test_split_precision_error_is_at_the_level_of_fp32_arithmetic():
     # the same problem through the exact fp32 kernel and through the three-piece path: both errors against the fp64
     # oracle are reported; the three-piece path must stay within a small multiple of the exact kernel's error
@@ -74,5 +90,5 @@ def test_split_precision_full_size_square():
     p = dataclasses.replace(config_problems(2)[2], name="sq4096_tc")      # 4096^3, alpha = 1.5, beta = 0.5
     A, B, C0 = p.operands()
     C, cfg = run_problem(p, A, B, C0, check_inputs=False, api_dtype=TC)
-    assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR
+    assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["launches"] == 3, cfg      # two splitting passes, one multiplication
     check_large(p, A, B, C0, C, cfg, seed=5)
