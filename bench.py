@@ -73,14 +73,14 @@ TRAFFIC = {
         "bytes": 3575662080 + 273164288, "source": "paper_2310_17408_b200/csrc/simt_fast.cu",
         "sha256": "9804c708bee85f95cd74403ad6bf228cfae6c0ec4a7f5c2cc2a687e997c259e9"},
     ("tc_gemm_pair_kernel", "8192x8192x8192", "bf16"): {
-        "bytes": 1101455104 + 261325312, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
-        "sha256": "8d1968c394593bfd009d17f5e7fd973d9745ffc862c1a1d0bf45dbe54b790fbb"},
+        "bytes": 1102845440 + 261591296, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
+        "sha256": "685014adedc009c9b779c6688ae86bec26bc19f5f047537ceaf5adfa1302e6b9"},
     ("tc_gemm_pair_kernel", "16384x16384x16384", "bf16"): {
-        "bytes": 14162072320 + 1103334144, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
-        "sha256": "8d1968c394593bfd009d17f5e7fd973d9745ffc862c1a1d0bf45dbe54b790fbb"},
+        "bytes": 17754797056 + 1102154240, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
+        "sha256": "685014adedc009c9b779c6688ae86bec26bc19f5f047537ceaf5adfa1302e6b9"},
     ("tc_gemm_pair_kernel", "16384x16384x16384", "f16"): {
-        "bytes": 18260333568 + 1103571712, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
-        "sha256": "8d1968c394593bfd009d17f5e7fd973d9745ffc862c1a1d0bf45dbe54b790fbb"},
+        "bytes": 22216240384 + 1103545344, "source": "paper_2310_17408_b200/csrc/tc_gemm_pair.cu",
+        "sha256": "685014adedc009c9b779c6688ae86bec26bc19f5f047537ceaf5adfa1302e6b9"},
 }
 
 
