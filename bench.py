@@ -290,7 +290,7 @@ def cpu_baseline(problems, operands, budget_s=30.0):
 # ------------------------------------------------------------------------------------------ CUDA arm
 
 def run_probes(g, torch, stream, peaks):
-    """The library's own peak-confirmation probes on this device: HBM copy, register-only fp32 FMA loops and
+    """The library's own peak-confirmation probes on this device: HBM copy, fp32 FMA loops (register-only chains and the SIMT micro-kernel fed from shared memory) and
     tcgen05.mma on shared-memory-resident operands.  Each is run a few times; best and median are reported."""
     out = {}
 

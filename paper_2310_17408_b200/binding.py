@@ -214,7 +214,8 @@ def gemm_probe_copy(dst, src, nbytes, stream=0):
 
 
 def gemm_probe_ffma(pattern, iters, stream=0):
-    """(rc, TFLOP/s, ms) of the register-only fp32 FMA loops (pattern 0 chains, 1 8x8 block, 2 packed 8x8 block)."""
+    """(rc, TFLOP/s, ms) of the fp32 FMA probes (pattern 0: register-only chains; 1 / 2: the SIMT kernel's 8 x 8 micro-kernel
+    fed from shared memory, scalar / packed)."""
     return _probe(_lib.gemm_probe_ffma, pattern, iters, stream)
 
 
