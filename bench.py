@@ -618,6 +618,9 @@ def measure_workload(ctx, problems, operands, workload_name, e2e_steps=None, ste
     if e2e:
         line["e2e"] = {"value": aggregate_throughput(flops_step, e2e_ms, world), "unit": "TFLOP/s",
                        "h2d_bytes_per_step": e2e[1], "d2h_bytes_per_step": e2e[2], "steps": e2e[3],
+                       # average rates over the whole step (the wire is idle while the last panels are multiplied)
+                       "h2d_gbs": e2e[1] / (e2e_ms * 1e-3) / 1e9, "d2h_gbs": e2e[2] / (e2e_ms * 1e-3) / 1e9,
+                       "ms_per_step": e2e_ms,
                        "api": "gemm_host (pinned host buffers, copies inside the timed region)"}
     g.gemm_set_workspace(0, 0, 0)
     del dev, host, ws
