@@ -26,6 +26,8 @@ SMALL = [
     (3, 10, 10, 128, 136, 3, 3, 2, 1),
     (1, 20, 17, 64, 40, 5, 5, 1, 2),
     (2, 6, 6, 192, 260, 1, 1, 2, 0),      # 1 x 1 with stride 2: a real gather
+    (2, 24, 25, 64, 48, 3, 3, 1, 1),      # 1200 pixels, 48 output channels (half-empty MMA rows on the tensor path)
+    (1, 70, 66, 128, 64, 3, 3, 2, 1),     # exactly 64 output channels, stride 2, 1155 pixels (ragged last tile)
     (1, 5, 150, 3, 4, 3, 3, 2, 1),        # a long image row with few channels
     (2, 4, 70, 5, 3, 5, 5, 1, 2),         # 70 per row, C_in = 5, wide filter
 ]
