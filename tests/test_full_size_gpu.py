@@ -140,3 +140,21 @@ def test_result_with_more_than_2_31_entries(dtype):
     assert not bool(torch.isnan(dC).any())
     del dC
     torch.cuda.empty_cache()
+
+
+def test_gemm_host_at_the_end_to_end_size_of_the_bench():
+    # config 2's largest member through the host-buffer entry point, as bench.py's e2e leg calls it (pinned buffers,
+    # alpha = 1.5, beta = 0.5): eight k panels of A, leading column panels joining one by one, the first panel and the
+    # first k panel cut in two.  Different summation order than gemm(), same bound.
+    import torch
+    p = config_problems(2)[3]
+    A, B, C0 = p.operands()
+    C = C0.copy()
+    pinned = [torch.from_numpy(x.buf).pin_memory() for x in (A, B, C)]
+    rc = g.gemm_host(p.api_dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, pinned[0].data_ptr(), A.ld, pinned[1].data_ptr(),
+                     B.ld, p.beta, pinned[2].data_ptr(), C.ld, torch.cuda.current_stream().cuda_stream)
+    assert rc == 0, g.gemm_status_string(rc)
+    assert g.gemm_poll_status() == 0
+    C.buf[:] = pinned[2].numpy()
+    cfg = g.gemm_last_config()
+    check_large(p, A, B, C0, C, cfg, seed=11)
