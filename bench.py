@@ -46,6 +46,9 @@ WORKLOADS = {
     "cfg5_bf16_squares": lambda: config_problems(5, dtype=DTYPE_BF16)[:3],
     # config 5 with the result in the operands' 16-bit type as well (the library's GEMM_BF16_C16)
     "cfg5_bf16_c16": lambda: config_problems(5, dtype=DTYPE_BF16, c16=True),
+    # the paper's f16 arithmetic: binary16 operands, accumulator and result (GEMM_F16_ACC16)
+    "cfg5_f16_acc16": lambda: [__import__("dataclasses").replace(p, name=p.name + "_acc16", acc16=True)
+                               for p in config_problems(5, dtype=DTYPE_F16, c16=True)],
     # second workload (VGG16, batch 32) and the paper's own orientation (m = batch*pixels, n = channels)
     "vgg16_fp32": lambda: im2row_problems("vgg16"),
     "vgg16_bf16": lambda: im2row_problems("vgg16", dtype=DTYPE_BF16),

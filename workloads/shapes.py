@@ -111,6 +111,7 @@ class Problem:
     pad: tuple = field(default=(0, 0, 0))   # extra leading-dimension rows for A, B, C
     c16: bool = False                       # C in the 16-bit type of A and B (the library's *_C16 data types)
     tc3: bool = False                       # fp32 data multiplied on the tensor cores as three bfloat16 pieces (GEMM_F32_TC)
+    acc16: bool = False                     # binary16 data, binary16 accumulator (GEMM_F16_ACC16; set together with c16)
 
     @property
     def flops(self) -> float:
@@ -121,6 +122,8 @@ class Problem:
         """Data-type code of the library call: dtype, or its all-16-bit form (3 = f16, 4 = bf16) when C is 16-bit."""
         if self.tc3:
             return 5
+        if self.acc16:
+            return 6
         return self.dtype + 2 if self.c16 else self.dtype
 
     def algorithmic_bytes(self) -> float:
