@@ -44,6 +44,9 @@ WORKLOADS = {
     "cfg5_bf16": lambda: config_problems(5, dtype=DTYPE_BF16),
     "cfg5_f16_squares": lambda: config_problems(5, dtype=DTYPE_F16)[:3],
     "cfg5_bf16_squares": lambda: config_problems(5, dtype=DTYPE_BF16)[:3],
+    # the same squares with A stored transposed (both operands contiguous along k), for information
+    "cfg5_bf16_squares_tn": lambda: [__import__("dataclasses").replace(p, name=p.name + "_tn", transA="T")
+                                     for p in config_problems(5, dtype=DTYPE_BF16)[:3]],
     # config 5 with the result in the operands' 16-bit type as well (the library's GEMM_BF16_C16)
     "cfg5_bf16_c16": lambda: config_problems(5, dtype=DTYPE_BF16, c16=True),
     # the paper's f16 arithmetic: binary16 operands, accumulator and result (GEMM_F16_ACC16)
@@ -527,7 +530,18 @@ def measure_workload(ctx, problems, operands, workload_name, e2e_steps=None, ste
             except Exception as exc:          # graph capture is a measurement convenience, not part of the contract
                 sys.stderr.write(f"graph timing skipped for {p.name}: {exc}\n")
                 graph_ms = None
-        return stream_ms, host_us, nsets, reps, graph_ms
+        # twenty calls timed one by one (an event pair around each; the pair itself costs a few microseconds, which shows
+        # on the shortest calls): median and best
+        singles = []
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+        for r, (a0, a1) in enumerate(pairs):
+            a0.record()
+            call(r)
+            a1.record()
+        torch.cuda.synchronize()
+        singles = sorted(a0.elapsed_time(a1) for a0, a1 in pairs)
+        one_by_one = {"median": statistics.median(singles), "best": singles[0]}
+        return stream_ms, host_us, nsets, reps, graph_ms, one_by_one
 
     b2b = []
     for i, p in enumerate(problems):
@@ -574,10 +588,11 @@ def measure_workload(ctx, problems, operands, workload_name, e2e_steps=None, ste
         avg = sum(ms) / len(ms)
         bound, peak, unit, amount = roofline_class(p, peaks)
         achieved = amount / (avg * 1e-3)
-        cold_ms, host_us, nsets, reps, graph_ms = b2b[i]
+        cold_ms, host_us, nsets, reps, graph_ms, one_by_one = b2b[i]
         shapes.append({"name": p.name, "m": p.m, "n": p.n, "k": p.k, "ms_in_step": avg, "ms": cold_ms,
                        "tflops": p.flops / (cold_ms * 1e-3) / 1e12, "gbs": p.algorithmic_bytes() / (cold_ms * 1e-3) / 1e9,
                        "bound": bound, "frac": amount / (cold_ms * 1e-3) / peak, "frac_in_step": achieved / peak,
+                       "ms_single_median": one_by_one["median"], "ms_single_best": one_by_one["best"],
                        "ms_graph": graph_ms, "frac_graph": (amount / (graph_ms * 1e-3) / peak) if graph_ms else None,
                        "host_us_per_call": host_us, "operand_sets": nsets, "calls": reps, "kernel": configs[i]["kernel"],
                        "tile": [configs[i]["tile_m"], configs[i]["tile_n"]], "split_k": configs[i]["split_k"], "tail_split": configs[i].get("tail_split", 0),
@@ -612,7 +627,7 @@ def measure_workload(ctx, problems, operands, workload_name, e2e_steps=None, ste
             "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": DTYPE_NAMES[problems[0].dtype], "data": "synthetic",
             "config": {"workload": workload_name, "problems": [f"{q.m}x{q.n}x{q.k}" for q in problems],
-                       "alpha": problems[0].alpha, "beta": problems[0].beta, "layout": "column-major N,N",
+                       "alpha": problems[0].alpha, "beta": problems[0].beta, "layout": f"column-major {problems[0].transA},{problems[0].transB}",
                        "l2": "inputs larger than L2: one step touches more than 126 MB of operands"
                              if sum(q.algorithmic_bytes() for q in problems) > 126e6 else
                              "working set smaller than L2 (warm-cache number)",
