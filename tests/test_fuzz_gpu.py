@@ -107,3 +107,63 @@ def test_random_convolution_layers(chunk):
             assert float(np.max(np.abs(got - ref))) <= slack, tag
         else:
             assert float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-30)) <= 1e-3, tag
+
+
+@pytest.mark.parametrize("chunk", range(3))
+def test_random_cases_on_the_special_paths(chunk):
+    """Shapes drawn where the selector leaves the common kernels: few rows and many columns (exchanged operand roles),
+    few tiles and long k (split k summed by clusters, or by the separate pass when forced), tiny problems (the kernel
+    without staging), fp32 data on the tensor cores in both of its forms, and host buffers through gemm_host."""
+    import torch
+    rng = np.random.default_rng(777 + chunk)
+    ensure_workspace(512 << 20)
+    for i in range(24):
+        g.gemm_force_kernel(g.GEMM_KERNEL_AUTO)
+        g.gemm_force_tile(0, 0, 0)
+        g.gemm_force_reduction(0)
+        what = str(rng.choice(["roles", "cluster", "tiny", "tc3", "tc3_one_launch", "host"]))
+        ta, tb = str(rng.choice(["N", "T"])), str(rng.choice(["N", "T"]))
+        alpha, beta = [(1.0, 0.0), (1.5, 0.5), (-1.0, 1.0), (0.25, -2.0)][int(rng.integers(0, 4))]
+        pad = tuple(int(x) for x in rng.choice([0, 1, 3, 4, 8], 3))
+        integer = bool(rng.integers(0, 3) == 0)
+        api = None
+        if what == "roles":
+            dt = int(rng.choice([DTYPE_F16, DTYPE_BF16]))
+            m, n, k = int(rng.integers(1, 65)), int(rng.integers(1024, 6000)), int(rng.choice([8, 27, 64, 147, 152, 256, 576, 1000]))
+        elif what == "cluster":
+            dt = int(rng.choice([DTYPE_F32, DTYPE_BF16]))
+            m, n, k = int(rng.choice([64, 128, 200, 256, 512])), int(rng.choice([64, 128, 300, 512, 1568])), int(rng.choice([512, 1024, 2304, 4608]))
+            if rng.integers(0, 2):
+                g.gemm_force_reduction(int(rng.choice([1, 2])))
+        elif what == "tiny":
+            dt, (m, n, k) = DTYPE_F32, (int(rng.integers(1, 260)), int(rng.integers(1, 260)), int(rng.integers(1, 400)))
+        elif what == "tc3":
+            dt, api = DTYPE_F32, g.GEMM_F32_TC
+            m, n, k = int(rng.integers(129, 900)), int(rng.integers(128, 900)), int(rng.integers(64, 1200))
+            g.gemm_force_kernel(g.GEMM_KERNEL_TENSOR)
+        elif what == "tc3_one_launch":
+            dt, api = DTYPE_F32, g.GEMM_F32_TC
+            m, n, k = int(rng.integers(1025, 2600)), int(rng.integers(1025, 2600)), int(rng.integers(64, 400))
+            g.gemm_force_kernel(g.GEMM_KERNEL_TENSOR)
+        else:
+            dt = int(rng.choice([DTYPE_F32, DTYPE_BF16]))
+            m, n, k = int(rng.integers(1, 700)), int(rng.integers(1, 3000)), int(rng.integers(0, 900))
+        kind = "int" if integer else ("uniform" if dt == DTYPE_F32 else "normal")
+        p = Problem("f", dt, m, n, k, alpha, beta, ta, tb, kindA=kind, kindB=kind, kindC="int" if integer else "uniform",
+                    seed=chunk * 100 + i, pad=pad)
+        tag = f"case {chunk}/{i}: {what} dtype={dt} {ta}{tb} {m}x{n}x{k} alpha={alpha} beta={beta} pad={pad} integer={integer}"
+        A, B, C0 = p.operands()
+        try:
+            if what == "host":
+                C = C0.copy()
+                rc = g.gemm_host(dt, ta, tb, m, n, k, alpha, A.buf.ctypes.data, A.ld, B.buf.ctypes.data, B.ld, beta,
+                                 C.buf.ctypes.data, C.ld, torch.cuda.current_stream().cuda_stream)
+                assert rc == 0 and g.gemm_poll_status() == 0 and C.padding_intact()
+            else:
+                C, _ = run_problem(p, A, B, C0, api_dtype=api)
+            check_against_oracle(p, A, B, C0, C, integer=integer)
+        except AssertionError as exc:
+            raise AssertionError(f"{tag}: {exc}") from exc
+        finally:
+            g.gemm_force_kernel(g.GEMM_KERNEL_AUTO)
+            g.gemm_force_reduction(0)
