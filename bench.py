@@ -754,6 +754,10 @@ BATCHED_WORKLOADS = {
     # (m, n, k, batch): many small fp32 problems in one call of gemm_strided_batched
     "batched_fp32_small": [(64, 64, 64, 4096), (32, 32, 32, 16384), (16, 16, 16, 65535), (128, 128, 128, 1024),
                            (96, 96, 200, 2048), (256, 256, 256, 128)],
+    # the same through the tensor cores: bf16 operands, fp32 results, one launch per call (problem index = third
+    # coordinate of the operand maps)
+    "batched_bf16_small": [(64, 64, 64, 4096), (128, 128, 128, 1024), (96, 96, 200, 2048), (256, 256, 256, 128),
+                           (512, 512, 512, 32), (128, 128, 64, 8192)],
 }
 
 
@@ -769,6 +773,8 @@ def run_batched(args, cases, workload_name):
     torch.cuda.set_device(0)
     peaks = load_peaks()
     stream = torch.cuda.current_stream().cuda_stream
+    half = "bf16" in workload_name
+    api_dtype, es, tdt = (DTYPE_BF16, 2, torch.bfloat16) if half else (DTYPE_F32, 4, torch.float32)
     rows, step_ms, step_flops, launches = [], 0.0, 0.0, 0
     sampler = ClockSampler(0)
     sampler.start()
@@ -777,15 +783,15 @@ def run_batched(args, cases, workload_name):
         A1 = torch.from_numpy(make_matrix(m, k, kind="uniform", seed=7000 + idx, matrix_id=0).buf).cuda()
         B1 = torch.from_numpy(make_matrix(k, n, kind="uniform", seed=7000 + idx, matrix_id=1).buf).cuda()
         sign = (1.0 - 2.0 * (torch.arange(batch, device="cuda") % 2)).float()[:, None]
-        bytes_call = 4.0 * (m * k + k * n + m * n) * batch
+        bytes_call = (es * (m * k + k * n) + 4.0 * m * n) * batch
         flops = 2.0 * m * n * k * batch
         nsets = int(min(16, max(1, -(-2 * 126e6 // bytes_call))))
-        sets = [((A1[None, :] * sign).contiguous(), (B1[None, :] * sign).contiguous(), torch.empty(batch * m * n, device="cuda"))
+        sets = [((A1[None, :] * sign).to(tdt).contiguous(), (B1[None, :] * sign).to(tdt).contiguous(), torch.empty(batch * m * n, device="cuda"))
                 for _ in range(nsets)]
 
         def call(r):
             a, b, c = sets[r % nsets]
-            rc = g.gemm_strided_batched(DTYPE_F32, "N", "N", m, n, k, 1.0, a.data_ptr(), m, m * k, b.data_ptr(), k, k * n, 0.0,
+            rc = g.gemm_strided_batched(api_dtype, "N", "N", m, n, k, 1.0, a.data_ptr(), m, m * k, b.data_ptr(), k, k * n, 0.0,
                                         c.data_ptr(), m, m * n, batch, stream)
             if rc != 0:
                 raise RuntimeError(f"gemm_strided_batched failed: {rc}")
@@ -802,9 +808,10 @@ def run_batched(args, cases, workload_name):
         ms = e0.elapsed_time(e1) / reps
         cfg = g.gemm_last_config()
         launches += reps * cfg["launches"]
-        t_cmp = flops / (fp32_alu_peak_tflops(peaks["sm_max_mhz"]) * 1e12)
+        cmp_peak = peaks["tensor_tflops"] if half else fp32_alu_peak_tflops(peaks["sm_max_mhz"])
+        t_cmp = flops / (cmp_peak * 1e12)
         t_hbm = bytes_call / (peaks["hbm_gbs"] * 1e9)
-        bound = "alu" if t_cmp >= t_hbm else "hbm"
+        bound = ("tensor" if half else "alu") if t_cmp >= t_hbm else "hbm"
         rows.append({"name": f"{m}x{n}x{k}x{batch}", "m": m, "n": n, "k": k, "batch": batch, "ms": ms,
                      "tflops": flops / (ms * 1e-3) / 1e12, "gbs": bytes_call / (ms * 1e-3) / 1e9, "bound": bound,
                      "frac": max(t_cmp, t_hbm) / (ms * 1e-3), "kernel": cfg["kernel"], "tile": [cfg["tile_m"], cfg["tile_n"]],
@@ -819,13 +826,15 @@ def run_batched(args, cases, workload_name):
     dom = max(rows, key=lambda r: r["ms"])
     line = {"metric": "gemm_tflops", "value": step_flops / (step_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": 1,
             "steps": max(args.steps, 10), "warmup": 3, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16" if half else "f32", "data": "synthetic",
             "config": {"workload": workload_name, "api": "gemm_strided_batched", "layout": "column-major N,N, dense strides",
                        "l2": "calls cycle through operand sets larger than L2", "parallelism": "single GPU"},
-            "roofline": {"bound": dom["bound"], "achieved": dom["tflops"] if dom["bound"] == "alu" else dom["gbs"],
-                         "peak": fp32_alu_peak_tflops(peaks["sm_max_mhz"]) if dom["bound"] == "alu" else peaks["hbm_gbs"],
-                         "unit": "TFLOP/s" if dom["bound"] == "alu" else "GB/s", "frac": dom["frac"], "traffic": None,
-                         "kernel": {2: "simt_batched_kernel", 4: "simt_direct_kernel", 1: "simt_generic_kernel"}.get(dom["kernel"], "?"),
+            "roofline": {"bound": dom["bound"], "achieved": dom["gbs"] if dom["bound"] == "hbm" else dom["tflops"],
+                         "peak": peaks["hbm_gbs"] if dom["bound"] == "hbm" else
+                                 (peaks["tensor_tflops"] if half else fp32_alu_peak_tflops(peaks["sm_max_mhz"])),
+                         "unit": "GB/s" if dom["bound"] == "hbm" else "TFLOP/s", "frac": dom["frac"], "traffic": None,
+                         "kernel": {2: "simt_batched_kernel", 4: "simt_direct_kernel", 1: "simt_generic_kernel",
+                                    3: "tc_gemm_kernel"}.get(dom["kernel"], "?"),
                          "problem": dom["name"]},
             "clocks": clocks, "gpu_launches": launches, "shapes": rows}
     print(json.dumps(line))

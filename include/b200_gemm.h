@@ -126,8 +126,10 @@ int gemm(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t k,
  * non-packed variant reads A where it lies, because for small problems the packing is not paid back); here
  * small fp32 problems (and every fp32 gemm() call below the same size) run in a kernel that reads its operands
  * from global memory straight into registers, without shared-memory staging, workspace or reduction pass, larger
- * ones share one launch of the register-blocked kernel, small 16-bit problems one launch of the bounds-checked
- * kernel, and problems large enough to fill the GPU on their own go through gemm() one by one.
+ * ones share one launch of the register-blocked kernel.  16-bit batches whose operands TMA can address (16-byte
+ * aligned A and B, lda, ldb, strideA and strideB multiples of 8 elements) run as ONE launch of the tensor-core
+ * kernel, the problem index being the third coordinate of the operand maps; other small 16-bit problems share one
+ * launch of the bounds-checked kernel, and what is left goes through gemm() one by one.
  * Returns GEMM_OK, -(position of the first invalid argument of THIS function; 10, 13, 17 = the strides, 18 = batch)
  * or a GEMM_ERR_* code.  Asynchronous on `stream`.
  */

@@ -758,6 +758,22 @@ int gemm_strided_batched(int dtype, char transA, char transB, int64_t m, int64_t
         t_last_cfg = cfg;
         return e == cudaSuccess ? GEMM_OK : fail_launch(e);
     }
+    // 16-bit batches on the tensor cores in one launch, when TMA can address the operands of every problem: 16-byte
+    // aligned bases, leading dimensions and batch strides (a shared operand, stride 0, is fine)
+    if (a.dtype != GEMM_F32 && !a.acc16 && forced != GEMM_KERNEL_SIMT_GENERIC && st->arch_ok && batch > 1 && k > 0 && alpha != 0.0f &&
+        g_force_tile_m == 0 && g_force_split == 0 && m <= 0x7FFFFFFFLL && n <= 0x7FFFFFFFLL && k <= 0x7FFFFFFFLL &&
+        (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (reinterpret_cast<uintptr_t>(B) & 15) == 0 && lda % 8 == 0 && ldb % 8 == 0 &&
+        strideA % 8 == 0 && strideB % 8 == 0 && strideA >= 0 && strideB >= 0 && (double)m * n * batch >= 128.0 * 128.0 * 8.0) {
+        const int tile_n = n <= 64 ? 64 : (n <= 128 ? 128 : 256);
+        e = launch_tensor_batched(a, tile_n, strideA, strideB, strideC, batch, &cfg);
+        if (e == cudaSuccess) {
+            cfg.launches = 1;
+            t_last_cfg = cfg;
+            return GEMM_OK;
+        }
+        (void)cudaGetLastError();      // a map the driver would not encode: the paths below take the batch
+        e = cudaSuccess;
+    }
     if (forced == GEMM_KERNEL_SIMT_GENERIC || (a.dtype != GEMM_F32 && work <= 128.0 * 128.0 * 128.0)) {
         for (int64_t b0 = 0; b0 < batch && e == cudaSuccess; b0 += CHUNK, ++launches)
             e = launch_simt_generic(at(b0), &cfg, strideA, strideB, strideC, std::min(CHUNK, batch - b0));

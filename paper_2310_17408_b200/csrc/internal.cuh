@@ -147,6 +147,8 @@ bool tensor_eligible(const GemmArgs& a);
 // distributed shared memory (no partials, no reduction pass)
 cudaError_t launch_tensor(const GemmArgs& a, int tile_n, KSplit ks, float* partials, gemm_config_t* cfg, bool cluster = false);
 // the same on CTA pairs (tcgen05 cta_group::2): 256 x 256 tiles, two SMs per tile
+cudaError_t launch_tensor_batched(const GemmArgs& a, int tile_n, int64_t strideA, int64_t strideB, int64_t strideC,
+                                  int64_t batch, gemm_config_t* cfg);
 cudaError_t launch_tensor_pair(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg);
 
 // copy op-independent stored matrix (rows x cols, ld) of 16-bit elements into an aligned layout (ld_out)

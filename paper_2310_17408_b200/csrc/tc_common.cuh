@@ -65,6 +65,13 @@ __device__ __forceinline__ void tma_load_2d(const CUtensorMap* tm, uint32_t dst,
         ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
+// the same from a 3-D map (a strided batch of matrices: the third coordinate is the problem index, the box one deep)
+__device__ __forceinline__ void tma_load_3d(const CUtensorMap* tm, uint32_t dst, uint32_t bar, int32_t c0, int32_t c1, int32_t c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
 // TMA load in im2col mode from an NHWC tensor (tensor map dimensions C, W, H, N): the box holds `pixelsPerColumn`
 // consecutive output pixels starting at the one whose receptive field begins at (w, h) of image n, each with
 // `channelsPerPixel` channels from c on, read at filter-tap offset (off_w, off_h); positions outside the image are
@@ -427,6 +434,9 @@ __device__ __forceinline__ void epilogue_tile16(uint32_t tmem_acc, int64_t row0,
 // (stride ld); 128-byte swizzle
 bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_t cols, int64_t ld,
               uint32_t box_rows, uint32_t box_cols);
+// map over a strided batch of such operands: dim2 = problem index, `stride` elements apart (a multiple of 8), box one deep
+bool make_map_batched(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_t cols, int64_t ld, int64_t stride,
+                      int64_t batch, uint32_t box_rows, uint32_t box_cols);
 // map over the split-k partial sums [split][n][m] (fp32, dense): 32 x 32 x 1 boxes
 bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits);
 // map over the result (fp32, or the 16-bit type out16) for the epilogue's tile stores: 32 x 32 boxes, no swizzle

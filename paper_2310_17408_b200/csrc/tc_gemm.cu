@@ -93,7 +93,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
-               uint32_t idesc, uint32_t* status, const ConvTma conv, int out16, int cluster_k) {
+               uint32_t idesc, uint32_t* status, const ConvTma conv, int out16, int cluster_k, int batched,
+               int64_t batch_c_bytes) {
+    // batched != 0: a strided batch of problems.  `splits` is then the number of problems and the slab index of a work
+    // item the problem index: tmA and tmB are 3-D maps with the problem as third coordinate (bit 1 / bit 2 of `batched`:
+    // A / B is one matrix shared by all problems), every item runs over the whole of k, and problem p's result starts
+    // batch_c_bytes * p behind C.
     using Cfg = TcCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     constexpr bool OUT16 = OUT == 1 || OUT == 2, ACC16 = OUT == 2, CT = OUT == 3;
@@ -162,6 +167,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tn = (tile % per_group) / gsz;
     };
     auto kblocks_of = [&](int sp, int64_t& kbeg) {
+        if (batched) { kbeg = 0; return (int)((k + TBK - 1) / TBK); }
         kbeg = (int64_t)sp * kchunk;
         const int64_t kend = min(k, kbeg + kchunk);
         return (int)((kend - kbeg + TBK - 1) / TBK);
@@ -189,6 +195,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t sb = sa + Cfg::A_BYTES;
                     const int32_t k0 = (int32_t)(kbeg + (int64_t)kb * TBK);
                     mbar_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+                    if (batched) {
+                        const int32_t pa = (batched & 2) ? 0 : sp, pb = (batched & 4) ? 0 : sp;
+                        if (A_MN) {
+#pragma unroll
+                            for (int c = 0; c < TBM / 64; ++c)
+                                tma_load_3d(&tmA, sa + c * (64 * TBK * 2), full_bar(s), m0 + c * 64, k0, pa);
+                        } else {
+                            tma_load_3d(&tmA, sa, full_bar(s), k0, m0, pa);
+                        }
+                        if (B_MN) {
+#pragma unroll
+                            for (int c = 0; c < BN / 64; ++c)
+                                tma_load_3d(&tmB, sb + c * (64 * TBK * 2), full_bar(s), n0 + c * 64, k0, pb);
+                        } else {
+                            tma_load_3d(&tmB, sb, full_bar(s), k0, n0, pb);
+                        }
+                        continue;
+                    }
                     if (A_MN) {
 #pragma unroll
                         for (int c = 0; c < TBM / 64; ++c) tma_load_2d(&tmA, sa + c * (64 * TBK * 2), full_bar(s), m0 + c * 64, k0);
@@ -276,8 +300,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                            STATUS_MARK | (ROLE_EPI << 16) | (BAR_TMEM_FULL << 8) | acc)) { ok = false; break; }
             tc_fence_after();
             const int64_t row0 = (int64_t)tm * TBM + q * 32;
-            const bool raw = splits > 1;
+            const bool raw = splits > 1 && !batched;
             float* out = raw ? partials + (int64_t)sp * m * n : C;
+            if (batched) out = reinterpret_cast<float*>(reinterpret_cast<char*>(C) + (int64_t)sp * batch_c_bytes);
             // store_via_tma: 0 = direct stores, 1 = tmC maps C (2-D), 2 = tmC maps the split-k partials (3-D: m, n, split)
             const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
             auto release = [&]() {      // the accumulator may be overwritten once this warp has read its last chunk
@@ -438,6 +463,27 @@ bool make_map(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_
     });
 }
 
+bool make_map_batched(CUtensorMap* tm, int dtype, const void* base, int64_t rows, int64_t cols, int64_t ld, int64_t stride,
+                      int64_t batch, uint32_t box_rows, uint32_t box_cols) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    if (batch > 1 && (stride <= 0 || stride % 8 != 0)) return false;
+    if (batch <= 1) stride = ld * (cols > 0 ? cols : 1);      // a single problem: any legal value
+    if (rows > 0xFFFFFFFFLL || cols > 0xFFFFFFFFLL || box_rows > 0xFFFF || box_cols > 0xFFFF) return false;
+    const MapKey k{{4, (uint64_t)dtype | ((uint64_t)box_rows << 16) | ((uint64_t)box_cols << 32), (uint64_t)(uintptr_t)base,
+                    ((uint64_t)rows << 32) | (uint64_t)cols, (uint64_t)ld, (uint64_t)stride, (uint64_t)batch}};
+    return cached_map(tm, k, [&](CUtensorMap* out) {
+        cuuint64_t dims[3] = {(cuuint64_t)rows, (cuuint64_t)cols, (cuuint64_t)batch};
+        cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)stride * 2};
+        cuuint32_t box[3] = {box_rows, box_cols, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = fn(out, dtype == GEMM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                        const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        return r == CUDA_SUCCESS;
+    });
+}
+
 // map over the split-k partial sums [split][n][m] (fp32, dense): 32 x 32 x 1 boxes
 bool make_partials_map(CUtensorMap* tm, const float* base, int64_t m, int64_t n, int splits) {
     EncodeTiledFn fn = encode_fn();
@@ -559,7 +605,7 @@ uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n, bool 
 template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
                              const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma,
-                             bool cluster = false) {
+                             bool cluster = false, int batched = 0, int64_t batch_c_bytes = 0) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
     static std::atomic<bool> attr_set[64];      // zero-initialised; set once per device
@@ -599,8 +645,46 @@ static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm
                                         (int)tiles_m, (int)tiles_n, ks.splits, ks.chunk,
                                         (ks.splits > 1 && !cluster) ? partials : (float*)nullptr,
                                         instr_desc(a.dtype, A_MN, B_MN, TBM, BN, OUT == 2), a.status, conv_tma_params(a.conv), a.out16,
-                                        cluster ? ks.splits : 0);
+                                        cluster ? ks.splits : 0, batched, batch_c_bytes);
     return le != cudaSuccess ? le : cudaGetLastError();
+}
+
+// A strided batch of 16-bit problems in one launch: 3-D maps of A and B (a shared operand, stride 0, keeps its 2-D
+// extent with one problem in the third dimension), KSplit.splits carries the number of problems.
+template <bool A_MN, bool B_MN>
+static cudaError_t launch_tc_batched(const GemmArgs& a, int tile_n, int64_t strideA, int64_t strideB, int64_t strideC,
+                                     int64_t batch, gemm_config_t* cfg) {
+    if (batch < 1 || batch > 0x7FFFFFFFLL || a.conv || a.acc16 || a.ct) return cudaErrorInvalidConfiguration;
+    CUtensorMap tmA, tmB;
+    const int64_t na = strideA == 0 ? 1 : batch, nb = strideB == 0 ? 1 : batch;
+    bool ok = A_MN ? make_map_batched(&tmA, a.dtype, a.A, a.m, a.k, a.lda, strideA, na, 64, TBK)
+                   : make_map_batched(&tmA, a.dtype, a.A, a.k, a.m, a.lda, strideA, na, TBK, TBM);
+    ok = ok && (B_MN ? make_map_batched(&tmB, a.dtype, a.B, a.n, a.k, a.ldb, strideB, nb, 64, TBK)
+                     : make_map_batched(&tmB, a.dtype, a.B, a.k, a.n, a.ldb, strideB, nb, TBK, (uint32_t)tile_n));
+    if (!ok) return cudaErrorInvalidValue;
+    const int flags = 1 | (strideA == 0 ? 2 : 0) | (strideB == 0 ? 4 : 0);
+    const int64_t c_bytes = strideC * (a.out16 ? 2 : 4);
+    const KSplit ks{(int)batch, a.k};
+    switch (tile_n) {
+        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, false, 1>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
+                                  : launch_tc<256, A_MN, B_MN, false, 0>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
+        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, false, 1>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
+                                  : launch_tc<128, A_MN, B_MN, false, 0>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
+        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, false, 1>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
+                                  : launch_tc<64, A_MN, B_MN, false, 0>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
+    }
+}
+
+cudaError_t launch_tensor_batched(const GemmArgs& a, int tile_n, int64_t strideA, int64_t strideB, int64_t strideC,
+                                  int64_t batch, gemm_config_t* cfg) {
+    cfg->kernel = GEMM_KERNEL_TENSOR;
+    cfg->split_k = 1;
+    cfg->vector_a = cfg->vector_b = 1;
+    const bool a_mn = !a.ta, b_mn = a.tb;
+    if (a_mn && b_mn) return launch_tc_batched<true, true>(a, tile_n, strideA, strideB, strideC, batch, cfg);
+    if (a_mn && !b_mn) return launch_tc_batched<true, false>(a, tile_n, strideA, strideB, strideC, batch, cfg);
+    if (!a_mn && b_mn) return launch_tc_batched<false, true>(a, tile_n, strideA, strideB, strideC, batch, cfg);
+    return launch_tc_batched<false, false>(a, tile_n, strideA, strideB, strideC, batch, cfg);
 }
 
 template <bool A_MN, bool B_MN, bool CONV>

@@ -150,10 +150,35 @@ def test_batched_16bit_inputs(dtype):
         cfg = run_batched(dtype, 40, 56, 72, ta, tb, 1.5, 0.5, 5, "int", pad=(8, 0, 1))
         assert cfg["kernel"] == g.GEMM_KERNEL_SIMT_GENERIC and cfg["launches"] == 1
         run_batched(dtype, 40, 56, 72, ta, tb, 1.0, 0.0, 3, "normal", seed=3)
-    # problems large enough for the tensor cores run through gemm() one by one
+    # operands TMA cannot address (leading dimension not a multiple of 8): problems large enough for the tensor cores
+    # run through gemm() one by one
     ensure_workspace(64 << 20)
-    cfg = run_batched(dtype, 256, 264, 320, "N", "N", 1.0, 0.0, 3, "int")
+    cfg = run_batched(dtype, 256, 264, 320, "N", "N", 1.0, 0.0, 3, "int", pad=(3, 0, 0))
     assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["launches"] >= 3
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+@pytest.mark.parametrize("ta,tb", TRANS)
+def test_batched_16bit_on_the_tensor_cores_in_one_launch(dtype, ta, tb):
+    # addressable operands (16-byte aligned bases, leading dimensions and batch strides): the whole batch is one launch
+    # of the tensor kernel, the problem index being the third coordinate of the operand maps.  Ragged m, n, k (the
+    # boxes are clipped per problem), padded leading dimensions, gaps between the problems, C read and written.
+    for (m, n, k), batch, pad, gap in [((64, 64, 64), 40, (0, 0, 0), (0, 0, 0)), ((200, 136, 72), 7, (8, 8, 3), (8, 16, 5)),
+                                       ((130, 300, 200), 5, (16, 0, 1), (0, 8, 0)), ((8, 520, 1000), 40, (0, 8, 0), (8, 0, 3))]:
+        # leading dimensions must come out as multiples of 8: stored rows are m, k or n depending on the flags
+        rows_a, rows_b = (m if ta == "N" else k), (k if tb == "N" else n)
+        pad_ok = ((-rows_a) % 8 + pad[0], (-rows_b) % 8 + pad[1], pad[2])
+        for kind, alpha, beta in (("int", 1.5, 0.5), ("normal", 1.0, 0.0), ("normal", -1.0, 1.0)):
+            cfg = run_batched(dtype, m, n, k, ta, tb, alpha, beta, batch, kind, seed=11, pad=pad_ok, gap=gap)
+            assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["launches"] == 1, (m, n, k, cfg)
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+def test_batched_16bit_shared_operands_on_the_tensor_cores(dtype):
+    for shared in (dict(shared_a=True), dict(shared_b=True), dict(shared_a=True, shared_b=True)):
+        cfg = run_batched(dtype, 136, 200, 264, "N", "T", 1.5, 0.5, 6, "int", seed=5, **shared)
+        assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["launches"] == 1, cfg
+        run_batched(dtype, 136, 200, 264, "T", "N", 1.0, 0.0, 6, "normal", seed=6, **shared)
 
 
 def test_batched_argument_checks():

@@ -174,3 +174,37 @@ def test_convolution_layers_with_sixteen_bit_results(dtype):
         u = ulp16(ref, dtype)
         slack = oracle.fp32_tolerance(k, p.alpha, p.beta, X.max_abs(), W.max_abs(), Y0.max_abs()) + u / 64
         assert not (np.abs(Y.as_f64() - ref) > u / 2 + slack).any()
+
+
+@pytest.mark.parametrize("dtype", [DTYPE_F16, DTYPE_BF16])
+def test_strided_batch_with_sixteen_bit_results_on_the_tensor_cores(dtype):
+    # a strided batch whose results are 16-bit as well: one launch of the tensor kernel, every problem's C found by its
+    # byte offset; ragged shapes, C with padded leading dimension and a gap between the problems
+    for (m, n, k), ta, tb, alpha, beta in [((72, 200, 136), "N", "N", 1.0, 0.0), ((130, 70, 264), "T", "N", 1.5, 0.5),
+                                           ((64, 64, 64), "N", "T", -1.0, 1.0)]:
+        batch, gap_c = 40, 5
+        probs, As, Bs, Cs = [], [], [], []
+        for b in range(batch):
+            p = problem(dtype, m, n, k, ta, tb, alpha, beta, "normal", ((-(m if ta == "N" else k)) % 8, (-(k if tb == "N" else n)) % 8, 3), seed=40 + b)
+            A, B, _ = p.operands()
+            probs.append(p); As.append(A); Bs.append(B); Cs.append(c0_16(p, dtype, "normal"))
+        sA, sB, sC = As[0].buf.size, Bs[0].buf.size, Cs[0].buf.size + gap_c
+        assert sA % 8 == 0 and sB % 8 == 0
+        hA = np.concatenate([a.buf for a in As]); hB = np.concatenate([b.buf for b in Bs])
+        hC = np.zeros(sC * batch, dtype=np.uint16)
+        for b in range(batch):
+            hC[b * sC: b * sC + Cs[b].buf.size] = Cs[b].buf
+        dev = lambda x: torch.from_numpy(x.view(np.int16)).cuda()
+        dA, dB, dC = dev(hA), dev(hB), dev(hC)
+        rc = g.gemm_strided_batched(OUT[dtype], ta, tb, m, n, k, alpha, dA.data_ptr(), As[0].ld, sA, dB.data_ptr(), Bs[0].ld, sB,
+                                    beta, dC.data_ptr(), Cs[0].ld, sC, batch, torch.cuda.current_stream().cuda_stream)
+        assert rc == 0, g.gemm_status_string(rc)
+        cfg = g.gemm_last_config()
+        assert cfg["kernel"] == g.GEMM_KERNEL_TENSOR and cfg["launches"] == 1, cfg
+        assert g.gemm_poll_status() == 0, hex(g.gemm_status_detail())
+        out = dC.cpu().numpy().view(np.uint16)
+        for b in range(batch):
+            C = Matrix(out[b * sC: b * sC + Cs[b].buf.size].copy(), m, n, Cs[b].ld, dtype)
+            assert C.padding_intact()
+            assert np.all(out[b * sC + Cs[b].buf.size: (b + 1) * sC] == 0)      # the gap keeps its zeros
+            check(probs[b], dtype, As[b], Bs[b], Cs[b], C)
