@@ -88,14 +88,14 @@ __device__ __noinline__ void cluster_sum_tile(uint32_t park_addr, int S, int64_t
 // OUT: 0 = fp32 result; 1 = 16-bit result (fp32 accumulator, one rounding at the store); 2 = binary16 accumulator
 // and binary16 result (the paper's all-f16 arithmetic, Section III-D); 3 = fp32 result stored transposed (the host
 // exchanged the roles of the operands: C is ldc-strided along the tile's rows and contiguous along its columns)
-template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
+template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT, bool BATCHED>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, int store_via_tma, int64_t m, int64_t n, int64_t k, float alpha, float beta, float* __restrict__ C, int64_t ldc,
                int tiles_m, int tiles_n, int splits, int64_t kchunk, float* __restrict__ partials,
                uint32_t idesc, uint32_t* status, const ConvTma conv, int out16, int cluster_k, int batched,
                int64_t batch_c_bytes) {
-    // batched != 0: a strided batch of problems.  `splits` is then the number of problems and the slab index of a work
+    // BATCHED (then batched != 0): a strided batch of problems.  `splits` is then the number of problems and the slab index of a work
     // item the problem index: tmA and tmB are 3-D maps with the problem as third coordinate (bit 1 / bit 2 of `batched`:
     // A / B is one matrix shared by all problems), every item runs over the whole of k, and problem p's result starts
     // batch_c_bytes * p behind C.
@@ -167,7 +167,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tn = (tile % per_group) / gsz;
     };
     auto kblocks_of = [&](int sp, int64_t& kbeg) {
-        if (batched) { kbeg = 0; return (int)((k + TBK - 1) / TBK); }
+        if (BATCHED) { kbeg = 0; return (int)((k + TBK - 1) / TBK); }
         kbeg = (int64_t)sp * kchunk;
         const int64_t kend = min(k, kbeg + kchunk);
         return (int)((kend - kbeg + TBK - 1) / TBK);
@@ -195,7 +195,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t sb = sa + Cfg::A_BYTES;
                     const int32_t k0 = (int32_t)(kbeg + (int64_t)kb * TBK);
                     mbar_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
-                    if (batched) {
+                    if constexpr (BATCHED) {
                         const int32_t pa = (batched & 2) ? 0 : sp, pb = (batched & 4) ? 0 : sp;
                         if (A_MN) {
 #pragma unroll
@@ -300,9 +300,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                            STATUS_MARK | (ROLE_EPI << 16) | (BAR_TMEM_FULL << 8) | acc)) { ok = false; break; }
             tc_fence_after();
             const int64_t row0 = (int64_t)tm * TBM + q * 32;
-            const bool raw = splits > 1 && !batched;
+            const bool raw = splits > 1 && !BATCHED;
             float* out = raw ? partials + (int64_t)sp * m * n : C;
-            if (batched) out = reinterpret_cast<float*>(reinterpret_cast<char*>(C) + (int64_t)sp * batch_c_bytes);
+            if (BATCHED) out = reinterpret_cast<float*>(reinterpret_cast<char*>(C) + (int64_t)sp * batch_c_bytes);
             // store_via_tma: 0 = direct stores, 1 = tmC maps C (2-D), 2 = tmC maps the split-k partials (3-D: m, n, split)
             const bool via_tma = raw ? (store_via_tma == 2) : (store_via_tma == 1);
             auto release = [&]() {      // the accumulator may be overwritten once this warp has read its last chunk
@@ -602,14 +602,14 @@ uint32_t instr_desc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n, bool 
     return d;
 }
 
-template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT>
+template <int BN, bool A_MN, bool B_MN, bool CONV, int OUT, bool BATCHED = false>
 static cudaError_t launch_tc(const GemmArgs& a, KSplit ks, float* partials, gemm_config_t* cfg,
                              const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmC, int store_via_tma,
                              bool cluster = false, int batched = 0, int64_t batch_c_bytes = 0) {
     using Cfg = TcCfg<BN>;
     // the opt-in to more than 48 KB of dynamic shared memory is per device
     static std::atomic<bool> attr_set[64];      // zero-initialised; set once per device
-    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV, OUT>;
+    auto kern = tc_gemm_kernel<BN, A_MN, B_MN, CONV, OUT, BATCHED>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64 || !attr_set[dev].load()) {
@@ -666,12 +666,12 @@ static cudaError_t launch_tc_batched(const GemmArgs& a, int tile_n, int64_t stri
     const int64_t c_bytes = strideC * (a.out16 ? 2 : 4);
     const KSplit ks{(int)batch, a.k};
     switch (tile_n) {
-        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, false, 1>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
-                                  : launch_tc<256, A_MN, B_MN, false, 0>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
-        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, false, 1>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
-                                  : launch_tc<128, A_MN, B_MN, false, 0>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
-        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, false, 1>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
-                                  : launch_tc<64, A_MN, B_MN, false, 0>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
+        case 256: return a.out16 ? launch_tc<256, A_MN, B_MN, false, 1, true>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
+                                  : launch_tc<256, A_MN, B_MN, false, 0, true>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
+        case 128: return a.out16 ? launch_tc<128, A_MN, B_MN, false, 1, true>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
+                                  : launch_tc<128, A_MN, B_MN, false, 0, true>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
+        default:  return a.out16 ? launch_tc<64, A_MN, B_MN, false, 1, true>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes)
+                                  : launch_tc<64, A_MN, B_MN, false, 0, true>(a, ks, nullptr, cfg, tmA, tmB, tmA, 0, false, flags, c_bytes);
     }
 }
 
