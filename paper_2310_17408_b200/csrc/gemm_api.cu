@@ -893,7 +893,8 @@ int gemm_host(int dtype, char transA, char transB, int64_t m, int64_t n, int64_t
             if (j == 0 && kpanel < k && panel >= 4 * tile && panel < n) col_edge.push_back(round_up(panel / 2, tile));
         }
         col_edge.push_back(n);
-        for (int64_t q = 0; q < (k > 0 ? k : 1); q += kpanel) {
+        const int64_t kstep = kpanel > 0 ? kpanel : 1;      // k = 0: one empty k panel
+        for (int64_t q = 0; q < (k > 0 ? k : 1); q += kstep) {
             k_edge.push_back(q);
             if (q == 0 && kpanel < k && kpanel >= 1024) k_edge.push_back(round_up(kpanel / 2, 256));
         }

@@ -67,8 +67,10 @@ def check_against_oracle(p: Problem, A: Matrix, B: Matrix, C0: Matrix, C: Matrix
         # every partial sum is an exactly representable integer multiple of 0.5: any summation order agrees bitwise
         want = oracle.gemm_l0(p.dtype, p.transA, p.transB, p.m, p.n, p.k, p.alpha, A.buf, A.ld, B.buf, B.ld,
                               p.beta, C0.buf, C0.ld, acc=oracle.ACC_F32)
-        assert np.array_equal(got.view(np.uint32) if got.flags.c_contiguous else np.ascontiguousarray(got).view(np.uint32),
-                              np.ascontiguousarray(want).view(np.uint32)), "integer-valued case is not bit-exact"
+        # compared as values: equal bit for bit except that -0.0 and +0.0 count as equal.  The only place the two sides
+        # can differ in the sign of a zero is the quick return for k = 0 or alpha = 0, where the library forms beta*C0 alone
+        # (the BLAS convention: -2 * 0 = -0) and the definition adds alpha*0 to it (+0); NaN never compares equal.
+        assert np.array_equal(np.ascontiguousarray(got), np.ascontiguousarray(want)), "integer-valued case is not bit-exact"
         return 0.0
     ref = oracle_f64(p, A, B, C0)
     if p.dtype == DTYPE_F32:

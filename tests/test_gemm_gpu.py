@@ -242,7 +242,10 @@ def test_gemm_host_pipelined_panels_match_oracle(dtype):
              (100, 90, 70, "N", "T", -1.0, 1.0, (1, 3, 1)),        # single panel
              (4500, 3000, 2100, "N", "N", 1.0, 0.5, (4, 0, 4)),    # A large enough to arrive in row panels
              (4400, 2900, 2050, "T", "N", 1.0, 0.0, (8, 8, 0)),    # same with A stored transposed
-             (4300, 2800, 2200, "N", "T", 1.5, 0.5, (0, 8, 4))]    # k slices of a transposed B beside A's
+             (4300, 2800, 2200, "N", "T", 1.5, 0.5, (0, 8, 4)),    # k slices of a transposed B beside A's
+             (40, 50, 0, "N", "N", 1.0, 0.5, (0, 0, 2)),           # k = 0: only beta*C
+             (300, 2000, 0, "T", "N", 1.0, 0.0, (0, 0, 0)),        # k = 0, several panels, C overwritten with zeros
+             (64, 1500, 33, "N", "N", 0.0, -2.0, (1, 1, 1))]       # alpha = 0: A and B are not read
     for (m, n, k, ta, tb, alpha, beta, pad) in cases:
         p = problem(dtype, m, n, k, ta, tb, alpha, beta, kind, pad, seed=m)
         A, B, C0 = p.operands()
