@@ -470,7 +470,7 @@ bool make_map_batched(CUtensorMap* tm, int dtype, const void* base, int64_t rows
     if (batch > 1 && (stride <= 0 || stride % 8 != 0)) return false;
     if (batch <= 1) stride = ld * (cols > 0 ? cols : 1);      // a single problem: any legal value
     if (rows > 0xFFFFFFFFLL || cols > 0xFFFFFFFFLL || box_rows > 0xFFFF || box_cols > 0xFFFF) return false;
-    const MapKey k{{4, (uint64_t)dtype | ((uint64_t)box_rows << 16) | ((uint64_t)box_cols << 32), (uint64_t)(uintptr_t)base,
+    const MapKey k{{5, (uint64_t)dtype | ((uint64_t)box_rows << 16) | ((uint64_t)box_cols << 32), (uint64_t)(uintptr_t)base,
                     ((uint64_t)rows << 32) | (uint64_t)cols, (uint64_t)ld, (uint64_t)stride, (uint64_t)batch}};
     return cached_map(tm, k, [&](CUtensorMap* out) {
         cuuint64_t dims[3] = {(cuuint64_t)rows, (cuuint64_t)cols, (cuuint64_t)batch};
