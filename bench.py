@@ -105,7 +105,8 @@ def recorded_traffic(kernel, p):
 
 
 def load_peaks():
-    """Roofline denominators: measured on this machine (MEASURED_PEAKS.json) or the stated fallback."""
+    """Roofline denominators: the measured copy bandwidth and library GEMM throughput of MEASURED_PEAKS.json when that file
+    exists, otherwise the fallback figures stated below."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
@@ -608,7 +609,7 @@ def measure_workload(ctx, problems, operands, workload_name, e2e_steps=None, ste
             "traffic": recorded_traffic(kname, p),
             "kernel": kname, "problem": p.name,
             "peak_source": (f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} lanes x 2 x {peaks['sm_max_mhz']:.0f} MHz (max SM clock)"
-                            if bound == "alu" else f"{peaks['source']} ({'MEASURED_PEAKS.json' if peaks['source'] == 'measured' else 'recipe fallback'})")}
+                            if bound == "alu" else f"{peaks['source']} ({'MEASURED_PEAKS.json' if peaks['source'] == 'measured' else 'fallback figures'})")}
     if bound == "alu" and clocks.get("sm_mhz"):
         roof["frac_at_sampled_clock"] = achieved / fp32_alu_peak_tflops(clocks["sm_mhz"])
     if bound == "tensor":
